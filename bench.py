@@ -1,0 +1,375 @@
+#!/usr/bin/env python
+"""Benchmark of the ROBE-Z hot path on B200.
+
+One step = one pass of the whole path over one batch: robe_forward (hash -> offset -> circular
+block gather -> bag sum-pool) followed by robe_backward (block scatter-add of the output
+gradient with the SGD step fused in).  The default workload is the multi-hot pooled
+configuration whose 1 GB array does not fit in L2 (26 tables, d=64, Z=16, batch 16384, bags of
+about 20 ids).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+prints ONE JSON line.  With N > 1 (launched by torch.distributed.run) every rank runs its own
+batch shard on its own replica of the array (weak scaling, no data-path collective) and rank 0
+reports the aggregate with the time taken as the maximum over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2108_02191_b200 import synth  # noqa: E402
+
+METRIC = "robe_lookups_per_s_fwd_bwd"
+UNIT = "ids/s"
+
+# DRAM bytes per launch of the dominant kernel of the default workload, from the ncu capture
+# summarised under profiles/ (dram__bytes_read.sum + dram__bytes_write.sum); None = not captured.
+NCU_TRAFFIC_BYTES = {
+    "cfg4_multihot": {"forward": None, "backward": None},
+}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+def algorithmic_bytes(w, nbags, nnz, bags):
+    """Bytes the method itself must move per launch (useful-bytes model):
+    forward  = 8 per id (index) + d*s_a per id (array elements read) + 8 per bag (offset, pooled
+               only) + 4d per bag (output row written);
+    backward = 8 per id + 2*4d per id (read-modify-write of the slots) + 8 per bag (pooled only)
+               + 4d per bag (gradient row read once)."""
+    s_a = 4 if w.array_dtype == "f32" else 2
+    off = 8 * (nbags + 1) if bags else 0
+    fwd = 8 * nnz + w.d * s_a * nnz + off + 4 * w.d * nbags
+    bwd = 8 * nnz + 2 * 4 * w.d * nnz + off + 4 * w.d * nbags
+    return fwd, bwd
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
+
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "50",
+                 "-i", str(self.gpu)], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        try:
+            for line in open(self.path):
+                f = [t.strip() for t in line.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1]))
+                    mx.append(float(f[2]))
+                except ValueError:
+                    continue
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown",
+                                      "sw_power_cap"), f[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out["sm_mhz"] = float(np.median(sm))
+            out["sm_max_mhz"] = float(max(mx))
+            out["samples"] = len(sm)
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+def visible_gpu_index(local_rank: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except Exception:
+            return local_rank
+    return local_rank
+
+
+def pick_workload(name: str):
+    table = {
+        "cfg2": synth.workload(2), "cfg3_z1": synth.workload(3, Z=1), "cfg3_z128": synth.workload(3, Z=128),
+        "cfg4": synth.workload(4), "cfg5": synth.workload(5),
+    }
+    return table[name]
+
+
+# -------------------------------------------------------------------------------------------
+# reference arm / cpu baseline: the oracle as it stands, on the host cores
+# -------------------------------------------------------------------------------------------
+
+def oracle_step_rate(w, sample_batch: int, array_h=None, variant=0):
+    """Times oracle forward + fp64 backward on `sample_batch` samples of workload w.
+    Returns (ids per second, ids in the sample, threads used, seconds)."""
+    from oracle import robe_oracle as orc
+    ids, offs = synth.make_ids(w, sample_batch, variant)
+    grad = synth.make_grad_out(w, sample_batch, variant)
+    if array_h is None:
+        array_h = synth.array_to_numpy(synth.make_array(w, "cpu"))
+    o = orc.Oracle(w.M, w.Z, w.d, w.num_tables, orc.hash_constants(w.hash_seed))
+    t0 = time.perf_counter()
+    o.forward(array_h, ids, offs, sample_batch)
+    o.backward_f64(grad, ids, offs, sample_batch)
+    dt = time.perf_counter() - t0
+    return len(ids) / dt, len(ids), orc.num_threads(), dt
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    sample_batch = max(1, w.batch // 16)
+    array_h = synth.array_to_numpy(synth.make_array(w, "cpu"))
+    for i in range(args.warmup):
+        oracle_step_rate(w, sample_batch, array_h, variant=i)
+    total_ids, total_t, threads = 0, 0.0, 1
+    for i in range(args.steps):
+        rate, n, threads, dt = oracle_step_rate(w, sample_batch, array_h, variant=100 + i)
+        total_ids += n
+        total_t += dt
+    value = total_ids / total_t
+    sample = f"{sample_batch} of {w.batch} samples per step (forward + fp64 backward)"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total_t / max(1, args.steps),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic", "config": {"workload": w.name, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+    return 0
+
+
+# -------------------------------------------------------------------------------------------
+# our arm
+# -------------------------------------------------------------------------------------------
+
+def run_ours(args, w):
+    import paper_2108_02191_b200 as robe
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    else:
+        dist = None
+
+    NB = 4  # distinct pre-generated id batches, rotated so ids are never L2-warm
+    bags = w.bag_rule is not None
+    B, T, d = w.batch, w.num_tables, w.d
+    nbags = B * T
+    batches = []
+    for v in range(NB):
+        ids, offs = synth.make_ids(w, B, variant=1000 * rank + v)
+        batches.append((ids, offs))
+    array = synth.make_array(w, dev)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(w.data_seed + 17 * rank)
+    grad_out = torch.randn(B, T, d, device=dev, dtype=torch.float32, generator=gen)
+    out = torch.empty(B, T, d, device=dev, dtype=torch.float32)
+    d_ids = [torch.from_numpy(b[0]).to(dev) for b in batches]
+    d_offs = [None if b[1] is None else torch.from_numpy(b[1]).to(dev) for b in batches]
+
+    h = robe.robe_create(w.M, w.Z, w.d, T, w.hash_seed)
+    robe.robe_attach_array(h, array)
+    lr = 1.0  # the paper trains its DLRM with plain SGD at learning rate 1.0 (Section 5)
+
+    def step(i, events=None):
+        k = i % NB
+        if events is not None:
+            events[0].record()
+        robe.robe_forward(h, d_ids[k], d_offs[k], B, out)
+        if events is not None:
+            events[1].record()
+        robe.robe_backward(h, grad_out, d_ids[k], d_offs[k], B, None, lr, None)
+        if events is not None:
+            events[2].record()
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        step(i)
+    barrier()
+    sampler = ClockSampler(visible_gpu_index(local_rank))
+    sampler.start()
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    barrier()
+    t_start = torch.cuda.Event(enable_timing=True)
+    t_end = torch.cuda.Event(enable_timing=True)
+    t_start.record()
+    for i in range(args.steps):
+        step(args.warmup + i, evs[i])
+    t_end.record()
+    barrier()
+    clocks = sampler.stop()
+    total_ms = t_start.elapsed_time(t_end)
+    fwd_ms = float(np.mean([e[0].elapsed_time(e[1]) for e in evs]))
+    bwd_ms = float(np.mean([e[1].elapsed_time(e[2]) for e in evs]))
+    nnz_per_step = float(np.mean([len(batches[(args.warmup + i) % NB][0]) for i in range(args.steps)]))
+
+    # ---- end to end: host buffers in, result out, every step ------------------------------
+    h_ids = [torch.from_numpy(b[0]).pin_memory() for b in batches]
+    h_offs = [None if b[1] is None else torch.from_numpy(b[1]).pin_memory() for b in batches]
+    h_grad = grad_out.cpu().pin_memory()
+    h_out = torch.empty(B, T, d, dtype=torch.float32).pin_memory()
+    e_ids = torch.empty(max(len(b[0]) for b in batches), dtype=torch.int64, device=dev)
+    e_offs = torch.empty(nbags + 1, dtype=torch.int64, device=dev) if bags else None
+    e_grad = torch.empty_like(grad_out)
+
+    def e2e_step(i):
+        k = i % NB
+        n = h_ids[k].numel()
+        ids_d = e_ids[:n]
+        ids_d.copy_(h_ids[k], non_blocking=True)
+        if bags:
+            e_offs.copy_(h_offs[k], non_blocking=True)
+        e_grad.copy_(h_grad, non_blocking=True)
+        robe.robe_forward(h, ids_d, e_offs, B, out)
+        robe.robe_backward(h, e_grad, ids_d, e_offs, B, None, lr, None)
+        h_out.copy_(out, non_blocking=True)
+
+    e2e_steps = max(3, min(args.steps, 10))
+    for i in range(2):
+        e2e_step(i)
+    barrier()
+    s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    s0.record()
+    for i in range(e2e_steps):
+        e2e_step(i)
+    s1.record()
+    barrier()
+    e2e_ms = s0.elapsed_time(s1)
+    e2e_nnz = float(np.mean([len(batches[i % NB][0]) for i in range(e2e_steps)]))
+    h2d = int(8 * e2e_nnz + (8 * (nbags + 1) if bags else 0) + 4 * nbags * d)
+    d2h = int(4 * nbags * d)
+
+    # ---- max over ranks --------------------------------------------------------------------
+    times = torch.tensor([total_ms, e2e_ms, fwd_ms, bwd_ms], dtype=torch.float64, device=dev)
+    if dist is not None:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    total_ms, e2e_ms, fwd_ms, bwd_ms = [float(v) for v in times.tolist()]
+
+    robe.robe_destroy(h)
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return 0
+
+    peak, peak_kind = measured_peaks()
+    fwd_bytes, bwd_bytes = algorithmic_bytes(w, nbags, nnz_per_step, bags)
+    dominant = "backward" if bwd_ms >= fwd_ms else "forward"
+    dom_bytes, dom_ms = (bwd_bytes, bwd_ms) if dominant == "backward" else (fwd_bytes, fwd_ms)
+    traffic = NCU_TRAFFIC_BYTES.get(w.name, {})
+
+    def roof(nbytes, ms, which):
+        ach = nbytes / (ms * 1e-3) / 1e9
+        return {"kernel": which, "bound": "hbm", "achieved": ach, "peak": peak, "unit": "GB/s",
+                "frac": ach / peak, "peak_kind": f"of {peak_kind}", "traffic": traffic.get(which),
+                "ms_per_launch": ms, "algorithmic_bytes": int(nbytes)}
+
+    value = world * nnz_per_step * args.steps / (total_ms * 1e-3)
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": w.name, "num_tables": T, "d": d, "Z": w.Z, "M": w.M, "batch_per_gpu": B,
+                   "ids_per_step_per_gpu": nnz_per_step, "bags": bags, "backward": "atomic, SGD fused",
+                   "l2": "1 GB array and 4 rotated id batches exceed L2; no flush",
+                   "parallelism": f"dp{world} replicas, no collective"},
+        "clocks": clocks,
+        "e2e": {"value": world * e2e_nnz * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT,
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
+                "ms_per_step": e2e_ms / e2e_steps},
+        "gpu_launches": 2 * args.steps,
+        "roofline": roof(dom_bytes, dom_ms, dominant),
+        "roofline_forward": roof(fwd_bytes, fwd_ms, "forward"),
+        "roofline_backward": roof(bwd_bytes, bwd_ms, "backward"),
+        "forward_only": {"value": world * nnz_per_step / (fwd_ms * 1e-3), "unit": UNIT,
+                         "bags_per_s": world * nbags / (fwd_ms * 1e-3), "ms": fwd_ms},
+    }
+    if not args.no_cpu_baseline and world == 1:
+        sample_batch = max(1, w.batch // 8)
+        rate, n, threads, dt = oracle_step_rate(w, sample_batch, synth.array_to_numpy(array), variant=7)
+        line["cpu_baseline"] = {"value": rate, "unit": UNIT, "cores": threads, "kind": "oracle",
+                                "sample": f"{sample_batch} of {w.batch} samples ({n} ids), forward + "
+                                          f"fp64 backward, {dt:.1f} s"}
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg4", choices=["cfg2", "cfg3_z1", "cfg3_z128", "cfg4", "cfg5"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    w = pick_workload(args.workload)
+    if args.impl == "reference":
+        return run_reference(args, w)
+    return run_ours(args, w)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -1,0 +1,173 @@
+/*
+ * robe.h - C ABI of the B200 (sm_100a) ROBE-Z embedding library.
+ *
+ * ROBE (Random Offset Block Embedding array, arXiv 2108.02191) replaces all
+ * embedding tables of a recommendation model by ONE circular array M of m learned
+ * scalars.  The d-dimensional embedding of token x of table e is assembled from
+ * ceil(d/Z) blocks of Z consecutive array elements; block c starts at the
+ * universal-hash offset h(e,x,c) and wraps around the end of the array
+ * (Section 3.1 "ROBE-D", Section 3.2 "ROBE-Z").  The backward pass adds the
+ * output gradients back into the slots they were read from (Section 3.1,
+ * backward equation).
+ *
+ * Conventions shared by every entry point
+ *   - All sizes are in ELEMENTS unless a name says bytes.
+ *   - "device pointer" = memory of the CUDA device that is current when the call
+ *     is made; "host pointer" = ordinary host memory.  The library never
+ *     allocates or frees device memory, and never synchronises, except where an
+ *     entry point says otherwise.
+ *   - Bags are sample-major.  With T tables and a batch of B samples there are
+ *     B*T bags; bag k = n*T + e belongs to sample n and table e = k mod T and
+ *     covers indices[offsets[k] .. offsets[k+1]).  offsets == NULL means one id
+ *     per bag (one-hot): bag k is indices[k] and nnz must equal B*T.
+ *   - Output / output-gradient element (n, e, i) lives at ((n*T + e)*d + i).
+ *   - Every function returns a robe_status; invalid arguments launch nothing.
+ *     No exception, abort or device trap crosses this boundary.
+ *   - Launches are asynchronous on the given stream (a cudaStream_t passed as
+ *     void*; NULL is the legacy default stream).
+ */
+#ifndef ROBE_H_
+#define ROBE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct robe_ctx* robe_handle_t; /* opaque; host memory owned by the library */
+
+typedef enum {
+    ROBE_OK = 0,
+    ROBE_ERR_INVALID_ARG = -1, /* null pointer, zero size, Z > d, d > M, M + d > 2^32, ... */
+    ROBE_ERR_NO_ARRAY = -2,    /* forward/backward before robe_attach_array            */
+    ROBE_ERR_WORKSPACE = -3,   /* deterministic backward: workspace missing/too small  */
+    ROBE_ERR_CUDA = -4,        /* the CUDA runtime reported an error at launch         */
+    ROBE_ERR_UNSUPPORTED = -5  /* valid request that this build does not implement     */
+} robe_status;
+
+/* array element types */
+#define ROBE_F32 0
+#define ROBE_BF16 1
+
+/* option keys for robe_set_option */
+#define ROBE_OPT_SIGN 1     /* 0 (default) | 1: multiply by the sign hash g(e,x,i)        */
+#define ROBE_OPT_BWD_MODE 2 /* ROBE_BWD_ATOMIC (default) | ROBE_BWD_DETERMINISTIC         */
+#define ROBE_OPT_VALIDATE 3 /* 0 (default) | 1: range-check ids/offsets on the device and
+                               record the first violation in a status word instead of
+                               using the bad value                                        */
+#define ROBE_OPT_FWD_KERNEL 4 /* 0 = automatic (default); other values pick one forward
+                                 kernel variant, for benchmarking only                    */
+#define ROBE_OPT_BWD_KERNEL 5 /* same for the atomic backward                             */
+
+#define ROBE_BWD_ATOMIC 0
+#define ROBE_BWD_DETERMINISTIC 1
+
+/* values of the device status word (robe_last_device_status) */
+#define ROBE_DEV_OK 0
+#define ROBE_DEV_BAD_INDEX 1  /* an id was negative                         */
+#define ROBE_DEV_BAD_OFFSETS 2 /* offsets not monotone or out of [0, nnz]   */
+
+/*
+ * robe_create - make a handle for one ROBE array shape (Section 3.2).
+ *   out         host pointer receiving the handle.
+ *   M           array length m = |M| in elements; 1 <= d <= M and M + d <= 2^32.
+ *   Z           block size, 1 <= Z <= d.  Z = d is ROBE-D (one block per
+ *               embedding, Section 3.1); Z = 1 hashes every element on its own
+ *               (Section 3.3).  If Z does not divide d the last block is short.
+ *   d           embedding dimension (one d per handle; several handles may share
+ *               one array, Section 3.1 "Multiple embedding tables").
+ *   num_tables  T >= 1; the table id e of bag k is k mod T.
+ *   hash_seed   seeds the draw of the hash constants: P = 2^61 - 1 and, from a
+ *               SplitMix64 stream, A_h B_h C_h D_h A_g B_g C_g D_g (61-bit draws,
+ *               redrawn when outside [1,P-1] for multipliers / [0,P-1] for the
+ *               additive terms), as the paper's hash family requires.
+ * Errors: ROBE_ERR_INVALID_ARG.
+ */
+int robe_create(robe_handle_t* out, uint64_t M, uint32_t Z, uint32_t d, uint32_t num_tables,
+                uint64_t hash_seed);
+
+/* robe_destroy - free the host handle.  Device buffers stay the caller's. */
+int robe_destroy(robe_handle_t h);
+
+/* robe_set_option - see the ROBE_OPT_* keys.  ROBE_ERR_INVALID_ARG on a bad key/value. */
+int robe_set_option(robe_handle_t h, int key, int64_t value);
+
+/*
+ * robe_attach_array - name the parameter array M (Section 3: "a single array for
+ * learned parameters" shared by all tables).
+ *   dev_array  device pointer to M elements of `dtype`, 16-byte aligned, owned by the
+ *              caller, read by forward and updated in place by the fused-SGD backward.
+ *   dtype      ROBE_F32 or ROBE_BF16 (bf16 is read-only: widened exactly to fp32).
+ */
+int robe_attach_array(robe_handle_t h, void* dev_array, int dtype);
+
+/*
+ * robe_get_hash_constants - copy out {P, A_h, B_h, C_h, D_h, A_g, B_g, C_g, D_g}
+ * (host pointer to 9 words) so that a checker can be handed numbers, not code.
+ *   h(e,x,c) = ((A_h e + B_h x + C_h c + D_h) mod P) mod M           (Section 3.2)
+ *   g(e,x,i) = 2 (((A_g e + B_g x + C_g i + D_g) mod P) mod 2) - 1   (Section 3.1)
+ */
+int robe_get_hash_constants(robe_handle_t h, uint64_t out[9]);
+
+/*
+ * robe_forward - embedding lookup with optional sum pooling (Section 3.2 forward).
+ *   out[n,e,i] = sum over ids x_p of bag (n,e), in bag order, sequentially in fp32
+ *                (first term initialises), of g(e,x_p,i) * M[(h(e,x_p,i/Z) + i%Z) mod M]
+ *   indices  device pointer, int64 [nnz], ids >= 0.
+ *   offsets  device pointer, int64 [batch*T + 1], offsets[0] = 0, non-decreasing,
+ *            offsets[batch*T] = nnz; or NULL for one-hot (then nnz == batch*T).
+ *   batch    number of samples B >= 0;  nnz >= 0 total ids.
+ *   out      device pointer, fp32 [batch, T, d], fully overwritten; an empty bag gives +0.
+ * Errors: ROBE_ERR_INVALID_ARG, ROBE_ERR_NO_ARRAY, ROBE_ERR_CUDA.
+ */
+int robe_forward(robe_handle_t h, const int64_t* indices, const int64_t* offsets, int64_t batch,
+                 int64_t nnz, float* out, void* stream);
+
+/*
+ * robe_backward_workspace_bytes - bytes of caller-provided device scratch that
+ * robe_backward needs in the handle's current backward mode for a call of this
+ * size (0 in atomic mode).  Returns 0 for a bad handle.
+ */
+size_t robe_backward_workspace_bytes(robe_handle_t h, int64_t batch, int64_t nnz);
+
+/*
+ * robe_backward - scatter-add of the output gradient (Section 3.1 backward equation):
+ *   delta[j] = sum over (p, i) with idx(e, x_p, i) = j of g(e,x_p,i) * grad_out[bag(p), i]
+ * every occurrence of an id contributes, duplicates included.
+ *   grad_out    device pointer, fp32 [batch, T, d].
+ *   grad_array  device pointer, fp32 [M]: delta is ADDED to it (the caller zeroes it
+ *               when a plain gradient is wanted).  NULL selects the fused SGD step
+ *               M[j] <- M[j] - lr * delta[j] applied in place to the attached fp32
+ *               array (the paper trains its DLRM with plain SGD, Section 5).
+ *   lr          learning rate, used only when grad_array == NULL.
+ *   workspace   device pointer to workspace_bytes bytes, 256-byte aligned; may be NULL
+ *               in atomic mode.
+ * Atomic mode adds with red.global (fp32, order not fixed).  Deterministic mode sorts
+ * the blocks by start offset (stable) and lets each array slot sum its terms in that
+ * order in fp32 from +0, then applies ONE add (dense) or ONE fma (SGD) per touched
+ * slot: results are bit-reproducible.
+ * Errors: ROBE_ERR_INVALID_ARG (also: fused SGD on a bf16 array), ROBE_ERR_NO_ARRAY,
+ * ROBE_ERR_WORKSPACE, ROBE_ERR_CUDA.
+ */
+int robe_backward(robe_handle_t h, const float* grad_out, const int64_t* indices,
+                  const int64_t* offsets, int64_t batch, int64_t nnz, float* grad_array, float lr,
+                  void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * robe_set_status_word - give the handle a device int32 (caller-owned, zeroed by the
+ * caller) that kernels write a ROBE_DEV_* code into when ROBE_OPT_VALIDATE is on.
+ * robe_last_device_status - synchronise `stream`, read that word (device-to-host copy)
+ * and return it (>= 0), or a negative robe_status.
+ */
+int robe_set_status_word(robe_handle_t h, int32_t* dev_word);
+int robe_last_device_status(robe_handle_t h, void* stream);
+
+/* robe_status_string - static host string for a robe_status value. */
+const char* robe_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ROBE_H_ */

@@ -1,0 +1,165 @@
+"""Thin ctypes binding of librobe.so: argument marshalling only.
+
+Every function has the name of the C entry point it calls (see include/robe.h) and does
+no arithmetic of the method itself.  torch is used for device memory and streams.  There
+is no fallback: if the shared library is missing or does not load, importing this module
+raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "librobe.so")
+
+ROBE_OK = 0
+ROBE_ERR_INVALID_ARG = -1
+ROBE_ERR_NO_ARRAY = -2
+ROBE_ERR_WORKSPACE = -3
+ROBE_ERR_CUDA = -4
+ROBE_ERR_UNSUPPORTED = -5
+
+ROBE_F32 = 0
+ROBE_BF16 = 1
+
+ROBE_OPT_SIGN = 1
+ROBE_OPT_BWD_MODE = 2
+ROBE_OPT_VALIDATE = 3
+ROBE_OPT_FWD_KERNEL = 4
+ROBE_OPT_BWD_KERNEL = 5
+
+ROBE_BWD_ATOMIC = 0
+ROBE_BWD_DETERMINISTIC = 1
+
+EXPORTS = [
+    "robe_create", "robe_destroy", "robe_set_option", "robe_attach_array",
+    "robe_get_hash_constants", "robe_forward", "robe_backward_workspace_bytes", "robe_backward",
+    "robe_set_status_word", "robe_last_device_status", "robe_status_string",
+]
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        f"{LIB_PATH} is missing: build it with `python -m paper_2108_02191_b200.build` "
+        "(there is no CPU or PyTorch fallback)")
+
+_lib = C.CDLL(LIB_PATH)
+
+_vp, _i64, _u64, _u32 = C.c_void_p, C.c_int64, C.c_uint64, C.c_uint32
+_lib.robe_create.argtypes = [C.POINTER(_vp), _u64, _u32, _u32, _u32, _u64]
+_lib.robe_destroy.argtypes = [_vp]
+_lib.robe_set_option.argtypes = [_vp, C.c_int, _i64]
+_lib.robe_attach_array.argtypes = [_vp, _vp, C.c_int]
+_lib.robe_get_hash_constants.argtypes = [_vp, C.POINTER(_u64)]
+_lib.robe_forward.argtypes = [_vp, _vp, _vp, _i64, _i64, _vp, _vp]
+_lib.robe_backward_workspace_bytes.argtypes = [_vp, _i64, _i64]
+_lib.robe_backward_workspace_bytes.restype = C.c_size_t
+_lib.robe_backward.argtypes = [_vp, _vp, _vp, _vp, _i64, _i64, _vp, C.c_float, _vp, C.c_size_t, _vp]
+_lib.robe_set_status_word.argtypes = [_vp, _vp]
+_lib.robe_last_device_status.argtypes = [_vp, _vp]
+_lib.robe_status_string.argtypes = [C.c_int]
+_lib.robe_status_string.restype = C.c_char_p
+for _name in EXPORTS:
+    if _name not in ("robe_backward_workspace_bytes", "robe_status_string"):
+        getattr(_lib, _name).restype = C.c_int
+
+
+class RobeError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {robe_status_string(status)} ({status})")
+
+
+def _check(status: int, where: str) -> None:
+    if status != ROBE_OK:
+        raise RobeError(status, where)
+
+
+def _dev_ptr(t, dtype=None):
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError("expected a CUDA tensor")
+    if dtype is not None and t.dtype != dtype:
+        raise TypeError(f"expected {dtype}, got {t.dtype}")
+    if not t.is_contiguous():
+        raise ValueError("expected a contiguous tensor")
+    return t.data_ptr()
+
+
+def _stream_ptr(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def robe_status_string(status: int) -> str:
+    return _lib.robe_status_string(status).decode()
+
+
+def robe_create(M: int, Z: int, d: int, num_tables: int, hash_seed: int):
+    h = _vp()
+    if not (0 <= M < 2**64 and 0 <= Z < 2**32 and 0 <= d < 2**32 and 0 <= num_tables < 2**32):
+        raise RobeError(ROBE_ERR_INVALID_ARG, "robe_create")
+    _check(_lib.robe_create(C.byref(h), M, Z, d, num_tables, hash_seed & (2**64 - 1)), "robe_create")
+    return h
+
+
+def robe_destroy(h) -> None:
+    _check(_lib.robe_destroy(h), "robe_destroy")
+
+
+def robe_set_option(h, key: int, value: int) -> None:
+    _check(_lib.robe_set_option(h, key, value), "robe_set_option")
+
+
+def robe_attach_array(h, array: torch.Tensor) -> None:
+    if array.dtype == torch.float32:
+        dt = ROBE_F32
+    elif array.dtype == torch.bfloat16:
+        dt = ROBE_BF16
+    else:
+        raise TypeError("array must be float32 or bfloat16")
+    _check(_lib.robe_attach_array(h, _dev_ptr(array), dt), "robe_attach_array")
+
+
+def robe_get_hash_constants(h):
+    out = (_u64 * 9)()
+    _check(_lib.robe_get_hash_constants(h, out), "robe_get_hash_constants")
+    return [int(v) for v in out]
+
+
+def robe_forward(h, indices, offsets, batch: int, out, stream=None) -> None:
+    _check(_lib.robe_forward(h, _dev_ptr(indices, torch.int64), _dev_ptr(offsets, torch.int64),
+                             batch, indices.numel(), _dev_ptr(out, torch.float32),
+                             _stream_ptr(stream)), "robe_forward")
+
+
+def robe_backward_workspace_bytes(h, batch: int, nnz: int) -> int:
+    return int(_lib.robe_backward_workspace_bytes(h, batch, nnz))
+
+
+def robe_backward(h, grad_out, indices, offsets, batch: int, grad_array=None, lr: float = 0.0,
+                  workspace=None, stream=None) -> None:
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(_lib.robe_backward(h, _dev_ptr(grad_out, torch.float32), _dev_ptr(indices, torch.int64),
+                              _dev_ptr(offsets, torch.int64), batch, indices.numel(),
+                              _dev_ptr(grad_array, torch.float32), lr, _dev_ptr(workspace),
+                              ws_bytes, _stream_ptr(stream)), "robe_backward")
+
+
+def robe_set_status_word(h, word) -> None:
+    _check(_lib.robe_set_status_word(h, _dev_ptr(word, torch.int32)), "robe_set_status_word")
+
+
+def robe_last_device_status(h, stream=None) -> int:
+    return int(_lib.robe_last_device_status(h, _stream_ptr(stream)))
+
+
+# Host-pointer variants of forward/backward calls for callers that drive the C ABI with raw
+# addresses (the benchmark's end-to-end leg uses torch tensors like everything else).
+def raw():
+    """The ctypes library object itself."""
+    return _lib

@@ -1,0 +1,281 @@
+// C ABI of librobe.so: handle, options, argument checks, hash-constant draw, dispatch.
+// The entry points are documented in include/robe.h.
+#include <new>
+
+#include "../../include/robe.h"
+#include "robe_internal.h"
+
+using namespace robe;
+
+struct robe_ctx {
+    uint64_t M;
+    uint32_t Z, d, T;
+    uint64_t consts[9];  // P, A_h, B_h, C_h, D_h, A_g, B_g, C_g, D_g
+    MapParams mp;
+    void* array;
+    int dtype;
+    int sign;
+    int bwd_mode;
+    int validate;
+    int fwd_variant;
+    int bwd_variant;
+    int32_t* status_word;
+};
+
+namespace {
+
+// SplitMix64 (Steele, Lea, Flood): the stream the hash constants are drawn from.
+uint64_t splitmix_next(uint64_t& s) {
+    s += 0x9E3779B97F4A7C15ull;
+    uint64_t z = s;
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    return z ^ (z >> 31);
+}
+
+// Section 3.2: A_h, B_h, C_h in {1..P-1}, D_h in {0..P-1}; same ranges for the sign hash.
+void draw_constants(uint64_t seed, uint64_t out[9]) {
+    uint64_t s = seed;
+    out[0] = kP61;
+    for (int k = 1; k <= 8; ++k) {
+        const bool additive = (k == 4 || k == 8);
+        uint64_t v;
+        do {
+            v = splitmix_next(s) >> 3;
+        } while (v >= kP61 || (!additive && v == 0));
+        out[k] = v;
+    }
+}
+
+__global__ void validate_kernel(const int64_t* indices, const int64_t* offsets, int64_t nbags,
+                                int64_t nnz, int32_t* status) {
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t < nnz && indices[t] < 0) atomicCAS(status, ROBE_DEV_OK, ROBE_DEV_BAD_INDEX);
+    if (offsets != nullptr && t <= nbags) {
+        const int64_t o = offsets[t];
+        bool bad = o < 0 || o > nnz;
+        if (t == 0 && o != 0) bad = true;
+        if (t == nbags && o != nnz) bad = true;
+        if (t < nbags && offsets[t + 1] < o) bad = true;
+        if (bad) atomicCAS(status, ROBE_DEV_OK, ROBE_DEV_BAD_OFFSETS);
+    }
+}
+
+bool check_sizes(robe_ctx* h, const int64_t* indices, const int64_t* offsets, int64_t batch,
+                 int64_t nnz) {
+    if (h == nullptr || batch < 0 || nnz < 0) return false;
+    if (nnz > 0 && indices == nullptr) return false;
+    const int64_t nbags = batch * (int64_t)h->T;
+    if (batch != 0 && nbags / batch != (int64_t)h->T) return false;  // overflow
+    if (offsets == nullptr && nnz != nbags) return false;
+    return true;
+}
+
+Problem make_problem(robe_ctx* h, const int64_t* indices, const int64_t* offsets, int64_t batch,
+                     int64_t nnz) {
+    Problem pb;
+    pb.mp = h->mp;
+    pb.array = h->array;
+    pb.dtype = h->dtype;
+    pb.sign = h->sign;
+    pb.indices = indices;
+    pb.offsets = offsets;
+    pb.nbags = batch * (int64_t)h->T;
+    pb.nnz = nnz;
+    pb.status = (h->validate && h->status_word) ? h->status_word : nullptr;
+    return pb;
+}
+
+}  // namespace
+
+namespace robe {
+cudaError_t launch_validate(const Problem& pb, cudaStream_t st) {
+    if (pb.status == nullptr) return cudaSuccess;
+    const int64_t n = (pb.nnz > pb.nbags + 1 ? pb.nnz : pb.nbags + 1);
+    validate_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(pb.indices, pb.offsets, pb.nbags,
+                                                                 pb.nnz, pb.status);
+    return cudaGetLastError();
+}
+}  // namespace robe
+
+extern "C" {
+
+int robe_create(robe_handle_t* out, uint64_t M, uint32_t Z, uint32_t d, uint32_t num_tables,
+                uint64_t hash_seed) {
+    if (out == nullptr) return ROBE_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (M == 0 || Z == 0 || d == 0 || num_tables == 0) return ROBE_ERR_INVALID_ARG;
+    if (Z > d || (uint64_t)d > M) return ROBE_ERR_INVALID_ARG;
+    if (d > 32768u) return ROBE_ERR_INVALID_ARG;
+    if (M + (uint64_t)d > (1ull << 32)) return ROBE_ERR_INVALID_ARG;
+    robe_ctx* h = new (std::nothrow) robe_ctx();
+    if (h == nullptr) return ROBE_ERR_INVALID_ARG;
+    h->M = M;
+    h->Z = Z;
+    h->d = d;
+    h->T = num_tables;
+    draw_constants(hash_seed, h->consts);
+    MapParams& mp = h->mp;
+    mp.h = HashConsts{h->consts[1], h->consts[2], h->consts[3], h->consts[4]};
+    mp.g = HashConsts{h->consts[5], h->consts[6], h->consts[7], h->consts[8]};
+    mp.m = (uint32_t)M;
+    mp.mu = (M == 1) ? ~0ull : (uint64_t)((((unsigned __int128)1) << 64) / M);
+    mp.T = num_tables;
+    mp.d = d;
+    mp.Z = Z;
+    mp.C = (d + Z - 1) / Z;
+    mp.log2Z = 0xFFFFFFFFu;
+    if ((Z & (Z - 1)) == 0) {
+        uint32_t l = 0;
+        while ((1u << l) < Z) ++l;
+        mp.log2Z = l;
+    }
+    mp.tmagic = 0xFFFFFFFFFFFFFFFFull / num_tables + 1;
+    h->array = nullptr;
+    h->dtype = ROBE_F32;
+    h->sign = 0;
+    h->bwd_mode = ROBE_BWD_ATOMIC;
+    h->validate = 0;
+    h->fwd_variant = 0;
+    h->bwd_variant = 0;
+    h->status_word = nullptr;
+    *out = h;
+    return ROBE_OK;
+}
+
+int robe_destroy(robe_handle_t h) {
+    if (h == nullptr) return ROBE_ERR_INVALID_ARG;
+    delete h;
+    return ROBE_OK;
+}
+
+int robe_set_option(robe_handle_t h, int key, int64_t value) {
+    if (h == nullptr) return ROBE_ERR_INVALID_ARG;
+    switch (key) {
+        case ROBE_OPT_SIGN:
+            if (value != 0 && value != 1) return ROBE_ERR_INVALID_ARG;
+            h->sign = (int)value;
+            return ROBE_OK;
+        case ROBE_OPT_BWD_MODE:
+            if (value != ROBE_BWD_ATOMIC && value != ROBE_BWD_DETERMINISTIC)
+                return ROBE_ERR_INVALID_ARG;
+            h->bwd_mode = (int)value;
+            return ROBE_OK;
+        case ROBE_OPT_VALIDATE:
+            if (value != 0 && value != 1) return ROBE_ERR_INVALID_ARG;
+            h->validate = (int)value;
+            return ROBE_OK;
+        case ROBE_OPT_FWD_KERNEL:
+            if (value < 0 || value > 2) return ROBE_ERR_INVALID_ARG;
+            h->fwd_variant = (int)value;
+            return ROBE_OK;
+        case ROBE_OPT_BWD_KERNEL:
+            if (value < 0 || value > 2) return ROBE_ERR_INVALID_ARG;
+            h->bwd_variant = (int)value;
+            return ROBE_OK;
+        default:
+            return ROBE_ERR_INVALID_ARG;
+    }
+}
+
+int robe_attach_array(robe_handle_t h, void* dev_array, int dtype) {
+    if (h == nullptr || dev_array == nullptr) return ROBE_ERR_INVALID_ARG;
+    if (dtype != ROBE_F32 && dtype != ROBE_BF16) return ROBE_ERR_INVALID_ARG;
+    if (((uintptr_t)dev_array & 15u) != 0) return ROBE_ERR_INVALID_ARG;
+    h->array = dev_array;
+    h->dtype = dtype;
+    return ROBE_OK;
+}
+
+int robe_get_hash_constants(robe_handle_t h, uint64_t out[9]) {
+    if (h == nullptr || out == nullptr) return ROBE_ERR_INVALID_ARG;
+    for (int k = 0; k < 9; ++k) out[k] = h->consts[k];
+    return ROBE_OK;
+}
+
+int robe_set_status_word(robe_handle_t h, int32_t* dev_word) {
+    if (h == nullptr) return ROBE_ERR_INVALID_ARG;
+    h->status_word = dev_word;
+    return ROBE_OK;
+}
+
+int robe_last_device_status(robe_handle_t h, void* stream) {
+    if (h == nullptr || h->status_word == nullptr) return ROBE_ERR_INVALID_ARG;
+    int32_t v = 0;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (cudaMemcpyAsync(&v, h->status_word, sizeof v, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return ROBE_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return ROBE_ERR_CUDA;
+    return (int)v;
+}
+
+int robe_forward(robe_handle_t h, const int64_t* indices, const int64_t* offsets, int64_t batch,
+                 int64_t nnz, float* out, void* stream) {
+    if (!check_sizes(h, indices, offsets, batch, nnz)) return ROBE_ERR_INVALID_ARG;
+    if (batch > 0 && out == nullptr) return ROBE_ERR_INVALID_ARG;
+    if (h->array == nullptr) return ROBE_ERR_NO_ARRAY;
+    if (h->validate && h->status_word == nullptr) return ROBE_ERR_INVALID_ARG;
+    const Problem pb = make_problem(h, indices, offsets, batch, nnz);
+    cudaStream_t st = (cudaStream_t)stream;
+    if (launch_validate(pb, st) != cudaSuccess) return ROBE_ERR_CUDA;
+    if (launch_forward(pb, out, h->fwd_variant, st) != cudaSuccess) return ROBE_ERR_CUDA;
+    return ROBE_OK;
+}
+
+size_t robe_backward_workspace_bytes(robe_handle_t h, int64_t batch, int64_t nnz) {
+    if (h == nullptr || batch < 0 || nnz < 0) return 0;
+    if (h->bwd_mode != ROBE_BWD_DETERMINISTIC) return 0;
+    // the pooled layout is the larger of the two; a caller may size once for both
+    return det_workspace_bytes(h->mp, batch * (int64_t)h->T, nnz, true);
+}
+
+int robe_backward(robe_handle_t h, const float* grad_out, const int64_t* indices,
+                  const int64_t* offsets, int64_t batch, int64_t nnz, float* grad_array, float lr,
+                  void* workspace, size_t workspace_bytes, void* stream) {
+    if (!check_sizes(h, indices, offsets, batch, nnz)) return ROBE_ERR_INVALID_ARG;
+    if (batch > 0 && grad_out == nullptr) return ROBE_ERR_INVALID_ARG;
+    if (h->validate && h->status_word == nullptr) return ROBE_ERR_INVALID_ARG;
+    const bool sgd = grad_array == nullptr;
+    if (sgd) {
+        if (h->array == nullptr) return ROBE_ERR_NO_ARRAY;
+        if (h->dtype != ROBE_F32) return ROBE_ERR_INVALID_ARG;
+    }
+    float* target = sgd ? (float*)h->array : grad_array;
+    const Problem pb = make_problem(h, indices, offsets, batch, nnz);
+    cudaStream_t st = (cudaStream_t)stream;
+    if (h->bwd_mode == ROBE_BWD_ATOMIC) {
+        if (launch_validate(pb, st) != cudaSuccess) return ROBE_ERR_CUDA;
+        if (launch_backward_atomic(pb, grad_out, target, sgd ? -lr : 1.0f, h->bwd_variant, st) !=
+            cudaSuccess)
+            return ROBE_ERR_CUDA;
+        return ROBE_OK;
+    }
+    // deterministic: 32-bit block numbers and a grid of one thread per (block, offset)
+    const uint64_t nb = (uint64_t)nnz * h->mp.C;
+    uint32_t zp = 1;
+    while (zp < h->mp.Z) zp <<= 1;
+    if (nb >= (1ull << 32) || (uint64_t)pb.nbags >= (1ull << 32)) return ROBE_ERR_UNSUPPORTED;
+    if (nb * zp / 256 >= (1ull << 31)) return ROBE_ERR_UNSUPPORTED;
+    const size_t need = det_workspace_bytes(h->mp, pb.nbags, nnz, offsets != nullptr);
+    if (nnz > 0 && (workspace == nullptr || workspace_bytes < need)) return ROBE_ERR_WORKSPACE;
+    if (((uintptr_t)workspace & 255u) != 0) return ROBE_ERR_WORKSPACE;
+    if (launch_validate(pb, st) != cudaSuccess) return ROBE_ERR_CUDA;
+    if (launch_backward_det(pb, grad_out, target, sgd ? 1 : 0, lr, workspace, workspace_bytes,
+                            st) != cudaSuccess)
+        return ROBE_ERR_CUDA;
+    return ROBE_OK;
+}
+
+const char* robe_status_string(int status) {
+    switch (status) {
+        case ROBE_OK: return "ok";
+        case ROBE_ERR_INVALID_ARG: return "invalid argument";
+        case ROBE_ERR_NO_ARRAY: return "no array attached";
+        case ROBE_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case ROBE_ERR_CUDA: return "CUDA runtime error at launch";
+        case ROBE_ERR_UNSUPPORTED: return "size not supported by this build";
+        default: return "unknown status";
+    }
+}
+
+}  // extern "C"

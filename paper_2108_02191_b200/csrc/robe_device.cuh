@@ -1,0 +1,124 @@
+// Device-side integer arithmetic of the ROBE-Z location mapping (Section 3.2:
+// h(e,x,c) = ((A e + B x + C c + D) mod P) mod m, idx = (h + i mod Z) mod m) and of the
+// optional sign hash (Section 3.1, g equation), for P = 2^61 - 1 and m < 2^32.
+//
+// Everything here is exact integer work, restructured for 32-bit integer ALUs:
+//   * a product with a 61-bit constant is a 64x64->128 multiply folded with
+//     2^61 = 1 (mod P);
+//   * the per-(table,id) part of the sum is reduced once and the per-chunk part
+//     C*c mod P is added afterwards (sums of residues, then one conditional subtract);
+//   * "mod m" is a Barrett reduction with mu = floor(2^64 / m) and one correction.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace robe {
+
+constexpr uint64_t kP61 = (1ull << 61) - 1ull;
+
+struct HashConsts {  // all < P
+    uint64_t A, B, C, D;
+};
+
+// Everything a kernel needs to map (e, x, c) to a block start.
+struct MapParams {
+    HashConsts h;      // location hash
+    HashConsts g;      // sign hash
+    uint64_t mu;       // floor(2^64 / m)  (2^64 - 1 when m == 1)
+    uint32_t m;        // array length (m + d <= 2^32)
+    uint32_t T;        // number of tables
+    uint32_t d;        // embedding dimension
+    uint32_t Z;        // block size
+    uint32_t C;        // chunks per embedding = ceil(d / Z)
+    uint32_t log2Z;    // valid when Z is a power of two, else 0xFFFFFFFF
+    uint64_t tmagic;   // floor((2^64 - 1) / T) + 1, for k mod T with k < 2^32
+};
+
+// (hi * 2^64 + lo) mod P for hi < 2^61.
+__device__ __forceinline__ uint64_t fold_p61(uint64_t hi, uint64_t lo) {
+    uint64_t v0 = lo & kP61;
+    uint64_t v1 = ((lo >> 61) | (hi << 3)) & kP61;
+    uint64_t v2 = hi >> 58;
+    uint64_t s = v0 + v1 + v2;       // < 2^62 + 2^6
+    s = (s & kP61) + (s >> 61);      // <= P + 2
+    return s >= kP61 ? s - kP61 : s;
+}
+
+// (a * b) mod P, a < P, b any 64-bit value.
+__device__ __forceinline__ uint64_t mulmod_p61(uint64_t a, uint64_t b) {
+    return fold_p61(__umul64hi(a, b), a * b);
+}
+
+// (a * b) mod P, a < P, b < 2^32: the product has at most 93 bits.
+__device__ __forceinline__ uint64_t mulmod_p61_u32(uint64_t a, uint32_t b) {
+    uint64_t lo = (a & 0xFFFFFFFFull) * b;   // < 2^64
+    uint64_t hi = (a >> 32) * b;             // < 2^61, weight 2^32
+    // value = hi * 2^32 + lo ; split hi * 2^32 into 61-bit limbs
+    uint64_t w0 = (hi << 32) & kP61;         // low 29 bits of hi, shifted
+    uint64_t w1 = hi >> 29;                  // weight 2^61 = 1
+    uint64_t s = (lo & kP61) + (lo >> 61) + w0 + w1;  // < 2^63
+    s = (s & kP61) + (s >> 61);
+    return s >= kP61 ? s - kP61 : s;
+}
+
+__device__ __forceinline__ uint64_t addmod_p61(uint64_t a, uint64_t b) {  // a, b < P
+    uint64_t s = a + b;
+    return s >= kP61 ? s - kP61 : s;
+}
+
+// t mod m for t < 2^64, m < 2^32 (mu = floor(2^64/m)): the quotient estimate is at most
+// one too small, so one conditional subtract finishes it.
+__device__ __forceinline__ uint32_t mod_m(uint64_t t, uint32_t m, uint64_t mu) {
+    uint64_t q = __umul64hi(t, mu);
+    uint64_t r = t - q * m;
+    return (uint32_t)(r >= m ? r - m : r);
+}
+
+// k mod T for k < 2^32 (Lemire's fastmod with a 64-bit magic number).
+__device__ __forceinline__ uint32_t table_of_bag(uint64_t k, const MapParams& mp) {
+    if (k >> 32) return (uint32_t)(k % mp.T);
+    uint64_t low = mp.tmagic * (uint32_t)k;
+    return (uint32_t)__umul64hi(low, (uint64_t)mp.T);
+}
+
+// (A e + B x + D) mod P : the part of the hash argument shared by all chunks of one id.
+__device__ __forceinline__ uint64_t hash_base(const HashConsts& k, uint32_t e, uint64_t x) {
+    uint64_t s = mulmod_p61_u32(k.A, e) + mulmod_p61(k.B, x) + k.D;  // < 3P < 2^63
+    s = (s & kP61) + (s >> 61);
+    return s >= kP61 ? s - kP61 : s;
+}
+
+// Block start h(e,x,c) given the base of (e,x).
+__device__ __forceinline__ uint32_t block_start(const MapParams& mp, uint64_t base, uint32_t c) {
+    uint64_t t = addmod_p61(base, mulmod_p61_u32(mp.h.C, c));
+    return mod_m(t, mp.m, mp.mu);
+}
+
+// Sign g(e,x,i) as +1.0f / -1.0f given the sign-hash base of (e,x).
+__device__ __forceinline__ float sign_of(const MapParams& mp, uint64_t gbase, uint32_t i) {
+    uint64_t t = addmod_p61(gbase, mulmod_p61_u32(mp.g.C, i));
+    return (t & 1ull) ? 1.0f : -1.0f;
+}
+
+// chunk id and in-chunk offset of element i
+__device__ __forceinline__ void chunk_of(const MapParams& mp, uint32_t i, uint32_t& c, uint32_t& o) {
+    if (mp.log2Z != 0xFFFFFFFFu) {
+        c = i >> mp.log2Z;
+        o = i & (mp.Z - 1);
+    } else {
+        c = i / mp.Z;
+        o = i - c * mp.Z;
+    }
+}
+
+__device__ __forceinline__ float bf16_bits_to_float(uint16_t b) {
+    return __uint_as_float((uint32_t)b << 16);
+}
+
+template <int DT>
+__device__ __forceinline__ float load_elem(const void* array, uint32_t j) {
+    if (DT == 0) return __ldg((const float*)array + j);
+    return bf16_bits_to_float(__ldg((const unsigned short*)array + j));
+}
+
+}  // namespace robe

@@ -1,0 +1,39 @@
+// Host-side declarations shared by the translation units of librobe.so.
+#pragma once
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "robe_device.cuh"
+
+namespace robe {
+
+struct Problem {
+    MapParams mp;
+    const void* array;       // device, M elements
+    int dtype;               // 0 fp32, 1 bf16
+    int sign;                // 0 / 1
+    const int64_t* indices;  // device [nnz]
+    const int64_t* offsets;  // device [nbags+1] or nullptr (one-hot)
+    int64_t nbags;           // batch * T
+    int64_t nnz;
+    int32_t* status;         // device status word or nullptr (validation off)
+};
+
+// forward: out [nbags, d]
+cudaError_t launch_forward(const Problem& pb, float* out, int variant, cudaStream_t st);
+
+// atomic backward: adds scale * g * grad_out into target (fp32 [M])
+cudaError_t launch_backward_atomic(const Problem& pb, const float* grad_out, float* target,
+                                   float scale, int variant, cudaStream_t st);
+
+// deterministic backward
+size_t det_workspace_bytes(const MapParams& mp, int64_t nbags, int64_t nnz, bool bags);
+// sgd != 0: target = attached array, target[j] = fma(-lr, delta, target[j]); else target[j] += delta
+cudaError_t launch_backward_det(const Problem& pb, const float* grad_out, float* target, int sgd,
+                                float lr, void* workspace, size_t workspace_bytes, cudaStream_t st);
+
+// id / offset range check into the status word
+cudaError_t launch_validate(const Problem& pb, cudaStream_t st);
+
+}  // namespace robe

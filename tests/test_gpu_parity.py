@@ -1,0 +1,413 @@
+"""Parity of the CUDA library (called through its C ABI binding) with the CPU oracle.
+
+Bars: forward bit-exact; atomic backward within 1e-5 of the per-slot L1 gradient mass;
+deterministic backward bit-exact with the oracle's canonical-order fp32 gradient."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2108_02191_b200 as robe
+from oracle import robe_oracle as orc
+from paper_2108_02191_b200 import synth
+from robe_testlib import Case, assert_bits_equal, assert_within_l1
+
+pytestmark = pytest.mark.gpu
+
+FWD_KERNELS = [0, 1, 2]  # automatic, direct, warp
+
+
+def small(**kw):
+    """A small workload that still spans several CTAs and a ragged tail."""
+    base = dict(name="small", num_tables=3, vocab_rule="list", vocab_arg=(50, 7, 1000), d=16, Z=4,
+                M=1000, batch=333, array_init="normal0.01", array_dtype="f32", id_dist="uniform",
+                bag_rule=None, hash_seed=77, data_seed=5)
+    base.update(kw)
+    return synth.RobeWorkload(**base)
+
+
+# ---------------------------------------------------------------------------------------
+# forward
+# ---------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("sign", [False, True])
+@pytest.mark.parametrize("kernel", FWD_KERNELS)
+def test_cfg1_forward(kernel, sign):
+    with Case(synth.workload(1), sign=sign) as c:
+        assert_bits_equal(c.forward(kernel).cpu().numpy(), c.oracle_forward(), "cfg1 forward")
+
+
+SHAPES = [
+    # (d, Z, M) - powers of two, ragged, Z not dividing d, tiny arrays that wrap all the time
+    (16, 4, 1000), (16, 16, 17), (16, 4, 17), (16, 1, 16), (1, 1, 1), (1, 1, 5), (2, 2, 3),
+    (128, 1, 4099), (128, 2, 4099), (128, 8, 4099), (128, 32, 129), (128, 128, 128),
+    (128, 128, 100003), (64, 16, 70), (100, 32, 1013), (96, 64, 1013), (33, 1, 64), (7, 2, 9),
+    (12, 5, 64), (48, 3, 49), (130, 2, 1000), (200, 64, 777), (256, 1, 513), (37, 37, 37),
+]
+
+
+@pytest.mark.parametrize("bags", [None, (3, 0, 9)])
+@pytest.mark.parametrize("d,Z,M", SHAPES)
+def test_forward_shapes(d, Z, M, bags):
+    w = small(d=d, Z=Z, M=M, bag_rule=bags, batch=97)
+    for sign in (False, True):
+        with Case(w, sign=sign) as c:
+            want = c.oracle_forward()
+            warp_ok = (Z & (Z - 1)) == 0 and d <= 128
+            for kernel in ([0, 1, 2] if warp_ok else [0, 1]):
+                assert_bits_equal(c.forward(kernel).cpu().numpy(), want, f"d={d} Z={Z} M={M} k={kernel}")
+            if not warp_ok:
+                with pytest.raises(robe.RobeError):
+                    c.forward(2)
+
+
+def test_forward_bf16_array():
+    w = small(array_dtype="bf16", d=64, Z=16, M=5000, bag_rule=(4, 0, 12))
+    with Case(w) as c:
+        want = c.oracle_forward()
+        for kernel in FWD_KERNELS:
+            assert_bits_equal(c.forward(kernel).cpu().numpy(), want, "bf16")
+
+
+def test_forward_empty_and_degenerate_inputs():
+    w = small(bag_rule=(2, 0, 5))
+    with Case(w, batch=4) as c:
+        # all bags empty
+        c.offsets = torch.zeros(c.nbags + 1, dtype=torch.int64, device=c.dev)
+        c.indices = torch.zeros(0, dtype=torch.int64, device=c.dev)
+        out = c.forward().cpu().numpy()
+        assert np.all(out == 0) and not np.any(np.signbit(out))
+    with Case(small(), batch=1) as c:
+        assert_bits_equal(c.forward().cpu().numpy(), c.oracle_forward(), "batch 1")
+    with Case(small()) as c:
+        # batch 0 launches nothing and succeeds
+        out = torch.empty(0, c.T, c.w.d, device=c.dev)
+        robe.robe_forward(c.h, torch.zeros(0, dtype=torch.int64, device=c.dev), None, 0, out)
+
+
+def test_forward_huge_ids_and_negative_zero():
+    # ids up to 2^63-1 go through the full 128-bit product; -0.0 in the array must survive
+    # (the first term initialises the sum: +0 + -0 would turn it into +0)
+    w = small(d=8, Z=4, M=64, num_tables=1, vocab_arg=(10,), bag_rule=(2, 1, 3))
+    ids = np.array([2**63 - 1, 2**62 + 12345, (1 << 61) - 1, 1 << 61, 5, 5, 2**40 + 1], dtype=np.int64)
+    offsets = np.array([0, 1, 2, 3, 4, 6, 7], dtype=np.int64)
+    arr = torch.full((64,), -0.0, dtype=torch.float32)
+    with Case(w, batch=6, ids=(ids, offsets), array=arr) as c:
+        got = c.forward().cpu().numpy()
+        want = c.oracle_forward()
+        assert_bits_equal(got, want, "huge ids / -0")
+        assert np.all(np.signbit(got))
+
+
+def test_forward_max_array_size():
+    # M + d = 2^32: block starts near 2^32 must not overflow 32-bit slot arithmetic.  The array
+    # (bf16, 8.6 GB) is filled on the device by the counter-based generator; the oracle side
+    # evaluates the same generator only at the slots it needs.
+    d, Z = 128, 128
+    M = (1 << 32) - d
+    w = synth.workload(5, M=M, Z=Z, array_dtype="bf16", batch=64)
+    free, _ = torch.cuda.mem_get_info()
+    if free < 12 * 2**30:
+        pytest.skip("not enough free device memory")
+    with Case(w, host_array=False) as c:
+        got = c.forward().cpu().numpy().reshape(c.nbags, d)
+        near_end = 0
+        for bag in range(0, c.nbags, 7):
+            slots = c.oracle.locate(bag % c.T, int(c.indices_h[bag])).astype(np.int64)
+            near_end += int(slots.max() > (1 << 32) - 4 * d)
+            want = synth.array_values_at(w, torch.from_numpy(slots)).to(torch.bfloat16).to(torch.float32)
+            assert_bits_equal(got[bag], want.numpy(), "max M")
+    # force blocks that wrap around the very end: solve B*x = v - D - A*e (mod P) for a start v
+    # within d of M (Python integers; the library only hands out its constants)
+    with Case(w.with_(batch=1), host_array=False) as c:
+        P_, A_, B_, _, D_ = [int(v) for v in robe.robe_get_hash_constants(c.h)[:5]]
+        starts = [M - 1, M - 5, M - d + 1, M - 64]
+        found = [((v - D_) * pow(B_, -1, P_)) % P_ for v in starts]
+        ids = np.zeros((len(found), c.T), dtype=np.int64)
+        ids[:, 0] = found
+        c.B, c.nbags = len(found), len(found) * c.T
+        c.indices_h = ids.reshape(-1)
+        c.indices = torch.from_numpy(c.indices_h).to(c.dev)
+        got = c.forward().cpu().numpy()
+        for r, (xx, v) in enumerate(zip(found, starts)):
+            assert c.oracle.h(0, int(xx), 0) == v
+            slots = c.oracle.locate(0, int(xx)).astype(np.int64)
+            assert slots.max() == M - 1 and slots.min() == 0
+            want = synth.array_values_at(w, torch.from_numpy(slots)).to(torch.bfloat16).to(torch.float32)
+            assert_bits_equal(got[r, 0], want.numpy(), "wrap at 2^32")
+
+
+# ---------------------------------------------------------------------------------------
+# backward, small shapes: all modes
+# ---------------------------------------------------------------------------------------
+
+def _grad(c, seed=0, integer=False):
+    rng = np.random.default_rng(seed)
+    if integer:
+        g = rng.integers(-4, 5, size=(c.B, c.T, c.w.d)).astype(np.float32)
+    else:
+        g = rng.standard_normal((c.B, c.T, c.w.d), dtype=np.float32)
+    return g, torch.from_numpy(g).to(c.dev)
+
+
+BWD_SHAPES = [
+    (16, 4, 4096), (16, 16, 17), (16, 4, 17), (1, 1, 1), (2, 2, 3), (128, 1, 4099), (128, 8, 4099),
+    (128, 32, 129), (128, 128, 128), (64, 16, 70), (100, 32, 1013), (12, 5, 64), (48, 3, 49),
+    (130, 2, 1000), (200, 64, 777), (37, 37, 37), (16, 8, 5000),
+]
+
+
+@pytest.mark.parametrize("bags", [None, (3, 0, 9)])
+@pytest.mark.parametrize("d,Z,M", BWD_SHAPES)
+def test_backward_shapes(d, Z, M, bags):
+    w = small(d=d, Z=Z, M=M, bag_rule=bags, batch=61)
+    for sign in (False, True):
+        with Case(w, sign=sign) as c:
+            g_h, g_d = _grad(c, 1)
+            delta64, l1 = c.oracle.backward_f64(g_h, c.indices_h, c.offsets_h, c.B)
+            can, touched = c.oracle.backward_canonical(g_h, c.indices_h, c.offsets_h, c.B)
+            warp_ok = (Z & (Z - 1)) == 0 and d <= 128
+            for kernel in ([0, 1, 2] if warp_ok else [0, 1]):
+                ga = c.backward(g_d, "atomic", kernel=kernel).cpu().numpy()
+                assert_within_l1(ga, delta64, l1, what=f"atomic d={d} Z={Z} M={M} k={kernel}")
+            det = c.backward(g_d, "det").cpu().numpy()
+            assert_bits_equal(det, can, f"deterministic d={d} Z={Z} M={M} sign={sign}")
+            # integer gradients: every order gives the same bits, so atomic == canonical == fp64
+            gi_h, gi_d = _grad(c, 2, integer=True)
+            di, _ = c.oracle.backward_f64(gi_h, c.indices_h, c.offsets_h, c.B)
+            assert_bits_equal(c.backward(gi_d, "atomic").cpu().numpy(), di.astype(np.float32), "int atomic")
+            assert_bits_equal(c.backward(gi_d, "det").cpu().numpy(), di.astype(np.float32), "int det")
+
+
+@pytest.mark.parametrize("mode", ["atomic", "det"])
+def test_cfg1_backward_dense_and_sgd(mode):
+    for sign in (False, True):
+        with Case(synth.workload(1), sign=sign) as c:
+            g_h = synth.make_grad_out(c.w)
+            g_d = torch.from_numpy(g_h).to(c.dev)
+            delta64, l1 = c.oracle.backward_f64(g_h, c.indices_h, c.offsets_h, c.B)
+            can, touched = c.oracle.backward_canonical(g_h, c.indices_h, c.offsets_h, c.B)
+            ga = c.backward(g_d, mode).cpu().numpy()
+            if mode == "atomic":
+                assert_within_l1(ga, delta64, l1, what="cfg1 atomic")
+            else:
+                assert_bits_equal(ga, can, "cfg1 det")
+            # accumulation into a non-zero gradient array
+            pre = torch.from_numpy(np.random.default_rng(3).standard_normal(c.w.M).astype(np.float32))
+            ga2 = c.backward(g_d, mode, grad_array=pre.to(c.dev).clone()).cpu().numpy()
+            if mode == "det":
+                want = pre.numpy().copy()
+                orc.accumulate(want, can, touched)
+                assert_bits_equal(ga2, want, "cfg1 det accumulate")
+            else:
+                assert_within_l1(ga2 - pre.numpy(), delta64, l1 + np.abs(pre.numpy()), what="cfg1 atomic acc")
+            # fused SGD step
+            lr = 0.5
+            before = c.array_h.copy()
+            c.backward(g_d, mode, sgd=True, lr=lr)
+            after = c.array.cpu().numpy()
+            if mode == "det":
+                want = before.copy()
+                orc.sgd_apply(want, can, touched, lr)
+                assert_bits_equal(after, want, "cfg1 det sgd")
+            else:
+                assert_within_l1(after, before.astype(np.float64) - lr * delta64,
+                                 lr * l1 + np.abs(before), what="cfg1 atomic sgd")
+                assert_bits_equal(after[l1 == 0], before[l1 == 0], "untouched slots")
+
+
+def test_deterministic_is_bit_reproducible_and_order_sensitive_case():
+    # a hot id: thousands of terms on the same slots; five runs must give identical bits
+    w = small(d=32, Z=8, M=300, batch=2000, vocab_arg=(2, 3, 1000))
+    with Case(w) as c:
+        g_h, g_d = _grad(c, 5)
+        can, _ = c.oracle.backward_canonical(g_h, c.indices_h, c.offsets_h, c.B)
+        runs = [c.backward(g_d, "det").cpu().numpy() for _ in range(5)]
+        for r in runs:
+            assert_bits_equal(r, can, "hot id deterministic")
+
+
+def test_backward_empty_inputs():
+    w = small(bag_rule=(2, 0, 5))
+    with Case(w, batch=4) as c:
+        c.offsets = torch.zeros(c.nbags + 1, dtype=torch.int64, device=c.dev)
+        c.indices = torch.zeros(0, dtype=torch.int64, device=c.dev)
+        _, g_d = _grad(c, 0)
+        for mode in ("atomic", "det"):
+            ga = c.backward(g_d, mode).cpu().numpy()
+            assert np.all(ga == 0)
+
+
+# ---------------------------------------------------------------------------------------
+# the five workloads at full size (the launch configurations the benchmark times)
+# ---------------------------------------------------------------------------------------
+
+def _sample_bags(nbags, n, seed):
+    rng = np.random.default_rng(seed)
+    n = min(n, nbags)
+    picks = rng.choice(nbags, size=n, replace=False)
+    picks[:4] = [0, 1, nbags - 2, nbags - 1][:len(picks[:4])]
+    return np.sort(picks).astype(np.int64)
+
+
+def _check_forward_sampled(c, nsample=20000):
+    got = c.forward().reshape(c.nbags, c.w.d)
+    bags = _sample_bags(c.nbags, nsample, 1)
+    want = c.oracle_forward_bags(bags)
+    assert_bits_equal(got[torch.from_numpy(bags).to(c.dev)].cpu().numpy(), want, c.w.name + " forward")
+    return got
+
+
+def test_cfg2_forward_full_size():
+    with Case(synth.workload(2)) as c:
+        got = c.forward()
+        # the whole output, not a sample: the oracle needs a few seconds for 1.7M rows
+        assert_bits_equal(got.cpu().numpy(), c.oracle_forward(), "cfg2 forward (all rows)")
+
+
+@pytest.mark.parametrize("Z", [1, 128])
+def test_cfg3_forward_backward_full_size(Z):
+    w = synth.workload(3, Z=Z)
+    with Case(w) as c:
+        _check_forward_sampled(c)
+        g_h = synth.make_grad_out(w)
+        g_d = torch.from_numpy(g_h).to(c.dev)
+        delta64, l1 = c.oracle.backward_f64(g_h, c.indices_h, c.offsets_h, c.B)
+        ga = c.backward(g_d, "atomic").cpu().numpy()
+        assert_within_l1(ga, delta64, l1, what=f"cfg3 Z={Z} atomic")
+        det = c.backward(g_d, "det").cpu().numpy()
+        assert_within_l1(det, delta64, l1, what=f"cfg3 Z={Z} det vs fp64")
+        assert_bits_equal(c.backward(g_d, "det").cpu().numpy(), det, "cfg3 det repeat")
+        if Z == 128:
+            can, touched = c.oracle.backward_canonical(g_h, c.indices_h, c.offsets_h, c.B)
+            assert_bits_equal(det, can, "cfg3 Z=128 det vs canonical")
+            before = c.array_h.copy()
+            c.backward(g_d, "det", sgd=True, lr=1.0)
+            want = before.copy()
+            orc.sgd_apply(want, can, touched, 1.0)
+            assert_bits_equal(c.array.cpu().numpy(), want, "cfg3 det sgd")
+        else:
+            before = c.array_h.copy()
+            c.backward(g_d, "atomic", sgd=True, lr=1.0)
+            assert_within_l1(c.array.cpu().numpy(), before.astype(np.float64) - delta64,
+                             l1 + np.abs(before), what="cfg3 atomic sgd")
+
+
+def test_cfg3_z1_deterministic_vs_canonical_reduced_batch():
+    # the canonical oracle sorts every block on one core; 2048 samples x 26 x 128 blocks is its size
+    w = synth.workload(3, Z=1)
+    with Case(w, batch=2048) as c:
+        g_h = synth.make_grad_out(w, 2048)
+        g_d = torch.from_numpy(g_h).to(c.dev)
+        can, _ = c.oracle.backward_canonical(g_h, c.indices_h, c.offsets_h, c.B)
+        assert_bits_equal(c.backward(g_d, "det").cpu().numpy(), can, "cfg3 Z=1 det")
+
+
+def test_cfg4_forward_backward_full_size():
+    w = synth.workload(4)
+    with Case(w) as c:
+        _check_forward_sampled(c)
+        g_h = synth.make_grad_out(w)
+        g_d = torch.from_numpy(g_h).to(c.dev)
+        delta64, l1 = c.oracle.backward_f64(g_h, c.indices_h, c.offsets_h, c.B)
+        ga = c.backward(g_d, "atomic").cpu().numpy()
+        assert_within_l1(ga, delta64, l1, what="cfg4 atomic")
+        # gradient mass is conserved (holds at any size)
+        lengths = np.diff(c.offsets_h)
+        mass = float((lengths * g_h.astype(np.float64).reshape(c.nbags, -1).sum(axis=1)).sum())
+        assert abs(float(ga.astype(np.float64).sum()) - mass) < 1e-6 * float(l1.sum())
+        del delta64, l1
+        det = c.backward(g_d, "det").cpu().numpy()
+        can, _ = c.oracle.backward_canonical(g_h, c.indices_h, c.offsets_h, c.B, j0=1_000_000, jn=3_000_000)
+        assert_bits_equal(det[1_000_000:4_000_000], can, "cfg4 det window")
+        can0, _ = c.oracle.backward_canonical(g_h, c.indices_h, c.offsets_h, c.B, j0=0, jn=100_000)
+        assert_bits_equal(det[:100_000], can0, "cfg4 det low slots")
+        canl, _ = c.oracle.backward_canonical(g_h, c.indices_h, c.offsets_h, c.B, j0=w.M - 100_000, jn=100_000)
+        assert_bits_equal(det[w.M - 100_000:], canl, "cfg4 det high slots")
+
+
+@pytest.mark.parametrize("M,Z,dtype", [
+    (262_144, 1, "f32"), (262_144, 32, "f32"), (25_000_000, 2, "f32"), (25_000_000, 8, "f32"),
+    (25_000_000, 128, "f32"), (25_000_000, 32, "bf16"),
+])
+def test_cfg5_forward_full_size(M, Z, dtype):
+    w = synth.workload(5, M=M, Z=Z, array_dtype=dtype)
+    with Case(w) as c:
+        _check_forward_sampled(c)
+
+
+@pytest.mark.parametrize("Z", [1, 32])
+def test_cfg5_forward_10gb_array(Z):
+    w = synth.workload(5, M=2_500_000_000, Z=Z)
+    free, _ = torch.cuda.mem_get_info()
+    if free < 16 * 2**30:
+        pytest.skip("not enough free device memory")
+    with Case(w, host_array=False) as c:
+        got = c.forward().reshape(c.nbags, w.d)
+        bags = _sample_bags(c.nbags, 3000, 2)
+        rows = got[torch.from_numpy(bags).to(c.dev)].cpu().numpy()
+        for r, bag in enumerate(bags):
+            slots = c.oracle.locate(int(bag % c.T), int(c.indices_h[bag])).astype(np.int64)
+            want = synth.array_values_at(w, torch.from_numpy(slots)).numpy()
+            assert_bits_equal(rows[r], want, "cfg5 10 GB")
+
+
+def test_cfg5_backward_full_size():
+    w = synth.workload(5, M=25_000_000, Z=32)
+    with Case(w) as c:
+        g_h = synth.make_grad_out(w)
+        g_d = torch.from_numpy(g_h).to(c.dev)
+        delta64, l1 = c.oracle.backward_f64(g_h, c.indices_h, c.offsets_h, c.B)
+        ga = c.backward(g_d, "atomic").cpu().numpy()
+        assert_within_l1(ga, delta64, l1, what="cfg5 atomic")
+        det = c.backward(g_d, "det").cpu().numpy()
+        can, _ = c.oracle.backward_canonical(g_h, c.indices_h, c.offsets_h, c.B)
+        assert_bits_equal(det, can, "cfg5 det")
+
+
+# ---------------------------------------------------------------------------------------
+# validation mode and argument errors that need a device pointer
+# ---------------------------------------------------------------------------------------
+
+def test_validate_mode_reports_bad_inputs_without_faulting():
+    w = small(bag_rule=(2, 0, 5))
+    with Case(w, batch=8) as c:
+        word = torch.zeros(1, dtype=torch.int32, device=c.dev)
+        robe.robe_set_status_word(c.h, word)
+        robe.robe_set_option(c.h, robe.ROBE_OPT_VALIDATE, 1)
+        good = c.forward().cpu().numpy()
+        assert robe.robe_last_device_status(c.h) == 0
+        assert_bits_equal(good, c.oracle_forward(), "validated forward")
+        bad = c.offsets.clone()
+        bad[3] = bad[4] + 5  # not monotone
+        keep = c.offsets
+        c.offsets = bad
+        out = c.forward()
+        assert robe.robe_last_device_status(c.h) == 2
+        assert torch.isnan(out).all()  # nothing was written
+        c.offsets = keep
+        word.zero_()
+        neg = c.indices.clone()
+        neg[0] = -5
+        c.indices = neg
+        c.forward()
+        assert robe.robe_last_device_status(c.h) == 1
+
+
+def test_argument_errors_on_device():
+    with Case(small()) as c:
+        out = torch.empty(c.B, c.T, c.w.d, device=c.dev)
+        with pytest.raises(robe.RobeError) as ei:
+            robe.robe_forward(c.h, c.indices[:-1], None, c.B, out)  # nnz != batch*T
+        assert ei.value.status == robe.ROBE_ERR_INVALID_ARG
+        robe.robe_set_option(c.h, robe.ROBE_OPT_BWD_MODE, robe.ROBE_BWD_DETERMINISTIC)
+        g = torch.zeros(c.B, c.T, c.w.d, device=c.dev)
+        ga = torch.zeros(c.w.M, device=c.dev)
+        with pytest.raises(robe.RobeError) as ei:
+            robe.robe_backward(c.h, g, c.indices, None, c.B, ga, 0.0, None)
+        assert ei.value.status == robe.ROBE_ERR_WORKSPACE
+    w = small(array_dtype="bf16")
+    with Case(w) as c:
+        g = torch.zeros(c.B, c.T, c.w.d, device=c.dev)
+        with pytest.raises(robe.RobeError) as ei:
+            robe.robe_backward(c.h, g, c.indices, None, c.B, None, 0.1, None)  # SGD on bf16
+        assert ei.value.status == robe.ROBE_ERR_INVALID_ARG
