@@ -81,6 +81,16 @@ __device__ __forceinline__ uint32_t table_of_bag(uint64_t k, const MapParams& mp
     return (uint32_t)__umul64hi(low, (uint64_t)mp.T);
 }
 
+// (a * b) mod P, a < P, any b: ids below 2^32 (the common case) take the short product.
+__device__ __forceinline__ uint64_t mulmod_p61_any(uint64_t a, uint64_t b) {
+    return (b >> 32) == 0 ? mulmod_p61_u32(a, (uint32_t)b) : mulmod_p61(a, b);
+}
+
+// (A e + D) mod P : the part of the hash argument that depends on the table only.
+__device__ __forceinline__ uint64_t table_term(const HashConsts& k, uint32_t e) {
+    return addmod_p61(mulmod_p61_u32(k.A, e), k.D);
+}
+
 // (A e + B x + D) mod P : the part of the hash argument shared by all chunks of one id.
 __device__ __forceinline__ uint64_t hash_base(const HashConsts& k, uint32_t e, uint64_t x) {
     uint64_t s = mulmod_p61_u32(k.A, e) + mulmod_p61(k.B, x) + k.D;  // < 3P < 2^63
@@ -119,6 +129,23 @@ template <int DT>
 __device__ __forceinline__ float load_elem(const void* array, uint32_t j) {
     if (DT == 0) return __ldg((const float*)array + j);
     return bf16_bits_to_float(__ldg((const unsigned short*)array + j));
+}
+
+// Array read of the gather kernels: read-only path, with the 64-byte L2 fetch hint.  Random
+// Z-blocks gain nothing from the wider default fetch; measured on B200 this hint shortens a
+// random 64-byte-block gather from a 1 GB array by about 13 %.
+template <int DT>
+__device__ __forceinline__ float gather_elem(const void* array, uint32_t j) {
+    if (DT == 0) {
+        float v;
+        asm("ld.global.nc.L2::64B.f32 %0, [%1];" : "=f"(v) : "l"((const float*)array + j));
+        return v;
+    }
+    unsigned short b;
+    asm("ld.global.nc.L2::64B.u16 %0, [%1];"
+                 : "=h"(b)
+                 : "l"((const unsigned short*)array + j));
+    return bf16_bits_to_float(b);
 }
 
 }  // namespace robe

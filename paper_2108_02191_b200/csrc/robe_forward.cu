@@ -65,10 +65,14 @@ __global__ void __launch_bounds__(256) fwd_direct_kernel(FwdArgs a) {
     }
 }
 
-// EPL = elements per lane (d <= 32*EPL); U = ids whose loads are issued before the first use.
-template <int EPL, int DT, bool SIGN, bool BAGS>
+// EPL   elements per lane (d <= 32*EPL)
+// MULTI chunks per embedding C > 32: a lane holds up to four block starts (chunks cl + 32k)
+// FULLD d == 32*EPL: no lane is ever past the end of the row
+// U     ids whose loads are issued before the first add
+template <int EPL, int DT, bool SIGN, bool BAGS, bool MULTI, bool FULLD>
 __global__ void __launch_bounds__(256) fwd_warp_kernel(FwdArgs a, uint32_t log2sub) {
-    constexpr int U = 4;
+    constexpr int U = (EPL == 4) ? 2 : 4;
+    constexpr int KS = MULTI ? 4 : 1;
     constexpr unsigned FULL = 0xFFFFFFFFu;
     const MapParams& mp = a.mp;
     const int64_t warp = ((int64_t)blockIdx.x * 256 + threadIdx.x) >> 5;
@@ -80,24 +84,14 @@ __global__ void __launch_bounds__(256) fwd_warp_kernel(FwdArgs a, uint32_t log2s
 
     if (a.status != nullptr && *a.status != 0) return;
 
-    // per-lane constants of the gather: element i = lane + 32u, its chunk and offset
-    uint32_t off[EPL], src[EPL], slot[EPL];
-#pragma unroll
-    for (int u = 0; u < EPL; ++u) {
-        uint32_t i = lane + 32u * u;
-        if (i >= mp.d) i = mp.d - 1;
-        uint32_t c = i >> mp.log2Z;
-        off[u] = i & (mp.Z - 1);
-        src[u] = c & (sub - 1);
-        slot[u] = c >> 5;  // warp-uniform (non-zero only when C > 32)
-    }
-
     int64_t row0, lo, hi;
-    uint32_t e_bag = 0;
+    uint64_t tterm = 0, gterm = 0;  // (A e + D) mod P of the bag's table (pooled mode)
     if (BAGS) {
         if (warp >= a.nbags) return;
         bag_range(a.offsets, a.nnz, warp, lo, hi);
-        e_bag = table_of_bag((uint64_t)warp, mp);
+        const uint32_t e_bag = table_of_bag((uint64_t)warp, mp);
+        tterm = table_term(mp.h, e_bag);
+        if (SIGN) gterm = table_term(mp.g, e_bag);
         row0 = warp;
     } else {
         row0 = warp * (int64_t)G;  // this warp serves rows [row0, row0 + G)
@@ -106,27 +100,52 @@ __global__ void __launch_bounds__(256) fwd_warp_kernel(FwdArgs a, uint32_t log2s
         hi = row0 + G < a.nbags ? row0 + G : a.nbags;
     }
 
+    // per-lane constants of the gather: element i = lane + 32u, its chunk and offset
+    uint32_t off[EPL], src[EPL], slot[EPL];
+    bool live[EPL];
+#pragma unroll
+    for (int u = 0; u < EPL; ++u) {
+        uint32_t i = lane + 32u * u;
+        live[u] = FULLD || i < mp.d;
+        if (!live[u]) i = mp.d - 1;
+        const uint32_t c = i >> mp.log2Z;
+        off[u] = i & (mp.Z - 1);
+        src[u] = c & (sub - 1);
+        slot[u] = c >> 5;  // warp-uniform (non-zero only when C > 32)
+    }
+    // per-lane constants of the hash pass: (C_h * c) mod P for the chunks this lane evaluates
+    uint64_t cterm[KS];
+#pragma unroll
+    for (int k = 0; k < KS; ++k) cterm[k] = mulmod_p61_u32(mp.h.C, cl + 32u * k);
+
+    // -0 + v == v for every v (also for v = -0), so starting from -0 makes the first term
+    // initialise the sum exactly as the definition says
     float acc[EPL];
 #pragma unroll
-    for (int u = 0; u < EPL; ++u) acc[u] = 0.0f;
-    bool first = true;
+    for (int u = 0; u < EPL; ++u) acc[u] = -0.0f;
+
+    uint64_t x_next = 0;
+    if (lo + gl < hi) x_next = (uint64_t)__ldg(a.indices + lo + gl);
 
     for (int64_t p0 = lo; p0 < hi; p0 += G) {
         const uint32_t cnt = (uint32_t)((hi - p0) < (int64_t)G ? (hi - p0) : (int64_t)G);
         // ---- hash pass: lane (gl, cl) evaluates the starts of id p0+gl, chunks cl (+32k)
-        uint32_t st[4] = {0, 0, 0, 0};
+        uint32_t st[KS];
         uint64_t gbase = 0;
-        if (gl < cnt) {
-            const int64_t p = p0 + gl;
-            const uint64_t x = (uint64_t)__ldg(a.indices + p);
-            const uint32_t e = BAGS ? e_bag : table_of_bag((uint64_t)p, mp);
-            const uint64_t base = hash_base(mp.h, e, x);
-            if (SIGN) gbase = hash_base(mp.g, e, x);
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                uint32_t c = cl + 32u * k;
-                if (c < mp.C) st[k] = block_start(mp, base, c);
+        {
+            const uint64_t x = x_next;
+            if (p0 + G + gl < hi) x_next = (uint64_t)__ldg(a.indices + p0 + G + gl);
+            uint64_t tt = tterm;
+            if (!BAGS) {
+                const uint32_t e = table_of_bag((uint64_t)(p0 + gl), mp);
+                tt = table_term(mp.h, e);
+                if (SIGN) gterm = table_term(mp.g, e);
             }
+            const uint64_t base = addmod_p61(tt, mulmod_p61_any(mp.h.B, x));
+            if (SIGN) gbase = addmod_p61(gterm, mulmod_p61_any(mp.g.B, x));
+#pragma unroll
+            for (int k = 0; k < KS; ++k)
+                st[k] = mod_m(addmod_p61(base, cterm[k]), mp.m, mp.mu);
         }
         // ---- gather pass
         for (uint32_t g0 = 0; g0 < cnt; g0 += U) {
@@ -139,14 +158,15 @@ __global__ void __launch_bounds__(256) fwd_warp_kernel(FwdArgs a, uint32_t log2s
                 if (SIGN) gb = __shfl_sync(FULL, gbase, gs << log2sub);
 #pragma unroll
                 for (int u = 0; u < EPL; ++u) {
-                    uint32_t mine = slot[u] == 0 ? st[0] : slot[u] == 1 ? st[1]
-                                  : slot[u] == 2 ? st[2] : st[3];
-                    uint32_t s = __shfl_sync(FULL, mine, (gs << log2sub) + src[u]);
+                    uint32_t mine = st[0];
+                    if (MULTI) mine = slot[u] == 0 ? st[0] : slot[u] == 1 ? st[1 % KS]
+                                    : slot[u] == 2 ? st[2 % KS] : st[3 % KS];
+                    const uint32_t s = __shfl_sync(FULL, mine, (gs << log2sub) + src[u]);
                     uint32_t j = s + off[u];
                     if (j >= mp.m) j -= mp.m;
                     float val = 0.0f;
-                    if (g < cnt && lane + 32u * u < mp.d) {
-                        val = load_elem<DT>(a.array, j);
+                    if (g < cnt && live[u]) {
+                        val = gather_elem<DT>(a.array, j);
                         if (SIGN) val = sign_of(mp, gb, lane + 32u * u) * val;
                     }
                     v[gg][u] = val;
@@ -157,8 +177,7 @@ __global__ void __launch_bounds__(256) fwd_warp_kernel(FwdArgs a, uint32_t log2s
                 for (int gg = 0; gg < U; ++gg) {
                     if (g0 + gg < cnt) {
 #pragma unroll
-                        for (int u = 0; u < EPL; ++u) acc[u] = first ? v[gg][u] : acc[u] + v[gg][u];
-                        first = false;
+                        for (int u = 0; u < EPL; ++u) acc[u] = acc[u] + v[gg][u];
                     }
                 }
             } else {
@@ -168,7 +187,7 @@ __global__ void __launch_bounds__(256) fwd_warp_kernel(FwdArgs a, uint32_t log2s
                         float* orow = a.out + (p0 + g0 + gg) * (int64_t)mp.d;
 #pragma unroll
                         for (int u = 0; u < EPL; ++u)
-                            if (lane + 32u * u < mp.d) __stcs(orow + lane + 32u * u, v[gg][u]);
+                            if (live[u]) __stcs(orow + lane + 32u * u, v[gg][u]);
                     }
                 }
             }
@@ -176,9 +195,10 @@ __global__ void __launch_bounds__(256) fwd_warp_kernel(FwdArgs a, uint32_t log2s
     }
     if (BAGS) {
         float* orow = a.out + row0 * (int64_t)mp.d;
+        const bool empty = hi <= lo;
 #pragma unroll
         for (int u = 0; u < EPL; ++u)
-            if (lane + 32u * u < mp.d) __stcs(orow + lane + 32u * u, acc[u]);
+            if (live[u]) __stcs(orow + lane + 32u * u, empty ? 0.0f : acc[u]);
     }
 }
 
@@ -188,26 +208,48 @@ static uint32_t log2_sub_for(uint32_t C) {
     return l;
 }
 
-template <int EPL, int DT, bool SIGN>
+template <int EPL, int DT, bool SIGN, bool MULTI, bool FULLD>
 static void launch_warp(const FwdArgs& a, bool bags, cudaStream_t st) {
     const uint32_t l2s = log2_sub_for(a.mp.C);
     const int64_t G = 32 >> l2s;
     const int64_t warps = bags ? a.nbags : (a.nbags + G - 1) / G;
     const unsigned blocks = (unsigned)((warps + 7) / 8);
     if (bags)
-        fwd_warp_kernel<EPL, DT, SIGN, true><<<blocks, 256, 0, st>>>(a, l2s);
+        fwd_warp_kernel<EPL, DT, SIGN, true, MULTI, FULLD><<<blocks, 256, 0, st>>>(a, l2s);
     else
-        fwd_warp_kernel<EPL, DT, SIGN, false><<<blocks, 256, 0, st>>>(a, l2s);
+        fwd_warp_kernel<EPL, DT, SIGN, false, MULTI, FULLD><<<blocks, 256, 0, st>>>(a, l2s);
 }
 
-template <int DT, bool SIGN>
-static void launch_warp_epl(const FwdArgs& a, bool bags, cudaStream_t st) {
+template <int EPL, int DT>
+static void launch_warp_flags(const FwdArgs& a, bool bags, bool sign, cudaStream_t st) {
+    const bool multi = a.mp.C > 32;
+    const bool fulld = a.mp.d == 32u * EPL;
+    if (sign) {  // the sign hash is off in every timed configuration: one generic variant
+        launch_warp<EPL, DT, true, true, false>(a, bags, st);
+        return;
+    }
+    if (EPL == 1) {  // d <= 32 means C <= 32
+        if (fulld) launch_warp<EPL, DT, false, false, true>(a, bags, st);
+        else launch_warp<EPL, DT, false, false, false>(a, bags, st);
+        return;
+    }
+    if (multi) {
+        if (fulld) launch_warp<EPL, DT, false, true, true>(a, bags, st);
+        else launch_warp<EPL, DT, false, true, false>(a, bags, st);
+    } else {
+        if (fulld) launch_warp<EPL, DT, false, false, true>(a, bags, st);
+        else launch_warp<EPL, DT, false, false, false>(a, bags, st);
+    }
+}
+
+template <int DT>
+static void launch_warp_epl(const FwdArgs& a, bool bags, bool sign, cudaStream_t st) {
     if (a.mp.d <= 32)
-        launch_warp<1, DT, SIGN>(a, bags, st);
+        launch_warp_flags<1, DT>(a, bags, sign, st);
     else if (a.mp.d <= 64)
-        launch_warp<2, DT, SIGN>(a, bags, st);
+        launch_warp_flags<2, DT>(a, bags, sign, st);
     else
-        launch_warp<4, DT, SIGN>(a, bags, st);
+        launch_warp_flags<4, DT>(a, bags, sign, st);
 }
 
 cudaError_t launch_forward(const Problem& pb, float* out, int variant, cudaStream_t st) {
@@ -218,13 +260,8 @@ cudaError_t launch_forward(const Problem& pb, float* out, int variant, cudaStrea
     if (variant == 2 && !warp_ok) return cudaErrorInvalidValue;
     const bool use_warp = variant == 2 || (variant == 0 && warp_ok);
     if (use_warp) {
-        if (pb.dtype == 0) {
-            if (pb.sign) launch_warp_epl<0, true>(a, bags, st);
-            else launch_warp_epl<0, false>(a, bags, st);
-        } else {
-            if (pb.sign) launch_warp_epl<1, true>(a, bags, st);
-            else launch_warp_epl<1, false>(a, bags, st);
-        }
+        if (pb.dtype == 0) launch_warp_epl<0>(a, bags, pb.sign != 0, st);
+        else launch_warp_epl<1>(a, bags, pb.sign != 0, st);
     } else {
         const unsigned blocks = (unsigned)((pb.nbags + 7) / 8);
         if (pb.dtype == 0) {
