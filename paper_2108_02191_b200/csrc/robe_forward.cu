@@ -4,10 +4,10 @@
 //
 // Two kernels:
 //   fwd_direct_kernel  any Z, any d: every lane hashes the chunk of its own element.
-//   fwd_warp_kernel    Z a power of two and d <= 128: the 32 lanes of a warp first
-//                      evaluate 32 block starts at once (several ids x chunks), then
-//                      hand them to the lanes that gather through warp shuffles, so the
-//                      hash cost per id does not depend on how many lanes read a block.
+//   fwd_staged_kernel  d <= 128: a warp first evaluates the block starts of a whole batch of
+//                      ids (one (id, chunk) pair per lane) into a warp-private staging area in
+//                      shared memory, then gathers without further integer work, so the hash
+//                      cost per id does not depend on how many lanes read a block.
 #include "robe_internal.h"
 
 namespace robe {
@@ -65,136 +65,141 @@ __global__ void __launch_bounds__(256) fwd_direct_kernel(FwdArgs a) {
     }
 }
 
-// EPL   elements per lane (d <= 32*EPL)
-// MULTI chunks per embedding C > 32: a lane holds up to four block starts (chunks cl + 32k)
-// FULLD d == 32*EPL: no lane is ever past the end of the row
-// U     ids whose loads are issued before the first add
-template <int EPL, int DT, bool SIGN, bool BAGS, bool MULTI, bool FULLD>
-__global__ void __launch_bounds__(256) fwd_warp_kernel(FwdArgs a, uint32_t log2sub) {
-    constexpr int U = (EPL == 4) ? 2 : 4;
-    constexpr int KS = MULTI ? 4 : 1;
-    constexpr unsigned FULL = 0xFFFFFFFFu;
-    const MapParams& mp = a.mp;
-    const int64_t warp = ((int64_t)blockIdx.x * 256 + threadIdx.x) >> 5;
-    const uint32_t lane = threadIdx.x & 31;
-    const uint32_t sub = 1u << log2sub;   // lanes that hash one id: min(32, pow2ceil(C))
-    const uint32_t G = 32u >> log2sub;    // ids hashed per pass
-    const uint32_t gl = lane >> log2sub;  // which id of the pass this lane hashes
-    const uint32_t cl = lane & (sub - 1); // which chunk (plus multiples of 32 when C > 32)
+// Staged kernel (any Z, d <= 128).  One warp serves one bag (pooled) or one group of
+// consecutive rows (one-hot).  It works in two phases per batch of ids, with a warp-private
+// staging area in shared memory and only __syncwarp between the phases:
+//   hash phase    lanes take the ids of the batch, one id per lane, and store (A e + B x + D)
+//                 mod P; then lanes take the (id, chunk) pairs of the batch, 32 at a time, and
+//                 store the block starts h(e,x,c);
+//   gather phase  lane l owns elements l, l+32, ...; it reads its block start from shared
+//                 memory, adds its in-block offset, wraps, and loads; the loads of U ids are
+//                 issued before the first add.
+// EPL = elements per lane (d <= 32*EPL).  FULLD: d == 32*EPL (no lane is past the row end).
+constexpr int kStageEntries = 256;  // block starts per warp
+constexpr int kStageIds = 64;       // ids per warp batch
 
+struct StageSmem {
+    uint64_t cterm[128];                          // (C_h * c) mod P, c < C (d <= 128)
+    uint64_t base[8][kStageIds];                  // per warp: hash base of each staged id
+    uint32_t start[8][kStageEntries];             // per warp: block starts, id-major
+};
+
+template <int EPL, int DT, bool SIGN, bool BAGS, bool FULLD, int MINB>
+__global__ void __launch_bounds__(256, MINB)
+fwd_staged_kernel(FwdArgs a, uint32_t ids_per_batch, uint32_t cmagic) {
+    constexpr int U = (EPL == 4) ? 2 : 4;
+    __shared__ StageSmem sm;
+    const MapParams& mp = a.mp;
+    const uint32_t lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const int64_t warp = (int64_t)blockIdx.x * 8 + w;
+
+    if (threadIdx.x < mp.C) sm.cterm[threadIdx.x] = mulmod_p61_u32(mp.h.C, threadIdx.x);
+    __syncthreads();
     if (a.status != nullptr && *a.status != 0) return;
 
-    int64_t row0, lo, hi;
-    uint64_t tterm = 0, gterm = 0;  // (A e + D) mod P of the bag's table (pooled mode)
+    int64_t lo, hi;
+    uint64_t tterm = 0, gterm = 0;
     if (BAGS) {
         if (warp >= a.nbags) return;
         bag_range(a.offsets, a.nnz, warp, lo, hi);
         const uint32_t e_bag = table_of_bag((uint64_t)warp, mp);
         tterm = table_term(mp.h, e_bag);
         if (SIGN) gterm = table_term(mp.g, e_bag);
-        row0 = warp;
     } else {
-        row0 = warp * (int64_t)G;  // this warp serves rows [row0, row0 + G)
-        if (row0 >= a.nbags) return;
-        lo = row0;
-        hi = row0 + G < a.nbags ? row0 + G : a.nbags;
+        lo = warp * (int64_t)ids_per_batch;  // this warp serves rows [lo, lo + ids_per_batch)
+        if (lo >= a.nbags) return;
+        hi = lo + ids_per_batch < a.nbags ? lo + ids_per_batch : a.nbags;
     }
 
     // per-lane constants of the gather: element i = lane + 32u, its chunk and offset
-    uint32_t off[EPL], src[EPL], slot[EPL];
+    uint32_t off[EPL], chk[EPL];
     bool live[EPL];
 #pragma unroll
     for (int u = 0; u < EPL; ++u) {
         uint32_t i = lane + 32u * u;
         live[u] = FULLD || i < mp.d;
         if (!live[u]) i = mp.d - 1;
-        const uint32_t c = i >> mp.log2Z;
-        off[u] = i & (mp.Z - 1);
-        src[u] = c & (sub - 1);
-        slot[u] = c >> 5;  // warp-uniform (non-zero only when C > 32)
+        chunk_of(mp, i, chk[u], off[u]);
     }
-    // per-lane constants of the hash pass: (C_h * c) mod P for the chunks this lane evaluates
-    uint64_t cterm[KS];
-#pragma unroll
-    for (int k = 0; k < KS; ++k) cterm[k] = mulmod_p61_u32(mp.h.C, cl + 32u * k);
 
-    // -0 + v == v for every v (also for v = -0), so starting from -0 makes the first term
-    // initialise the sum exactly as the definition says
+    uint64_t* base_s = sm.base[w];
+    uint32_t* start_s = sm.start[w];
+    // the sign hash needs its own per-id base; it shares the staging area's upper half
+    // (the batch is halved when the sign is on)
+    uint64_t* gbase_s = base_s + kStageIds / 2;
+
+    // -0 + v == v for every v (also v = -0): starting from -0 makes the first term initialise
+    // the sum exactly as the definition says
     float acc[EPL];
 #pragma unroll
     for (int u = 0; u < EPL; ++u) acc[u] = -0.0f;
 
-    uint64_t x_next = 0;
-    if (lo + gl < hi) x_next = (uint64_t)__ldg(a.indices + lo + gl);
-
-    for (int64_t p0 = lo; p0 < hi; p0 += G) {
-        const uint32_t cnt = (uint32_t)((hi - p0) < (int64_t)G ? (hi - p0) : (int64_t)G);
-        // ---- hash pass: lane (gl, cl) evaluates the starts of id p0+gl, chunks cl (+32k)
-        uint32_t st[KS];
-        uint64_t gbase = 0;
-        {
-            const uint64_t x = x_next;
-            if (p0 + G + gl < hi) x_next = (uint64_t)__ldg(a.indices + p0 + G + gl);
-            uint64_t tt = tterm;
+    for (int64_t p0 = lo; p0 < hi; p0 += ids_per_batch) {
+        const uint32_t cnt = (uint32_t)((hi - p0) < (int64_t)ids_per_batch ? (hi - p0)
+                                                                            : (int64_t)ids_per_batch);
+        // ---- hash phase, step 1: one id per lane
+        for (uint32_t t = lane; t < cnt; t += 32) {
+            const uint64_t x = (uint64_t)__ldg(a.indices + p0 + t);
+            uint64_t tt = tterm, gt = gterm;
             if (!BAGS) {
-                const uint32_t e = table_of_bag((uint64_t)(p0 + gl), mp);
+                const uint32_t e = table_of_bag((uint64_t)(p0 + t), mp);
                 tt = table_term(mp.h, e);
-                if (SIGN) gterm = table_term(mp.g, e);
+                if (SIGN) gt = table_term(mp.g, e);
             }
-            const uint64_t base = addmod_p61(tt, mulmod_p61_any(mp.h.B, x));
-            if (SIGN) gbase = addmod_p61(gterm, mulmod_p61_any(mp.g.B, x));
-#pragma unroll
-            for (int k = 0; k < KS; ++k)
-                st[k] = mod_m(addmod_p61(base, cterm[k]), mp.m, mp.mu);
+            base_s[t] = addmod_p61(tt, mulmod_p61_any(mp.h.B, x));
+            if (SIGN) gbase_s[t] = addmod_p61(gt, mulmod_p61_any(mp.g.B, x));
         }
-        // ---- gather pass
+        __syncwarp();
+        // ---- hash phase, step 2: one (id, chunk) pair per lane
+        const uint32_t entries = cnt * mp.C;
+        for (uint32_t t = lane; t < entries; t += 32) {
+            const uint32_t idl = (t * cmagic) >> 20;  // t / C, exact for t < 8192
+            const uint32_t c = t - idl * mp.C;
+            start_s[t] = mod_m(addmod_p61(base_s[idl], sm.cterm[c]), mp.m, mp.mu);
+        }
+        __syncwarp();
+        // ---- gather phase
         for (uint32_t g0 = 0; g0 < cnt; g0 += U) {
             float v[U][EPL];
 #pragma unroll
             for (int gg = 0; gg < U; ++gg) {
-                const uint32_t g = g0 + gg;           // warp-uniform
-                const uint32_t gs = g < cnt ? g : cnt - 1;
-                uint64_t gb = 0;
-                if (SIGN) gb = __shfl_sync(FULL, gbase, gs << log2sub);
+                const uint32_t g = g0 + gg;  // warp-uniform
+                const bool on = g < cnt;
+                const uint32_t gs = on ? g : cnt - 1;
 #pragma unroll
                 for (int u = 0; u < EPL; ++u) {
-                    uint32_t mine = st[0];
-                    if (MULTI) mine = slot[u] == 0 ? st[0] : slot[u] == 1 ? st[1 % KS]
-                                    : slot[u] == 2 ? st[2 % KS] : st[3 % KS];
-                    const uint32_t s = __shfl_sync(FULL, mine, (gs << log2sub) + src[u]);
-                    uint32_t j = s + off[u];
+                    uint32_t j = start_s[gs * mp.C + chk[u]] + off[u];  // < m + d <= 2^32
                     if (j >= mp.m) j -= mp.m;
                     float val = 0.0f;
-                    if (g < cnt && live[u]) {
+                    if (on && live[u]) {
                         val = gather_elem<DT>(a.array, j);
-                        if (SIGN) val = sign_of(mp, gb, lane + 32u * u) * val;
+                        if (SIGN) val = sign_of(mp, gbase_s[gs], lane + 32u * u) * val;
                     }
                     v[gg][u] = val;
                 }
             }
             if (BAGS) {
 #pragma unroll
-                for (int gg = 0; gg < U; ++gg) {
+                for (int gg = 0; gg < U; ++gg)
                     if (g0 + gg < cnt) {
 #pragma unroll
                         for (int u = 0; u < EPL; ++u) acc[u] = acc[u] + v[gg][u];
                     }
-                }
             } else {
 #pragma unroll
-                for (int gg = 0; gg < U; ++gg) {
+                for (int gg = 0; gg < U; ++gg)
                     if (g0 + gg < cnt) {
                         float* orow = a.out + (p0 + g0 + gg) * (int64_t)mp.d;
 #pragma unroll
                         for (int u = 0; u < EPL; ++u)
                             if (live[u]) __stcs(orow + lane + 32u * u, v[gg][u]);
                     }
-                }
             }
         }
+        __syncwarp();  // the staging area is rewritten by the next batch
     }
     if (BAGS) {
-        float* orow = a.out + row0 * (int64_t)mp.d;
+        float* orow = a.out + warp * (int64_t)mp.d;
         const bool empty = hi <= lo;
 #pragma unroll
         for (int u = 0; u < EPL; ++u)
@@ -202,66 +207,67 @@ __global__ void __launch_bounds__(256) fwd_warp_kernel(FwdArgs a, uint32_t log2s
     }
 }
 
-static uint32_t log2_sub_for(uint32_t C) {
-    uint32_t l = 0;
-    while ((1u << l) < C && l < 5) ++l;
-    return l;
+// ids a warp stages per batch: as many as fit the staging area (and at least one)
+static uint32_t staged_ids_per_batch(const MapParams& mp, bool bags, bool sign) {
+    uint32_t cap = kStageEntries / mp.C;
+    const uint32_t idcap = sign ? kStageIds / 2 : kStageIds;
+    if (cap > idcap) cap = idcap;
+    if (cap < 1) cap = 1;
+    if (!bags) {
+        // one-hot: rows per warp; enough pairs to fill the lanes twice, not more, so that small
+        // batches still spread over many warps
+        uint32_t want = (64 + mp.C - 1) / mp.C;
+        if (want < 1) want = 1;
+        if (cap > want) cap = want;
+    }
+    return cap;
 }
 
-template <int EPL, int DT, bool SIGN, bool MULTI, bool FULLD>
-static void launch_warp(const FwdArgs& a, bool bags, cudaStream_t st) {
-    const uint32_t l2s = log2_sub_for(a.mp.C);
-    const int64_t G = 32 >> l2s;
-    const int64_t warps = bags ? a.nbags : (a.nbags + G - 1) / G;
+template <int EPL, int DT, bool SIGN, bool FULLD>
+static void launch_staged(const FwdArgs& a, bool bags, cudaStream_t st) {
+    constexpr int MINB = (EPL == 4) ? 6 : 8;
+    const uint32_t ipb = staged_ids_per_batch(a.mp, bags, SIGN);
+    const uint32_t cmagic = ((1u << 20) + a.mp.C - 1) / a.mp.C;
+    const int64_t warps = bags ? a.nbags : (a.nbags + ipb - 1) / ipb;
     const unsigned blocks = (unsigned)((warps + 7) / 8);
     if (bags)
-        fwd_warp_kernel<EPL, DT, SIGN, true, MULTI, FULLD><<<blocks, 256, 0, st>>>(a, l2s);
+        fwd_staged_kernel<EPL, DT, SIGN, true, FULLD, MINB><<<blocks, 256, 0, st>>>(a, ipb, cmagic);
     else
-        fwd_warp_kernel<EPL, DT, SIGN, false, MULTI, FULLD><<<blocks, 256, 0, st>>>(a, l2s);
+        fwd_staged_kernel<EPL, DT, SIGN, false, FULLD, MINB><<<blocks, 256, 0, st>>>(a, ipb, cmagic);
 }
 
 template <int EPL, int DT>
-static void launch_warp_flags(const FwdArgs& a, bool bags, bool sign, cudaStream_t st) {
-    const bool multi = a.mp.C > 32;
+static void launch_staged_flags(const FwdArgs& a, bool bags, bool sign, cudaStream_t st) {
     const bool fulld = a.mp.d == 32u * EPL;
     if (sign) {  // the sign hash is off in every timed configuration: one generic variant
-        launch_warp<EPL, DT, true, true, false>(a, bags, st);
-        return;
-    }
-    if (EPL == 1) {  // d <= 32 means C <= 32
-        if (fulld) launch_warp<EPL, DT, false, false, true>(a, bags, st);
-        else launch_warp<EPL, DT, false, false, false>(a, bags, st);
-        return;
-    }
-    if (multi) {
-        if (fulld) launch_warp<EPL, DT, false, true, true>(a, bags, st);
-        else launch_warp<EPL, DT, false, true, false>(a, bags, st);
+        launch_staged<EPL, DT, true, false>(a, bags, st);
+    } else if (fulld) {
+        launch_staged<EPL, DT, false, true>(a, bags, st);
     } else {
-        if (fulld) launch_warp<EPL, DT, false, false, true>(a, bags, st);
-        else launch_warp<EPL, DT, false, false, false>(a, bags, st);
+        launch_staged<EPL, DT, false, false>(a, bags, st);
     }
 }
 
 template <int DT>
-static void launch_warp_epl(const FwdArgs& a, bool bags, bool sign, cudaStream_t st) {
+static void launch_staged_epl(const FwdArgs& a, bool bags, bool sign, cudaStream_t st) {
     if (a.mp.d <= 32)
-        launch_warp_flags<1, DT>(a, bags, sign, st);
+        launch_staged_flags<1, DT>(a, bags, sign, st);
     else if (a.mp.d <= 64)
-        launch_warp_flags<2, DT>(a, bags, sign, st);
+        launch_staged_flags<2, DT>(a, bags, sign, st);
     else
-        launch_warp_flags<4, DT>(a, bags, sign, st);
+        launch_staged_flags<4, DT>(a, bags, sign, st);
 }
 
 cudaError_t launch_forward(const Problem& pb, float* out, int variant, cudaStream_t st) {
     if (pb.nbags == 0) return cudaSuccess;
     FwdArgs a{pb.mp, pb.array, pb.indices, pb.offsets, out, pb.nbags, pb.nnz, pb.status};
     const bool bags = pb.offsets != nullptr;
-    const bool warp_ok = pb.mp.log2Z != 0xFFFFFFFFu && pb.mp.d <= 128;
+    const bool warp_ok = pb.mp.d <= 128;
     if (variant == 2 && !warp_ok) return cudaErrorInvalidValue;
     const bool use_warp = variant == 2 || (variant == 0 && warp_ok);
     if (use_warp) {
-        if (pb.dtype == 0) launch_warp_epl<0>(a, bags, pb.sign != 0, st);
-        else launch_warp_epl<1>(a, bags, pb.sign != 0, st);
+        if (pb.dtype == 0) launch_staged_epl<0>(a, bags, pb.sign != 0, st);
+        else launch_staged_epl<1>(a, bags, pb.sign != 0, st);
     } else {
         const unsigned blocks = (unsigned)((pb.nbags + 7) / 8);
         if (pb.dtype == 0) {
