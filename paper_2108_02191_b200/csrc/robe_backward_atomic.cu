@@ -5,9 +5,10 @@
 // itself (scale = -lr: the SGD step fused into the scatter).  fp32 reductions in global
 // memory (red.global.add.f32); the order of the additions is not fixed.
 //
-// Same two shapes as the forward: a direct kernel for any (Z, d) and a warp kernel that
-// evaluates 32 block starts per pass and distributes them by shuffles.
+// Same two shapes as the forward: a direct kernel for any (Z, d) and a staged kernel
+// (d <= 128) that evaluates the block starts of a batch of ids into shared memory first.
 #include "robe_internal.h"
+#include "robe_stage.cuh"
 
 namespace robe {
 
@@ -23,21 +24,6 @@ struct BwdArgs {
     const int32_t* status;
 };
 
-__device__ __forceinline__ int64_t clamp64b(int64_t v, int64_t lo, int64_t hi) {
-    return v < lo ? lo : (v > hi ? hi : v);
-}
-
-__device__ __forceinline__ void bag_range_b(const int64_t* offsets, int64_t nnz, int64_t k,
-                                            int64_t& lo, int64_t& hi) {
-    if (offsets == nullptr) {
-        lo = k;
-        hi = k + 1;
-    } else {
-        lo = clamp64b(__ldg(offsets + k), 0, nnz);
-        hi = clamp64b(__ldg(offsets + k + 1), lo, nnz);
-    }
-}
-
 template <bool SIGN>
 __global__ void __launch_bounds__(256) bwd_atomic_direct_kernel(BwdArgs a) {
     const int64_t k = ((int64_t)blockIdx.x * 256 + threadIdx.x) >> 5;
@@ -46,7 +32,7 @@ __global__ void __launch_bounds__(256) bwd_atomic_direct_kernel(BwdArgs a) {
     if (a.status != nullptr && *a.status != 0) return;
     const MapParams& mp = a.mp;
     int64_t lo, hi;
-    bag_range_b(a.offsets, a.nnz, k, lo, hi);
+    bag_range(a.offsets, a.nnz, k, lo, hi);
     const uint32_t e = table_of_bag((uint64_t)k, mp);
     for (uint32_t i = lane; i < mp.d; i += 32) {
         uint32_t c, o;
@@ -63,122 +49,101 @@ __global__ void __launch_bounds__(256) bwd_atomic_direct_kernel(BwdArgs a) {
     }
 }
 
-template <int EPL, bool SIGN, bool BAGS>
-__global__ void __launch_bounds__(256) bwd_atomic_warp_kernel(BwdArgs a, uint32_t log2sub) {
-    constexpr unsigned FULL = 0xFFFFFFFFu;
+// Staged kernel (any Z, d <= 128): same two phases as the staged forward kernel - the warp
+// first evaluates the block starts of a batch of ids into its shared-memory staging area, then
+// every lane issues one fp32 reduction per (id, element) it owns.  The gradient row of a bag is
+// read once and kept in registers for all ids of the bag.
+template <int EPL, bool SIGN, bool BAGS, bool FULLD, int MINB>
+__global__ void __launch_bounds__(256, MINB)
+bwd_atomic_staged_kernel(BwdArgs a, uint32_t ids_per_batch, uint32_t cmagic) {
+    __shared__ StageSmem sm;
     const MapParams& mp = a.mp;
-    const int64_t warp = ((int64_t)blockIdx.x * 256 + threadIdx.x) >> 5;
-    const uint32_t lane = threadIdx.x & 31;
-    const uint32_t sub = 1u << log2sub;
-    const uint32_t G = 32u >> log2sub;
-    const uint32_t gl = lane >> log2sub;
-    const uint32_t cl = lane & (sub - 1);
+    const uint32_t lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const int64_t warp = (int64_t)blockIdx.x * 8 + w;
 
+    stage_init(sm, mp);
     if (a.status != nullptr && *a.status != 0) return;
 
-    uint32_t off[EPL], src[EPL], slot[EPL];
+    int64_t lo, hi;
+    uint64_t tterm = 0, gterm = 0;
+    if (BAGS) {
+        if (warp >= a.nbags) return;
+        bag_range(a.offsets, a.nnz, warp, lo, hi);
+        const uint32_t e_bag = table_of_bag((uint64_t)warp, mp);
+        tterm = table_term(mp.h, e_bag);
+        if (SIGN) gterm = table_term(mp.g, e_bag);
+    } else {
+        lo = warp * (int64_t)ids_per_batch;
+        if (lo >= a.nbags) return;
+        hi = lo + ids_per_batch < a.nbags ? lo + ids_per_batch : a.nbags;
+    }
+
+    uint32_t off[EPL], chk[EPL];
+    bool live[EPL];
+    float gv[EPL];
 #pragma unroll
     for (int u = 0; u < EPL; ++u) {
         uint32_t i = lane + 32u * u;
-        if (i >= mp.d) i = mp.d - 1;
-        uint32_t c = i >> mp.log2Z;
-        off[u] = i & (mp.Z - 1);
-        src[u] = c & (sub - 1);
-        slot[u] = c >> 5;
+        live[u] = FULLD || i < mp.d;
+        if (!live[u]) i = mp.d - 1;
+        chunk_of(mp, i, chk[u], off[u]);
+        gv[u] = 0.0f;
+        if (BAGS && live[u]) gv[u] = __ldcs(a.grad_out + warp * (int64_t)mp.d + i) * a.scale;
     }
+    const uint32_t* start_s = sm.start[w];
+    const uint64_t* gbase_s = sm.base[w] + kStageIds / 2;
 
-    int64_t lo, hi;
-    uint32_t e_bag = 0;
-    float gbag[EPL];
-    if (BAGS) {
-        if (warp >= a.nbags) return;
-        bag_range_b(a.offsets, a.nnz, warp, lo, hi);
-        e_bag = table_of_bag((uint64_t)warp, mp);
-#pragma unroll
-        for (int u = 0; u < EPL; ++u)
-            gbag[u] = lane + 32u * u < mp.d
-                          ? __ldcs(a.grad_out + warp * (int64_t)mp.d + lane + 32u * u) * a.scale
-                          : 0.0f;
-    } else {
-        lo = warp * (int64_t)G;
-        if (lo >= a.nbags) return;
-        hi = lo + G < a.nbags ? lo + G : a.nbags;
-    }
-
-    for (int64_t p0 = lo; p0 < hi; p0 += G) {
-        const uint32_t cnt = (uint32_t)((hi - p0) < (int64_t)G ? (hi - p0) : (int64_t)G);
-        uint32_t st[4] = {0, 0, 0, 0};
-        uint64_t gbase = 0;
-        if (gl < cnt) {
-            const int64_t p = p0 + gl;
-            const uint64_t x = (uint64_t)__ldg(a.indices + p);
-            const uint32_t e = BAGS ? e_bag : table_of_bag((uint64_t)p, mp);
-            const uint64_t base = hash_base(mp.h, e, x);
-            if (SIGN) gbase = hash_base(mp.g, e, x);
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                uint32_t c = cl + 32u * k;
-                if (c < mp.C) st[k] = block_start(mp, base, c);
-            }
-        }
+    for (int64_t p0 = lo; p0 < hi; p0 += ids_per_batch) {
+        const uint32_t cnt = (uint32_t)((hi - p0) < (int64_t)ids_per_batch ? (hi - p0)
+                                                                            : (int64_t)ids_per_batch);
+        stage_batch<SIGN, BAGS>(sm, mp, a.indices, p0, cnt, tterm, gterm, cmagic, w, lane);
         for (uint32_t g = 0; g < cnt; ++g) {
-            float gv[EPL];
-            if (BAGS) {
-#pragma unroll
-                for (int u = 0; u < EPL; ++u) gv[u] = gbag[u];
-            } else {
+            if (!BAGS) {
 #pragma unroll
                 for (int u = 0; u < EPL; ++u)
-                    gv[u] = lane + 32u * u < mp.d
-                                ? __ldcs(a.grad_out + (p0 + g) * (int64_t)mp.d + lane + 32u * u) *
-                                      a.scale
-                                : 0.0f;
+                    if (live[u])
+                        gv[u] = __ldcs(a.grad_out + (p0 + g) * (int64_t)mp.d + lane + 32u * u) * a.scale;
             }
-            uint64_t gb = 0;
-            if (SIGN) gb = __shfl_sync(FULL, gbase, g << log2sub);
 #pragma unroll
             for (int u = 0; u < EPL; ++u) {
-                uint32_t mine = slot[u] == 0 ? st[0] : slot[u] == 1 ? st[1]
-                              : slot[u] == 2 ? st[2] : st[3];
-                uint32_t s = __shfl_sync(FULL, mine, (g << log2sub) + src[u]);
-                uint32_t j = s + off[u];
+                uint32_t j = start_s[g * mp.C + chk[u]] + off[u];
                 if (j >= mp.m) j -= mp.m;
-                if (lane + 32u * u < mp.d) {
+                if (live[u]) {
                     float t = gv[u];
-                    if (SIGN) t = sign_of(mp, gb, lane + 32u * u) * t;
+                    if (SIGN) t = sign_of(mp, gbase_s[g], lane + 32u * u) * t;
                     atomicAdd(a.target + j, t);
                 }
             }
         }
+        __syncwarp();
     }
 }
 
-static uint32_t log2_sub_for_b(uint32_t C) {
-    uint32_t l = 0;
-    while ((1u << l) < C && l < 5) ++l;
-    return l;
-}
-
-template <int EPL, bool SIGN>
-static void launch_bwd_warp(const BwdArgs& a, bool bags, cudaStream_t st) {
-    const uint32_t l2s = log2_sub_for_b(a.mp.C);
-    const int64_t G = 32 >> l2s;
-    const int64_t warps = bags ? a.nbags : (a.nbags + G - 1) / G;
+template <int EPL, bool SIGN, bool FULLD>
+static void launch_bwd_staged(const BwdArgs& a, bool bags, cudaStream_t st) {
+    constexpr int MINB = (EPL == 4) ? 6 : 8;
+    const uint32_t ipb = staged_ids_per_batch(a.mp, bags, SIGN);
+    const uint32_t cmagic = chunk_magic(a.mp);
+    const int64_t warps = bags ? a.nbags : (a.nbags + ipb - 1) / ipb;
     const unsigned blocks = (unsigned)((warps + 7) / 8);
     if (bags)
-        bwd_atomic_warp_kernel<EPL, SIGN, true><<<blocks, 256, 0, st>>>(a, l2s);
+        bwd_atomic_staged_kernel<EPL, SIGN, true, FULLD, MINB><<<blocks, 256, 0, st>>>(a, ipb, cmagic);
     else
-        bwd_atomic_warp_kernel<EPL, SIGN, false><<<blocks, 256, 0, st>>>(a, l2s);
+        bwd_atomic_staged_kernel<EPL, SIGN, false, FULLD, MINB><<<blocks, 256, 0, st>>>(a, ipb, cmagic);
 }
 
-template <bool SIGN>
-static void launch_bwd_warp_epl(const BwdArgs& a, bool bags, cudaStream_t st) {
-    if (a.mp.d <= 32)
-        launch_bwd_warp<1, SIGN>(a, bags, st);
-    else if (a.mp.d <= 64)
-        launch_bwd_warp<2, SIGN>(a, bags, st);
-    else
-        launch_bwd_warp<4, SIGN>(a, bags, st);
+template <int EPL>
+static void launch_bwd_staged_flags(const BwdArgs& a, bool bags, bool sign, cudaStream_t st) {
+    const bool fulld = a.mp.d == 32u * EPL;
+    if (sign) launch_bwd_staged<EPL, true, false>(a, bags, st);
+    else if (fulld) launch_bwd_staged<EPL, false, true>(a, bags, st);
+    else launch_bwd_staged<EPL, false, false>(a, bags, st);
+}
+
+static void launch_bwd_staged_epl(const BwdArgs& a, bool bags, bool sign, cudaStream_t st) {
+    if (a.mp.d <= 32) launch_bwd_staged_flags<1>(a, bags, sign, st);
+    else if (a.mp.d <= 64) launch_bwd_staged_flags<2>(a, bags, sign, st);
+    else launch_bwd_staged_flags<4>(a, bags, sign, st);
 }
 
 cudaError_t launch_backward_atomic(const Problem& pb, const float* grad_out, float* target,
@@ -186,12 +151,11 @@ cudaError_t launch_backward_atomic(const Problem& pb, const float* grad_out, flo
     if (pb.nbags == 0) return cudaSuccess;
     BwdArgs a{pb.mp, grad_out, pb.indices, pb.offsets, target, scale, pb.nbags, pb.nnz, pb.status};
     const bool bags = pb.offsets != nullptr;
-    const bool warp_ok = pb.mp.log2Z != 0xFFFFFFFFu && pb.mp.d <= 128;
+    const bool warp_ok = pb.mp.d <= 128;
     if (variant == 2 && !warp_ok) return cudaErrorInvalidValue;
     const bool use_warp = variant == 2 || (variant == 0 && warp_ok);
     if (use_warp) {
-        if (pb.sign) launch_bwd_warp_epl<true>(a, bags, st);
-        else launch_bwd_warp_epl<false>(a, bags, st);
+        launch_bwd_staged_epl(a, bags, pb.sign != 0, st);
     } else {
         const unsigned blocks = (unsigned)((pb.nbags + 7) / 8);
         if (pb.sign) bwd_atomic_direct_kernel<true><<<blocks, 256, 0, st>>>(a);

@@ -9,6 +9,7 @@
 //                      shared memory, then gathers without further integer work, so the hash
 //                      cost per id does not depend on how many lanes read a block.
 #include "robe_internal.h"
+#include "robe_stage.cuh"
 
 namespace robe {
 
@@ -22,22 +23,6 @@ struct FwdArgs {
     int64_t nnz;
     const int32_t* status;
 };
-
-__device__ __forceinline__ int64_t clamp64(int64_t v, int64_t lo, int64_t hi) {
-    return v < lo ? lo : (v > hi ? hi : v);
-}
-
-// ids of bag k: indices[lo, hi); malformed offsets are clamped so no read leaves indices[].
-__device__ __forceinline__ void bag_range(const int64_t* offsets, int64_t nnz, int64_t k,
-                                          int64_t& lo, int64_t& hi) {
-    if (offsets == nullptr) {
-        lo = k;
-        hi = k + 1;
-    } else {
-        lo = clamp64(__ldg(offsets + k), 0, nnz);
-        hi = clamp64(__ldg(offsets + k + 1), lo, nnz);
-    }
-}
 
 template <int DT, bool SIGN>
 __global__ void __launch_bounds__(256) fwd_direct_kernel(FwdArgs a) {
@@ -75,15 +60,6 @@ __global__ void __launch_bounds__(256) fwd_direct_kernel(FwdArgs a) {
 //                 memory, adds its in-block offset, wraps, and loads; the loads of U ids are
 //                 issued before the first add.
 // EPL = elements per lane (d <= 32*EPL).  FULLD: d == 32*EPL (no lane is past the row end).
-constexpr int kStageEntries = 256;  // block starts per warp
-constexpr int kStageIds = 64;       // ids per warp batch
-
-struct StageSmem {
-    uint64_t cterm[128];                          // (C_h * c) mod P, c < C (d <= 128)
-    uint64_t base[8][kStageIds];                  // per warp: hash base of each staged id
-    uint32_t start[8][kStageEntries];             // per warp: block starts, id-major
-};
-
 template <int EPL, int DT, bool SIGN, bool BAGS, bool FULLD, int MINB>
 __global__ void __launch_bounds__(256, MINB)
 fwd_staged_kernel(FwdArgs a, uint32_t ids_per_batch, uint32_t cmagic) {
@@ -93,8 +69,7 @@ fwd_staged_kernel(FwdArgs a, uint32_t ids_per_batch, uint32_t cmagic) {
     const uint32_t lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     const int64_t warp = (int64_t)blockIdx.x * 8 + w;
 
-    if (threadIdx.x < mp.C) sm.cterm[threadIdx.x] = mulmod_p61_u32(mp.h.C, threadIdx.x);
-    __syncthreads();
+    stage_init(sm, mp);
     if (a.status != nullptr && *a.status != 0) return;
 
     int64_t lo, hi;
@@ -122,11 +97,8 @@ fwd_staged_kernel(FwdArgs a, uint32_t ids_per_batch, uint32_t cmagic) {
         chunk_of(mp, i, chk[u], off[u]);
     }
 
-    uint64_t* base_s = sm.base[w];
-    uint32_t* start_s = sm.start[w];
-    // the sign hash needs its own per-id base; it shares the staging area's upper half
-    // (the batch is halved when the sign is on)
-    uint64_t* gbase_s = base_s + kStageIds / 2;
+    const uint32_t* start_s = sm.start[w];
+    const uint64_t* gbase_s = sm.base[w] + kStageIds / 2;  // sign-hash bases (sign on only)
 
     // -0 + v == v for every v (also v = -0): starting from -0 makes the first term initialise
     // the sum exactly as the definition says
@@ -137,27 +109,7 @@ fwd_staged_kernel(FwdArgs a, uint32_t ids_per_batch, uint32_t cmagic) {
     for (int64_t p0 = lo; p0 < hi; p0 += ids_per_batch) {
         const uint32_t cnt = (uint32_t)((hi - p0) < (int64_t)ids_per_batch ? (hi - p0)
                                                                             : (int64_t)ids_per_batch);
-        // ---- hash phase, step 1: one id per lane
-        for (uint32_t t = lane; t < cnt; t += 32) {
-            const uint64_t x = (uint64_t)__ldg(a.indices + p0 + t);
-            uint64_t tt = tterm, gt = gterm;
-            if (!BAGS) {
-                const uint32_t e = table_of_bag((uint64_t)(p0 + t), mp);
-                tt = table_term(mp.h, e);
-                if (SIGN) gt = table_term(mp.g, e);
-            }
-            base_s[t] = addmod_p61(tt, mulmod_p61_any(mp.h.B, x));
-            if (SIGN) gbase_s[t] = addmod_p61(gt, mulmod_p61_any(mp.g.B, x));
-        }
-        __syncwarp();
-        // ---- hash phase, step 2: one (id, chunk) pair per lane
-        const uint32_t entries = cnt * mp.C;
-        for (uint32_t t = lane; t < entries; t += 32) {
-            const uint32_t idl = (t * cmagic) >> 20;  // t / C, exact for t < 8192
-            const uint32_t c = t - idl * mp.C;
-            start_s[t] = mod_m(addmod_p61(base_s[idl], sm.cterm[c]), mp.m, mp.mu);
-        }
-        __syncwarp();
+        stage_batch<SIGN, BAGS>(sm, mp, a.indices, p0, cnt, tterm, gterm, cmagic, w, lane);
         // ---- gather phase
         for (uint32_t g0 = 0; g0 < cnt; g0 += U) {
             float v[U][EPL];
@@ -207,27 +159,11 @@ fwd_staged_kernel(FwdArgs a, uint32_t ids_per_batch, uint32_t cmagic) {
     }
 }
 
-// ids a warp stages per batch: as many as fit the staging area (and at least one)
-static uint32_t staged_ids_per_batch(const MapParams& mp, bool bags, bool sign) {
-    uint32_t cap = kStageEntries / mp.C;
-    const uint32_t idcap = sign ? kStageIds / 2 : kStageIds;
-    if (cap > idcap) cap = idcap;
-    if (cap < 1) cap = 1;
-    if (!bags) {
-        // one-hot: rows per warp; enough pairs to fill the lanes twice, not more, so that small
-        // batches still spread over many warps
-        uint32_t want = (64 + mp.C - 1) / mp.C;
-        if (want < 1) want = 1;
-        if (cap > want) cap = want;
-    }
-    return cap;
-}
-
 template <int EPL, int DT, bool SIGN, bool FULLD>
 static void launch_staged(const FwdArgs& a, bool bags, cudaStream_t st) {
     constexpr int MINB = (EPL == 4) ? 6 : 8;
     const uint32_t ipb = staged_ids_per_batch(a.mp, bags, SIGN);
-    const uint32_t cmagic = ((1u << 20) + a.mp.C - 1) / a.mp.C;
+    const uint32_t cmagic = chunk_magic(a.mp);
     const int64_t warps = bags ? a.nbags : (a.nbags + ipb - 1) / ipb;
     const unsigned blocks = (unsigned)((warps + 7) / 8);
     if (bags)
