@@ -362,10 +362,14 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg4", choices=["cfg2", "cfg3_z1", "cfg3_z128", "cfg4", "cfg5"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--batch", type=int, default=0,
+                    help="samples per GPU instead of the workload's own batch (small profiler captures)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
     w = pick_workload(args.workload)
+    if args.batch > 0:
+        w = w.with_(batch=args.batch, name=f"{w.name}_batch{args.batch}")
     if args.impl == "reference":
         return run_reference(args, w)
     return run_ours(args, w)
