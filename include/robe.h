@@ -156,6 +156,50 @@ int robe_backward(robe_handle_t h, const float* grad_out, const int64_t* indices
                   void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * robe_backward_deterministic_static - the deterministic robe_backward for callers that
+ * cannot supply scratch memory.  (The paper has no counterpart: this is a convenience of
+ * this library, not part of the method.)
+ *
+ * Who needs it: code that runs where device allocation is off the table - for example a
+ * serving process whose memory pool already owns the whole device, so a cudaMalloc would
+ * fail or stall every stream while it synchronises the device, or an operator plugged
+ * into a host framework that hands it input and output buffers and nothing else.  Such a
+ * caller has no way to come up with the workspace robe_backward asks for in
+ * deterministic mode.  Here the workspace is a fixed array of ROBE_STATIC_SCRATCH_BYTES
+ * that is part of the library image itself: every device that loads librobe.so carries
+ * it from load until the process exits, whether or not this function is ever called.
+ *
+ * Arguments and result are those of robe_backward in ROBE_BWD_DETERMINISTIC mode (the
+ * handle's ROBE_OPT_BWD_MODE is ignored), minus workspace/workspace_bytes: the caller
+ * still passes grad_out, indices, offsets and grad_array (or NULL for the fused SGD step),
+ * and gets bit-identical output.  The function calls no cudaMalloc, cudaFree or other
+ * allocating routine.
+ *
+ * Limit: the call must fit the fixed array, i.e. the value robe_backward_workspace_bytes
+ * reports for it in deterministic mode (about 16 bytes per block, nnz * ceil(d/Z) blocks,
+ * plus 4 bytes per id and 0.6 MB of counters) must not exceed ROBE_STATIC_SCRATCH_BYTES;
+ * a larger call returns ROBE_ERR_WORKSPACE and launches nothing.
+ *
+ * First call on a device: the function looks up the device address of the array once per
+ * device (with that device current) and remembers it.  Make that first call during
+ * set-up, before any stream capture is begun.
+ *
+ * Sharing: all handles, streams and threads of the process use the same array on a given
+ * device, and it keeps whatever the previous call left in it.  The function re-initialises
+ * the parts that must start from zero on every call, so back-to-back calls on ONE stream
+ * are safe; two calls that may overlap on the GPU (different streams without an ordering
+ * between them) race on the array and give undefined results - order them yourself.
+ *
+ * Errors: as robe_backward, plus ROBE_ERR_WORKSPACE for a call beyond the limit and
+ * ROBE_ERR_CUDA if the address lookup fails.
+ */
+#define ROBE_STATIC_SCRATCH_BYTES (32u << 20) /* 32 MiB per device */
+int robe_backward_deterministic_static(robe_handle_t h, const float* grad_out,
+                                       const int64_t* indices, const int64_t* offsets,
+                                       int64_t batch, int64_t nnz, float* grad_array, float lr,
+                                       void* stream);
+
+/*
  * robe_set_status_word - give the handle a device int32 (caller-owned, zeroed by the
  * caller) that kernels write a ROBE_DEV_* code into when ROBE_OPT_VALIDATE is on.
  * robe_last_device_status - synchronise `stream`, read that word (device-to-host copy)

@@ -34,10 +34,13 @@ ROBE_OPT_BWD_KERNEL = 5
 ROBE_BWD_ATOMIC = 0
 ROBE_BWD_DETERMINISTIC = 1
 
+ROBE_STATIC_SCRATCH_BYTES = 32 << 20
+
 EXPORTS = [
     "robe_create", "robe_destroy", "robe_set_option", "robe_attach_array",
     "robe_get_hash_constants", "robe_forward", "robe_backward_workspace_bytes", "robe_backward",
     "robe_set_status_word", "robe_last_device_status", "robe_status_string",
+    "robe_backward_deterministic_static",
 ]
 
 if not os.path.exists(LIB_PATH):
@@ -57,6 +60,7 @@ _lib.robe_forward.argtypes = [_vp, _vp, _vp, _i64, _i64, _vp, _vp]
 _lib.robe_backward_workspace_bytes.argtypes = [_vp, _i64, _i64]
 _lib.robe_backward_workspace_bytes.restype = C.c_size_t
 _lib.robe_backward.argtypes = [_vp, _vp, _vp, _vp, _i64, _i64, _vp, C.c_float, _vp, C.c_size_t, _vp]
+_lib.robe_backward_deterministic_static.argtypes = [_vp, _vp, _vp, _vp, _i64, _i64, _vp, C.c_float, _vp]
 _lib.robe_set_status_word.argtypes = [_vp, _vp]
 _lib.robe_last_device_status.argtypes = [_vp, _vp]
 _lib.robe_status_string.argtypes = [C.c_int]
@@ -148,6 +152,17 @@ def robe_backward(h, grad_out, indices, offsets, batch: int, grad_array=None, lr
                               _dev_ptr(offsets, torch.int64), batch, indices.numel(),
                               _dev_ptr(grad_array, torch.float32), lr, _dev_ptr(workspace),
                               ws_bytes, _stream_ptr(stream)), "robe_backward")
+
+
+def robe_backward_deterministic_static(h, grad_out, indices, offsets, batch: int, grad_array=None,
+                                       lr: float = 0.0, stream=None) -> None:
+    """Deterministic backward on the library's built-in scratch array, for callers that cannot
+    allocate a workspace (include/robe.h has the limit and the sharing rules).  No tensor is
+    created here: the arguments are passed through as they are."""
+    _check(_lib.robe_backward_deterministic_static(
+        h, _dev_ptr(grad_out, torch.float32), _dev_ptr(indices, torch.int64),
+        _dev_ptr(offsets, torch.int64), batch, indices.numel(), _dev_ptr(grad_array, torch.float32),
+        lr, _stream_ptr(stream)), "robe_backward_deterministic_static")
 
 
 def robe_set_status_word(h, word) -> None:

@@ -1,11 +1,17 @@
 // C ABI of librobe.so: handle, options, argument checks, hash-constant draw, dispatch.
 // The entry points are documented in include/robe.h.
+#include <mutex>
 #include <new>
 
 #include "../../include/robe.h"
 #include "robe_internal.h"
 
 using namespace robe;
+
+// Scratch of robe_backward_deterministic_static: part of the library image, so every device
+// that loads the library holds these bytes until the process exits.  In host code this name
+// is only a stand-in for the symbol; the device address comes from cudaGetSymbolAddress.
+static __device__ __align__(256) unsigned char robe_static_scratch[ROBE_STATIC_SCRATCH_BYTES];
 
 struct robe_ctx {
     uint64_t M;
@@ -262,6 +268,62 @@ int robe_backward(robe_handle_t h, const float* grad_out, const int64_t* indices
     if (launch_validate(pb, st) != cudaSuccess) return ROBE_ERR_CUDA;
     if (launch_backward_det(pb, grad_out, target, sgd ? 1 : 0, lr, workspace, workspace_bytes,
                             st) != cudaSuccess)
+        return ROBE_ERR_CUDA;
+    return ROBE_OK;
+}
+
+// Device address of robe_static_scratch on the current device, looked up once per device.
+static int static_scratch_address(void** out) {
+    constexpr int kMaxDevices = 64;
+    static std::mutex mu;
+    static void* addr[kMaxDevices] = {};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return ROBE_ERR_CUDA;
+    if (dev < 0 || dev >= kMaxDevices) return ROBE_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(mu);
+    if (addr[dev] == nullptr) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, robe_static_scratch) != cudaSuccess || p == nullptr)
+            return ROBE_ERR_CUDA;
+        addr[dev] = p;
+    }
+    *out = addr[dev];
+    return ROBE_OK;
+}
+
+int robe_backward_deterministic_static(robe_handle_t h, const float* grad_out,
+                                       const int64_t* indices, const int64_t* offsets,
+                                       int64_t batch, int64_t nnz, float* grad_array, float lr,
+                                       void* stream) {
+    if (!check_sizes(h, indices, offsets, batch, nnz)) return ROBE_ERR_INVALID_ARG;
+    if (batch > 0 && grad_out == nullptr) return ROBE_ERR_INVALID_ARG;
+    if (h->validate && h->status_word == nullptr) return ROBE_ERR_INVALID_ARG;
+    const bool sgd = grad_array == nullptr;
+    if (sgd) {
+        if (h->array == nullptr) return ROBE_ERR_NO_ARRAY;
+        if (h->dtype != ROBE_F32) return ROBE_ERR_INVALID_ARG;
+    }
+    float* target = sgd ? (float*)h->array : grad_array;
+    const Problem pb = make_problem(h, indices, offsets, batch, nnz);
+    const uint64_t nb = (uint64_t)nnz * h->mp.C;
+    uint32_t zp = 1;
+    while (zp < h->mp.Z) zp <<= 1;
+    if (nb >= (1ull << 32) || (uint64_t)pb.nbags >= (1ull << 32)) return ROBE_ERR_UNSUPPORTED;
+    if (nb * zp / 256 >= (1ull << 31)) return ROBE_ERR_UNSUPPORTED;
+    // the fixed array is the whole workspace: a call that needs more is refused up front (by
+    // the same figure robe_backward_workspace_bytes reports, which covers pooled input too)
+    const size_t need = det_workspace_bytes(h->mp, pb.nbags, nnz, true);
+    if (need > (size_t)ROBE_STATIC_SCRATCH_BYTES) return ROBE_ERR_WORKSPACE;
+    void* scratch = nullptr;
+    const int rc = static_scratch_address(&scratch);
+    if (rc != ROBE_OK) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (launch_validate(pb, st) != cudaSuccess) return ROBE_ERR_CUDA;
+    // Stale contents are harmless: keys, values and digit counters are fully rewritten before
+    // they are read, and the one buffer that must start from zero (the bag number of each id,
+    // pooled input only) is cleared by the launch itself on the same stream.
+    if (launch_backward_det(pb, grad_out, target, sgd ? 1 : 0, lr, scratch,
+                            (size_t)ROBE_STATIC_SCRATCH_BYTES, st) != cudaSuccess)
         return ROBE_ERR_CUDA;
     return ROBE_OK;
 }
