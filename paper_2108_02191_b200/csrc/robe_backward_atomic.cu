@@ -96,7 +96,7 @@ bwd_atomic_staged_kernel(BwdArgs a, uint32_t ids_per_batch, uint32_t cmagic) {
     for (int64_t p0 = lo; p0 < hi; p0 += ids_per_batch) {
         const uint32_t cnt = (uint32_t)((hi - p0) < (int64_t)ids_per_batch ? (hi - p0)
                                                                             : (int64_t)ids_per_batch);
-        stage_batch<SIGN, BAGS>(sm, mp, a.indices, p0, cnt, tterm, gterm, cmagic, w, lane);
+        stage_batch<SIGN, BAGS>(sm, mp, a.indices, p0, cnt, ids_per_batch, tterm, gterm, cmagic, w, lane);
         for (uint32_t g = 0; g < cnt; ++g) {
             if (!BAGS) {
 #pragma unroll
@@ -106,7 +106,7 @@ bwd_atomic_staged_kernel(BwdArgs a, uint32_t ids_per_batch, uint32_t cmagic) {
             }
 #pragma unroll
             for (int u = 0; u < EPL; ++u) {
-                uint32_t j = start_s[g * mp.C + chk[u]] + off[u];
+                uint32_t j = start_s[chk[u] * ids_per_batch + g] + off[u];
                 if (j >= mp.m) j -= mp.m;
                 if (live[u]) {
                     float t = gv[u];

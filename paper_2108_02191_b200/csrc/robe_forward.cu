@@ -57,13 +57,90 @@ __global__ void __launch_bounds__(256) fwd_direct_kernel(FwdArgs a) {
 //                 mod P; then lanes take the (id, chunk) pairs of the batch, 32 at a time, and
 //                 store the block starts h(e,x,c);
 //   gather phase  lane l owns elements l, l+32, ...; it reads its block start from shared
-//                 memory, adds its in-block offset, wraps, and loads; the loads of U ids are
-//                 issued before the first add.
+//                 memory, adds its in-block offset (wrapping only if some block of the batch
+//                 reaches the array end), and loads; the loads of U ids are issued before the
+//                 first add.
 // EPL = elements per lane (d <= 32*EPL).  FULLD: d == 32*EPL (no lane is past the row end).
-template <int EPL, int DT, bool SIGN, bool BAGS, bool FULLD, int MINB>
+
+// Loads of one group of n <= U ids of the staged batch, ids g0 .. g0+n-1.  WRAP: slot numbers
+// are wrapped at the array end; TAIL: n may be below U.
+template <int EPL, int DT, bool SIGN, int U, bool WRAP, bool TAIL>
+__device__ __forceinline__ void gather_group(const FwdArgs& a, const uint32_t* const (&col)[EPL],
+                                             const uint32_t (&off)[EPL], const bool (&live)[EPL],
+                                             const uint64_t* gbase_s, uint32_t g0, uint32_t n,
+                                             uint32_t lane, float (&v)[U][EPL]) {
+    const MapParams& mp = a.mp;
+#pragma unroll
+    for (int gg = 0; gg < U; ++gg) {
+        const bool on = !TAIL || (uint32_t)gg < n;  // warp-uniform
+#pragma unroll
+        for (int u = 0; u < EPL; ++u) {
+            float val = 0.0f;
+            if (on && live[u]) {
+                uint32_t j = col[u][g0 + gg] + off[u];  // < m + d <= 2^32
+                if (WRAP && j >= mp.m) j -= mp.m;
+                val = gather_elem<DT>(a.array, j);
+                if (SIGN) val = sign_of(mp, gbase_s[g0 + gg], lane + 32u * u) * val;
+            }
+            v[gg][u] = val;
+        }
+    }
+}
+
+// Gather phase of one staged batch: pooled rows are added to acc in id order, one-hot rows are
+// stored straight to the output.
+template <int EPL, int DT, bool SIGN, bool BAGS, int U, bool WRAP>
+__device__ __forceinline__ void gather_batch(const FwdArgs& a, const uint32_t* const (&col)[EPL],
+                                             const uint32_t (&off)[EPL], const bool (&live)[EPL],
+                                             const uint64_t* gbase_s, uint32_t cnt, int64_t p0,
+                                             uint32_t lane, float (&acc)[EPL]) {
+    const MapParams& mp = a.mp;
+    uint32_t g0 = 0;
+    for (; g0 + U <= cnt; g0 += U) {
+        float v[U][EPL];
+        gather_group<EPL, DT, SIGN, U, WRAP, false>(a, col, off, live, gbase_s, g0, U, lane, v);
+        if (BAGS) {
+#pragma unroll
+            for (int gg = 0; gg < U; ++gg)
+#pragma unroll
+                for (int u = 0; u < EPL; ++u) acc[u] = acc[u] + v[gg][u];
+        } else {
+#pragma unroll
+            for (int gg = 0; gg < U; ++gg) {
+                float* orow = a.out + (p0 + g0 + gg) * (int64_t)mp.d;
+#pragma unroll
+                for (int u = 0; u < EPL; ++u)
+                    if (live[u]) __stcs(orow + lane + 32u * u, v[gg][u]);
+            }
+        }
+    }
+    if (g0 < cnt) {
+        const uint32_t n = cnt - g0;
+        float v[U][EPL];
+        gather_group<EPL, DT, SIGN, U, WRAP, true>(a, col, off, live, gbase_s, g0, n, lane, v);
+        if (BAGS) {
+#pragma unroll
+            for (int gg = 0; gg < U; ++gg)
+                if ((uint32_t)gg < n) {
+#pragma unroll
+                    for (int u = 0; u < EPL; ++u) acc[u] = acc[u] + v[gg][u];
+                }
+        } else {
+#pragma unroll
+            for (int gg = 0; gg < U; ++gg)
+                if ((uint32_t)gg < n) {
+                    float* orow = a.out + (p0 + g0 + gg) * (int64_t)mp.d;
+#pragma unroll
+                    for (int u = 0; u < EPL; ++u)
+                        if (live[u]) __stcs(orow + lane + 32u * u, v[gg][u]);
+                }
+        }
+    }
+}
+
+template <int EPL, int DT, bool SIGN, bool BAGS, bool FULLD, int MINB, int U>
 __global__ void __launch_bounds__(256, MINB)
 fwd_staged_kernel(FwdArgs a, uint32_t ids_per_batch, uint32_t cmagic) {
-    constexpr int U = (EPL == 4) ? 2 : 4;
     __shared__ StageSmem sm;
     const MapParams& mp = a.mp;
     const uint32_t lane = threadIdx.x & 31, w = threadIdx.x >> 5;
@@ -86,18 +163,20 @@ fwd_staged_kernel(FwdArgs a, uint32_t ids_per_batch, uint32_t cmagic) {
         hi = lo + ids_per_batch < a.nbags ? lo + ids_per_batch : a.nbags;
     }
 
-    // per-lane constants of the gather: element i = lane + 32u, its chunk and offset
-    uint32_t off[EPL], chk[EPL];
+    // per-lane constants of the gather: element i = lane + 32u, its in-block offset, and the
+    // column of the staging area that holds the starts of its chunk
+    uint32_t off[EPL];
+    const uint32_t* col[EPL];
     bool live[EPL];
 #pragma unroll
     for (int u = 0; u < EPL; ++u) {
         uint32_t i = lane + 32u * u;
         live[u] = FULLD || i < mp.d;
         if (!live[u]) i = mp.d - 1;
-        chunk_of(mp, i, chk[u], off[u]);
+        uint32_t chk;
+        chunk_of(mp, i, chk, off[u]);
+        col[u] = sm.start[w] + chk * ids_per_batch;
     }
-
-    const uint32_t* start_s = sm.start[w];
     const uint64_t* gbase_s = sm.base[w] + kStageIds / 2;  // sign-hash bases (sign on only)
 
     // -0 + v == v for every v (also v = -0): starting from -0 makes the first term initialise
@@ -109,45 +188,12 @@ fwd_staged_kernel(FwdArgs a, uint32_t ids_per_batch, uint32_t cmagic) {
     for (int64_t p0 = lo; p0 < hi; p0 += ids_per_batch) {
         const uint32_t cnt = (uint32_t)((hi - p0) < (int64_t)ids_per_batch ? (hi - p0)
                                                                             : (int64_t)ids_per_batch);
-        stage_batch<SIGN, BAGS>(sm, mp, a.indices, p0, cnt, tterm, gterm, cmagic, w, lane);
-        // ---- gather phase
-        for (uint32_t g0 = 0; g0 < cnt; g0 += U) {
-            float v[U][EPL];
-#pragma unroll
-            for (int gg = 0; gg < U; ++gg) {
-                const uint32_t g = g0 + gg;  // warp-uniform
-                const bool on = g < cnt;
-                const uint32_t gs = on ? g : cnt - 1;
-#pragma unroll
-                for (int u = 0; u < EPL; ++u) {
-                    uint32_t j = start_s[gs * mp.C + chk[u]] + off[u];  // < m + d <= 2^32
-                    if (j >= mp.m) j -= mp.m;
-                    float val = 0.0f;
-                    if (on && live[u]) {
-                        val = gather_elem<DT>(a.array, j);
-                        if (SIGN) val = sign_of(mp, gbase_s[gs], lane + 32u * u) * val;
-                    }
-                    v[gg][u] = val;
-                }
-            }
-            if (BAGS) {
-#pragma unroll
-                for (int gg = 0; gg < U; ++gg)
-                    if (g0 + gg < cnt) {
-#pragma unroll
-                        for (int u = 0; u < EPL; ++u) acc[u] = acc[u] + v[gg][u];
-                    }
-            } else {
-#pragma unroll
-                for (int gg = 0; gg < U; ++gg)
-                    if (g0 + gg < cnt) {
-                        float* orow = a.out + (p0 + g0 + gg) * (int64_t)mp.d;
-#pragma unroll
-                        for (int u = 0; u < EPL; ++u)
-                            if (live[u]) __stcs(orow + lane + 32u * u, v[gg][u]);
-                    }
-            }
-        }
+        const bool wraps = stage_batch<SIGN, BAGS>(sm, mp, a.indices, p0, cnt, ids_per_batch, tterm,
+                                                   gterm, cmagic, w, lane);
+        if (wraps)
+            gather_batch<EPL, DT, SIGN, BAGS, U, true>(a, col, off, live, gbase_s, cnt, p0, lane, acc);
+        else
+            gather_batch<EPL, DT, SIGN, BAGS, U, false>(a, col, off, live, gbase_s, cnt, p0, lane, acc);
         __syncwarp();  // the staging area is rewritten by the next batch
     }
     if (BAGS) {
@@ -159,17 +205,26 @@ fwd_staged_kernel(FwdArgs a, uint32_t ids_per_batch, uint32_t cmagic) {
     }
 }
 
+#ifndef ROBE_FWD_U_BAGS
+#define ROBE_FWD_U_BAGS 4
+#endif
+#ifndef ROBE_FWD_MINB
+#define ROBE_FWD_MINB 8
+#endif
+
 template <int EPL, int DT, bool SIGN, bool FULLD>
 static void launch_staged(const FwdArgs& a, bool bags, cudaStream_t st) {
-    constexpr int MINB = (EPL == 4) ? 6 : 8;
+    constexpr int MINB = (EPL == 4) ? 6 : ROBE_FWD_MINB;
+    constexpr int UB = (EPL == 4) ? 2 : ROBE_FWD_U_BAGS;
+    constexpr int UO = (EPL == 4) ? 2 : 4;
     const uint32_t ipb = staged_ids_per_batch(a.mp, bags, SIGN);
     const uint32_t cmagic = chunk_magic(a.mp);
     const int64_t warps = bags ? a.nbags : (a.nbags + ipb - 1) / ipb;
     const unsigned blocks = (unsigned)((warps + 7) / 8);
     if (bags)
-        fwd_staged_kernel<EPL, DT, SIGN, true, FULLD, MINB><<<blocks, 256, 0, st>>>(a, ipb, cmagic);
+        fwd_staged_kernel<EPL, DT, SIGN, true, FULLD, MINB, UB><<<blocks, 256, 0, st>>>(a, ipb, cmagic);
     else
-        fwd_staged_kernel<EPL, DT, SIGN, false, FULLD, MINB><<<blocks, 256, 0, st>>>(a, ipb, cmagic);
+        fwd_staged_kernel<EPL, DT, SIGN, false, FULLD, MINB, UO><<<blocks, 256, 0, st>>>(a, ipb, cmagic);
 }
 
 template <int EPL, int DT>

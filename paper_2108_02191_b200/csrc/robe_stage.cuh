@@ -24,10 +24,13 @@ __device__ __forceinline__ void bag_range(const int64_t* offsets, int64_t nnz, i
 constexpr int kStageEntries = 256;  // block starts per warp
 constexpr int kStageIds = 64;       // ids per warp batch
 
+// The block starts of a batch are kept chunk-major: start[c * stride + t] is the start of chunk c
+// of the t-th id of the batch, stride = ids per batch.  A lane that owns element i of every row
+// then reads one column, start[chunk(i) * stride + t] for t = 0, 1, ..: consecutive words.
 struct StageSmem {
     uint64_t cterm[128];               // (C_h * c) mod P, c < C (d <= 128)
     uint64_t base[8][kStageIds];       // per warp: hash base of each staged id
-    uint32_t start[8][kStageEntries];  // per warp: block starts, id-major
+    uint32_t start[8][kStageEntries];  // per warp: block starts, chunk-major
 };
 
 // ids a warp stages per batch: as many as fit the staging area (and at least one)
@@ -56,15 +59,16 @@ __device__ __forceinline__ void stage_init(StageSmem& sm, const MapParams& mp) {
 
 // Hash phase of one batch of cnt ids starting at position p0 (warp-collective).
 //   step 1: one id per lane          -> base_s[t] = (A e + B x + D) mod P  (and the sign base)
-//   step 2: one (id, chunk) per lane -> start_s[t*C + c] = h(e, x, c)
+//   step 2: one (id, chunk) per lane -> start_s[c*stride + t] = h(e, x, c)
 // In pooled mode tterm/gterm are the bag's table terms; in one-hot mode the table of row
 // p0+t is (p0+t) mod T.  The sign base shares the upper half of base_s (the batch is halved
-// when the sign is on).
+// when the sign is on).  Returns (warp-uniform) whether some block of the batch may run past
+// the end of the array, i.e. whether the gather has to wrap slot numbers at all.
 template <bool SIGN, bool BAGS>
-__device__ __forceinline__ void stage_batch(StageSmem& sm, const MapParams& mp,
+__device__ __forceinline__ bool stage_batch(StageSmem& sm, const MapParams& mp,
                                             const int64_t* indices, int64_t p0, uint32_t cnt,
-                                            uint64_t tterm, uint64_t gterm, uint32_t cmagic,
-                                            uint32_t w, uint32_t lane) {
+                                            uint32_t stride, uint64_t tterm, uint64_t gterm,
+                                            uint32_t cmagic, uint32_t w, uint32_t lane) {
     uint64_t* base_s = sm.base[w];
     uint64_t* gbase_s = base_s + kStageIds / 2;
     uint32_t* start_s = sm.start[w];
@@ -81,12 +85,18 @@ __device__ __forceinline__ void stage_batch(StageSmem& sm, const MapParams& mp,
     }
     __syncwarp();
     const uint32_t entries = cnt * mp.C;
+    const uint32_t last_fit = mp.m - mp.Z;  // a block starting beyond this reaches the array end
+    bool wraps = false;
     for (uint32_t t = lane; t < entries; t += 32) {
         const uint32_t idl = (t * cmagic) >> 20;  // t / C, exact for t < 8192
         const uint32_t c = t - idl * mp.C;
-        start_s[t] = mod_m(addmod_p61(base_s[idl], sm.cterm[c]), mp.m, mp.mu);
+        const uint32_t s = mod_m(addmod_p61(base_s[idl], sm.cterm[c]), mp.m, mp.mu);
+        start_s[c * stride + idl] = s;
+        wraps |= s > last_fit;
     }
-    __syncwarp();
+    const bool any = __any_sync(0xFFFFFFFFu, wraps);
+    __syncwarp();  // the stores above are visible to the whole warp from here on
+    return any;
 }
 
 }  // namespace robe
