@@ -262,6 +262,7 @@ int robe_backward(robe_handle_t h, const float* grad_out, const int64_t* indices
     while (zp < h->mp.Z) zp <<= 1;
     if (nb >= (1ull << 32) || (uint64_t)pb.nbags >= (1ull << 32)) return ROBE_ERR_UNSUPPORTED;
     if (nb * zp / 256 >= (1ull << 31)) return ROBE_ERR_UNSUPPORTED;
+    if ((uint64_t)pb.nbags * h->mp.d > (1ull << 32)) return ROBE_ERR_UNSUPPORTED;
     const size_t need = det_workspace_bytes(h->mp, pb.nbags, nnz, offsets != nullptr);
     if (nnz > 0 && (workspace == nullptr || workspace_bytes < need)) return ROBE_ERR_WORKSPACE;
     if (((uintptr_t)workspace & 255u) != 0) return ROBE_ERR_WORKSPACE;
@@ -310,6 +311,7 @@ int robe_backward_deterministic_static(robe_handle_t h, const float* grad_out,
     while (zp < h->mp.Z) zp <<= 1;
     if (nb >= (1ull << 32) || (uint64_t)pb.nbags >= (1ull << 32)) return ROBE_ERR_UNSUPPORTED;
     if (nb * zp / 256 >= (1ull << 31)) return ROBE_ERR_UNSUPPORTED;
+    if ((uint64_t)pb.nbags * h->mp.d > (1ull << 32)) return ROBE_ERR_UNSUPPORTED;
     // the fixed array is the whole workspace: a call that needs more is refused up front (by
     // the same figure robe_backward_workspace_bytes reports, which covers pooled input too)
     const size_t need = det_workspace_bytes(h->mp, pb.nbags, nnz, true);

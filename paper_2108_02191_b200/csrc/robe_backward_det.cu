@@ -1,15 +1,18 @@
 // Deterministic backward (Section 3.1 backward equation, evaluated in a fixed order).
 //
 // Blocks are numbered q = p*C + c in input order (p = position in indices, c = chunk).
-//   1. key kernel      key[q] = h(e, x_p, c), val[q] = q
-//   2. radix sort      stable LSD sort of (key, val) by key - our own three-kernel passes
-//                      (digit count per CTA range, exclusive scan, ranked scatter)
-//   3. apply kernel    one thread per touched array slot j walks the sorted blocks whose
-//                      key lies in [j-Z+1, j] in sorted order and sums their terms left to
-//                      right in fp32 from +0, then performs ONE add (dense gradient) or ONE
-//                      fma (SGD) on slot j.  Slots [0, Z-1), which also receive the wrapped
-//                      tails of blocks near the end of the array, are handled by a small
-//                      second kernel (those terms come last: their keys are the largest).
+//   1. key kernel      key[q] = h(e, x_p, c); val[q] = where the block's gradient elements
+//                      start in grad_out (sign off) or q itself (sign on)
+//   2. radix sort      stable LSD sort of (key, val) by key - our own passes: digit count per
+//                      CTA range, per-digit exclusive scan, ranked scatter through shared
+//                      memory (so that every digit's run leaves the CTA as one coalesced piece)
+//   3. apply kernel    one thread per touched array slot j sums, left to right in fp32 from +0,
+//                      the terms of the sorted blocks whose key lies in [j-Z+1, j], then performs
+//                      ONE add (dense gradient) or ONE fma (SGD) on slot j.  The thread that owns
+//                      slot j is the one at the first sorted block of that key window, so it only
+//                      ever walks forward through the sorted list.  Slots [0, Z-1), which also
+//                      receive the wrapped tails of blocks near the end of the array, are handled
+//                      by a small second kernel (those terms come last: their keys are the largest).
 // No atomics on floating-point data and no waits between CTAs: the result is bit-reproducible.
 #include "robe_internal.h"
 
@@ -69,86 +72,123 @@ __global__ void __launch_bounds__(256) det_bag_of_kernel(KeyArgs a, uint32_t* ba
     for (int64_t p = lo + lane; p < hi; p += 32) bag_of[p] = (uint32_t)k;
 }
 
-// key[q] = h(e, x_p, c), val[q] = q for q = p*C + c
+// key[q] = h(e, x_p, c) for q = p*C + c.  val[q] = q when the sign hash is on (the apply kernel
+// then needs the id again), else the position bag*d + c*Z of the block's first gradient element.
+template <bool SIGN>
 __global__ void __launch_bounds__(256)
 det_keys_kernel(KeyArgs a, const uint32_t* bag_of, uint32_t* keys, uint32_t* vals, uint64_t nb) {
     const uint64_t q = (uint64_t)blockIdx.x * 256 + threadIdx.x;
     if (q >= nb) return;
     const MapParams& mp = a.mp;
-    const uint64_t p = q / mp.C;
-    const uint32_t c = (uint32_t)(q - p * mp.C);
-    const uint64_t bag = bag_of ? (uint64_t)bag_of[p] : p;
+    const uint32_t p = (uint32_t)q / mp.C;
+    const uint32_t c = (uint32_t)q - p * mp.C;
+    const uint64_t bag = bag_of ? (uint64_t)bag_of[p] : (uint64_t)p;
     const uint32_t e = table_of_bag(bag, mp);
     const uint64_t x = (uint64_t)__ldg(a.indices + p);
     keys[q] = block_start(mp, hash_base(mp.h, e, x), c);
-    vals[q] = (uint32_t)q;
+    vals[q] = SIGN ? (uint32_t)q : (uint32_t)(bag * mp.d + c * mp.Z);
 }
 
 // ---- radix sort pass, kernel 1: digit histogram of each CTA's contiguous key range
 __global__ void __launch_bounds__(kSortThreads)
 sort_count_kernel(const uint32_t* keys, uint32_t* counts, uint64_t nb, uint64_t tiles,
                   uint32_t shift, uint32_t mask) {
-    __shared__ uint32_t hist[kRadix];
-    hist[threadIdx.x] = 0;
+    __shared__ uint32_t hist[kSortWarps][kRadix];
+    for (int k = 0; k < kSortWarps; ++k) hist[k][threadIdx.x] = 0;
     __syncthreads();
     uint64_t first, count;
     cta_tiles(tiles, gridDim.x, blockIdx.x, first, count);
     const uint64_t begin = first * kSortTile;
     uint64_t end = (first + count) * kSortTile;
     if (end > nb) end = nb;
+    uint32_t* mine = hist[threadIdx.x >> 5];
     for (uint64_t i = begin + threadIdx.x; i < end; i += kSortThreads)
-        atomicAdd(&hist[(keys[i] >> shift) & mask], 1u);
+        atomicAdd(&mine[(keys[i] >> shift) & mask], 1u);
     __syncthreads();
-    counts[(uint64_t)threadIdx.x * gridDim.x + blockIdx.x] = hist[threadIdx.x];
+    uint32_t total = 0;
+    for (int k = 0; k < kSortWarps; ++k) total += hist[k][threadIdx.x];
+    counts[(uint64_t)threadIdx.x * gridDim.x + blockIdx.x] = total;
 }
 
-// ---- kernel 2: exclusive scan of counts[digit][cta] in digit-major order (one CTA)
-__global__ void __launch_bounds__(1024) sort_scan_kernel(uint32_t* counts, uint32_t n) {
-    __shared__ uint32_t partial[1024];
-    const uint32_t per = (n + 1023) / 1024;
-    const uint32_t lo = threadIdx.x * per;
-    const uint32_t hi = lo + per < n ? lo + per : n;
-    uint32_t sum = 0;
-    for (uint32_t i = lo; i < hi; ++i) sum += counts[i];
-    partial[threadIdx.x] = sum;
+// Exclusive scan of the 256 values held one per thread (value v of thread t): returns the sum
+// of the values of threads below t.  All 256 threads of the CTA call it; contains __syncthreads.
+__device__ __forceinline__ uint32_t cta_exclusive_scan_256(uint32_t v, uint32_t* warp_sums) {
+    const uint32_t lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    uint32_t inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t n = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+        if (lane >= (uint32_t)o) inc += n;
+    }
+    if (lane == 31) warp_sums[w] = inc;
     __syncthreads();
-    // Hillis-Steele inclusive scan over the 1024 partial sums
-    for (uint32_t offs = 1; offs < 1024; offs <<= 1) {
-        uint32_t v = threadIdx.x >= offs ? partial[threadIdx.x - offs] : 0;
-        __syncthreads();
-        partial[threadIdx.x] += v;
-        __syncthreads();
-    }
-    uint32_t run = partial[threadIdx.x] - sum;  // exclusive prefix of this thread's range
-    for (uint32_t i = lo; i < hi; ++i) {
-        uint32_t c = counts[i];
-        counts[i] = run;
-        run += c;
-    }
+    uint32_t before = 0;
+    for (uint32_t k = 0; k < w; ++k) before += warp_sums[k];
+    __syncthreads();  // warp_sums may be reused by the caller's next scan
+    return before + inc - v;
 }
 
-// ---- kernel 3: stable ranked scatter
+// ---- kernel 2: one CTA per digit: exclusive scan of that digit's per-CTA counts, in place, and
+// the digit's total into totals[digit]
 __global__ void __launch_bounds__(kSortThreads)
-sort_scatter_kernel(const uint32_t* kin, const uint32_t* vin, uint32_t* kout, uint32_t* vout,
-                    const uint32_t* offsets, uint64_t nb, uint64_t tiles, uint32_t shift,
-                    uint32_t mask) {
-    __shared__ uint32_t base[kRadix];
+sort_scan_kernel(uint32_t* counts, uint32_t* totals, uint32_t grid) {
+    __shared__ uint32_t warp_sums[kSortWarps];
+    uint32_t* row = counts + (uint64_t)blockIdx.x * grid;
+    uint32_t carry = 0;
+    for (uint32_t b0 = 0; b0 < grid; b0 += kSortThreads) {
+        const uint32_t b = b0 + threadIdx.x;
+        const uint32_t v = b < grid ? row[b] : 0u;
+        const uint32_t ex = cta_exclusive_scan_256(v, warp_sums);
+        if (b < grid) row[b] = carry + ex;
+        // total of this chunk = exclusive prefix of the last thread + its value
+        __shared__ uint32_t chunk_total;
+        if (threadIdx.x == kSortThreads - 1) chunk_total = ex + v;
+        __syncthreads();
+        carry += chunk_total;
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) totals[blockIdx.x] = carry;
+}
+
+// ---- kernel 3: stable ranked scatter.  Per tile of 4096 pairs: every warp ranks its 512 pairs
+// by digit (16 rounds of __match_any_sync, earlier rounds and lower lanes first), the ranks are
+// extended over the warps, the pairs are laid out in shared memory in (digit, original order),
+// and then written out so that each digit's pairs go to consecutive addresses.
+__global__ void __launch_bounds__(kSortThreads, 3)
+sort_scatter_kernel(const uint32_t* __restrict__ kin, const uint32_t* __restrict__ vin,
+                    uint32_t* __restrict__ kout, uint32_t* __restrict__ vout,
+                    const uint32_t* __restrict__ cta_offsets, const uint32_t* __restrict__ totals,
+                    uint64_t nb, uint64_t tiles, uint32_t shift, uint32_t mask) {
+    __shared__ uint32_t skey[kSortTile];
+    __shared__ uint32_t sval[kSortTile];
     __shared__ uint32_t wcnt[kSortWarps][kRadix];
+    __shared__ uint32_t base[kRadix];    // where the next pair of this digit goes, minus dstart
+    __shared__ uint32_t dstart[kRadix];  // start of the digit's run inside the tile
+    __shared__ uint32_t warp_sums[kSortWarps];
     const uint32_t lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     const uint32_t lt = (1u << lane) - 1u;
-    base[threadIdx.x] = offsets[(uint64_t)threadIdx.x * gridDim.x + blockIdx.x];
+    {
+        // start of this digit in the output = pairs of lower digits + this digit's pairs in
+        // lower CTAs
+        const uint32_t below = cta_exclusive_scan_256(totals[threadIdx.x], warp_sums);
+        base[threadIdx.x] = below + cta_offsets[(uint64_t)threadIdx.x * gridDim.x + blockIdx.x];
+    }
     uint64_t first, count;
     cta_tiles(tiles, gridDim.x, blockIdx.x, first, count);
     for (uint64_t t = first; t < first + count; ++t) {
         for (int k = 0; k < kSortWarps; ++k) wcnt[k][threadIdx.x] = 0;
         __syncthreads();
-        const uint64_t wbegin = t * kSortTile + (uint64_t)w * (32 * kSortItems);
+        const uint64_t tbegin = t * kSortTile;
+        const uint64_t wbegin = tbegin + (uint64_t)w * (32 * kSortItems);
         uint32_t key[kSortItems], rank[kSortItems];
 #pragma unroll
         for (int r = 0; r < kSortItems; ++r) {
             const uint64_t idx = wbegin + r * 32 + lane;
-            const bool valid = idx < nb;
-            key[r] = valid ? kin[idx] : 0u;
+            key[r] = idx < nb ? kin[idx] : 0u;
+        }
+#pragma unroll
+        for (int r = 0; r < kSortItems; ++r) {
+            const bool valid = wbegin + r * 32 + lane < nb;
             const uint32_t dg = valid ? ((key[r] >> shift) & mask) : (uint32_t)kRadix;
             const uint32_t peers = __match_any_sync(0xFFFFFFFFu, dg);
             uint32_t before = 0;
@@ -159,31 +199,41 @@ sort_scatter_kernel(const uint32_t* kin, const uint32_t* vin, uint32_t* kout, ui
             rank[r] = before + __popc(peers & lt);
         }
         __syncthreads();
-        // exclusive prefix over the warps of this tile, per digit
+        // per digit: exclusive prefix over the warps of this tile, and the tile's total
         uint32_t tile_total = 0;
-        {
-            uint32_t run = 0;
-            for (int k = 0; k < kSortWarps; ++k) {
-                uint32_t c = wcnt[k][threadIdx.x];
-                wcnt[k][threadIdx.x] = run;
-                run += c;
-            }
-            tile_total = run;
+        for (int k = 0; k < kSortWarps; ++k) {
+            const uint32_t c = wcnt[k][threadIdx.x];
+            wcnt[k][threadIdx.x] = tile_total;
+            tile_total += c;
         }
+        const uint32_t ds = cta_exclusive_scan_256(tile_total, warp_sums);  // syncs inside
+        dstart[threadIdx.x] = ds;
+        // from here base[] holds (output position of the digit's next pair) - (its position in
+        // the tile), so that a pair at tile position lp goes to base[digit] + lp
+        base[threadIdx.x] -= ds;
         __syncthreads();
 #pragma unroll
         for (int r = 0; r < kSortItems; ++r) {
             const uint64_t idx = wbegin + r * 32 + lane;
             if (idx < nb) {
                 const uint32_t dg = (key[r] >> shift) & mask;
-                const uint32_t dst = base[dg] + wcnt[w][dg] + rank[r];
-                kout[dst] = key[r];
-                vout[dst] = vin[idx];
+                const uint32_t lp = dstart[dg] + wcnt[w][dg] + rank[r];
+                skey[lp] = key[r];
+                sval[lp] = vin[idx];  // payloads are only passed through: read them this late
             }
         }
         __syncthreads();
-        base[threadIdx.x] += tile_total;
+        const uint32_t in_tile = (uint32_t)(nb - tbegin < (uint64_t)kSortTile ? nb - tbegin
+                                                                               : (uint64_t)kSortTile);
+        for (uint32_t lp = threadIdx.x; lp < in_tile; lp += kSortThreads) {
+            const uint32_t k = skey[lp];
+            const uint32_t dst = base[(k >> shift) & mask] + lp;
+            kout[dst] = k;
+            vout[dst] = sval[lp];
+        }
         __syncthreads();
+        base[threadIdx.x] += ds + tile_total;  // undo the shift, advance past this tile's pairs
+        // (the next tile's first barrier orders this update before its readers)
     }
 }
 
@@ -197,23 +247,29 @@ struct ApplyArgs {
     const int32_t* status;
 };
 
-// The term block (key, q) contributes to slot at in-block offset o, or nothing if o is past
-// the (possibly short) block.
-template <bool SIGN>
-__device__ __forceinline__ bool block_term(const ApplyArgs& a, const uint32_t* bag_of, uint32_t q,
+// The term that the sorted block with payload v contributes to the slot at in-block offset o
+// (o < Z), or nothing if o is past the end of a short last block.
+template <bool SIGN, bool SHORT>
+__device__ __forceinline__ bool block_term(const ApplyArgs& a, const uint32_t* bag_of, uint32_t v,
                                            uint32_t o, float& term) {
     const MapParams& mp = a.mp;
-    const uint32_t p = q / mp.C;
-    const uint32_t c = q - p * mp.C;
-    const uint32_t i = c * mp.Z + o;
-    if (o >= mp.Z || i >= mp.d) return false;
-    const uint64_t bag = bag_of ? (uint64_t)__ldg(bag_of + p) : (uint64_t)p;
-    term = __ldg(a.grad_out + bag * mp.d + i);
-    if (SIGN) {
-        const uint32_t e = table_of_bag(bag, mp);
-        const uint64_t x = (uint64_t)__ldg(a.indices + p);
-        term = sign_of(mp, hash_base(mp.g, e, x), i) * term;
+    if (!SIGN) {
+        // v = bag*d + c*Z: the block's first element in grad_out
+        if (SHORT) {
+            const uint32_t cz = v - (v / mp.d) * mp.d;
+            if (cz + o >= mp.d) return false;
+        }
+        term = __ldg(a.grad_out + (uint64_t)v + o);
+        return true;
     }
+    const uint32_t p = v / mp.C;  // v = q
+    const uint32_t c = v - p * mp.C;
+    const uint32_t i = c * mp.Z + o;
+    if (i >= mp.d) return false;
+    const uint64_t bag = bag_of ? (uint64_t)__ldg(bag_of + p) : (uint64_t)p;
+    const uint32_t e = table_of_bag(bag, mp);
+    const uint64_t x = (uint64_t)__ldg(a.indices + p);
+    term = sign_of(mp, hash_base(mp.g, e, x), i) * __ldg(a.grad_out + bag * mp.d + i);
     return true;
 }
 
@@ -223,90 +279,129 @@ __device__ __forceinline__ void commit_slot(float* target, uint32_t j, float acc
     else target[j] = __fadd_rn(target[j], acc);
 }
 
-// Slots j in [Z-1, m): thread (i, u) serves slot K[i]+u if sorted position i starts a run of
-// equal keys and no later run starts at or before that slot.
-template <bool SIGN, bool SGD>
+// Slots j in [Z-1, m).  The sorted blocks that reach slot j are those with key in [j-Z+1, j];
+// the slot is served from the FIRST of them: position i serves slot K[i]+u iff i starts a run of
+// equal keys and the previous key is below K[i]+u-Z+1, i.e. u >= Z - min(Z, K[i]-K[i-1]).  The
+// server then only walks forward through the sorted list, adding terms while the key stays <= j.
+//
+// One warp takes 32 consecutive sorted positions (a tile).  Keys and payloads live in a
+// warp-private ring of 128 positions in shared memory, filled by coalesced loads.  The lanes
+// cover (position, offset) pairs: G = min(Zp, 32) lanes per position (Zp = Z rounded up to a
+// power of two), 32/G positions at a time, Zp/G offset chunks per position.  For the pairs that
+// serve a slot, all lanes step through the ring together, UN positions per step: ring reads,
+// then the UN gradient loads, then the adds in sorted order; the next 32 positions are fetched
+// one step ahead of their first use.
+template <bool SIGN, bool SGD, bool SHORT>
 __global__ void __launch_bounds__(256)
 det_apply_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint32_t* __restrict__ V,
                  const uint32_t* __restrict__ bag_of, uint32_t log2Zp) {
+    constexpr int UN = 8;
+    constexpr uint32_t kRing = 128;
+    constexpr uint32_t kNoKey = 0xFFFFFFFFu;  // above every slot number (m + d <= 2^32)
+    __shared__ uint2 ring_s[8][kRing];
     if (a.status != nullptr && *a.status != 0) return;
     const MapParams& mp = a.mp;
-    const uint64_t tid = (uint64_t)blockIdx.x * 256 + threadIdx.x;
-    const uint64_t i = tid >> log2Zp;
-    const uint32_t u = (uint32_t)(tid & ((1u << log2Zp) - 1u));
-    if (i >= a.nb || u >= mp.Z) return;
-    const uint32_t kh = K[i];
-    if (i > 0 && K[i - 1] == kh) return;  // not the first of its run
-    const uint64_t j64 = (uint64_t)kh + u;
-    if (j64 >= mp.m || j64 + 1 < mp.Z) return;  // wrapped part / low slots: other kernel
-    const uint32_t j = (uint32_t)j64;
+    const uint32_t lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const uint64_t i0 = ((uint64_t)blockIdx.x * 8 + w) * 32;  // first position of the tile
+    if (i0 >= a.nb) return;                                   // whole warp
+    uint2* ring = ring_s[w];
 
-    // end of the run of kh (galloping, then bisection)
-    uint64_t lo = i, hi = i + 1, step = 1;
-    while (hi < a.nb && K[hi] == kh) {
-        lo = hi;
-        step <<= 1;
-        hi = lo + step;
-    }
-    if (hi > a.nb) hi = a.nb;
-    while (hi - lo > 1) {
-        const uint64_t mid = lo + ((hi - lo) >> 1);
-        if (K[mid] == kh) lo = mid; else hi = mid;
-    }
-    const uint64_t run_end = hi;
-    if (run_end < a.nb && K[run_end] <= j) return;  // a later run owns slot j
+    // (key, payload) of tile-relative position r, or a key above every slot past the end
+    auto fetch = [&](uint32_t r) -> uint2 {
+        const uint64_t idx = i0 + r;
+        if (idx >= a.nb) return make_uint2(kNoKey, 0u);
+        return make_uint2(__ldg(K + idx), __ldg(V + idx));
+    };
+    const uint2 mine = fetch(lane);
+    ring[lane] = mine;
+    ring[32 + lane] = fetch(32 + lane);
+    uint32_t loaded_end = 64;  // the ring holds positions [loaded_end - 128, loaded_end)
 
-    // first sorted position whose key reaches slot j: key >= j - (Z-1)
-    const uint32_t lowkey = j - (mp.Z - 1);
-    uint64_t first = i;
-    if (lowkey < kh && i > 0) {
-        uint64_t h2 = i, l2 = i;
-        bool found_low = false;
-        step = 1;
-        while (h2 > 0) {
-            const uint64_t probe = h2 >= step ? h2 - step : 0;
-            if (K[probe] >= lowkey) {
-                h2 = probe;
-                step <<= 1;
-            } else {
-                l2 = probe;
-                found_low = true;
-                break;
-            }
+    // first offset served from this lane's position (Z = none)
+    uint32_t kprev = __shfl_up_sync(0xFFFFFFFFu, mine.x, 1);
+    if (lane == 0 && i0 > 0) kprev = __ldg(K + i0 - 1);
+    uint32_t own_lo = mp.Z;
+    if (i0 + lane < a.nb) {
+        if (i0 + lane == 0) own_lo = 0;
+        else if (kprev != mine.x) {
+            const uint32_t gap = mine.x - kprev;
+            own_lo = gap >= mp.Z ? 0u : mp.Z - gap;
         }
-        if (found_low) {
-            while (h2 - l2 > 1) {
-                const uint64_t mid = l2 + ((h2 - l2) >> 1);
-                if (K[mid] >= lowkey) h2 = mid; else l2 = mid;
-            }
-        }
-        first = h2;
     }
+    __syncwarp();
 
-    float acc = 0.0f;
-    bool touched = false;
-    constexpr int PF = 4;
-    for (uint64_t ii = first; ii < run_end; ii += PF) {
-        float term[PF];
-        bool ok[PF];
+    const uint32_t log2G = log2Zp < 5 ? log2Zp : 5;
+    const uint32_t G = 1u << log2G, EPW = 32u >> log2G, CH = 1u << (log2Zp - log2G);
+    const uint32_t sub = lane >> log2G, ul = lane & (G - 1);
+
+    for (uint32_t eb = 0; eb < 32; eb += EPW) {
+        const uint32_t e = eb + sub;
+        const uint32_t lo_e = __shfl_sync(0xFFFFFFFFu, own_lo, e);
+        const uint32_t s = __shfl_sync(0xFFFFFFFFu, mine.x, e);
+        for (uint32_t ch = 0; ch < CH; ++ch) {
+            const uint32_t u = ch * G + ul;
+            const uint64_t j64 = (uint64_t)s + u;
+            // j64 >= m: wrapped part, j64 < Z-1: low slots - both belong to the other kernel
+            const bool active = u >= lo_e && u < mp.Z && j64 < mp.m && j64 + 1 >= mp.Z;
+            if (__ballot_sync(0xFFFFFFFFu, active) == 0) continue;
+            const uint32_t j = (uint32_t)j64;
+            float old = 0.0f;
+            if (active) old = a.target[j];
+
+            if (loaded_end > eb + kRing) {  // an earlier long walk moved the ring past this tile
+                __syncwarp();
+                ring[lane] = mine;
+                ring[32 + lane] = fetch(32 + lane);
+                loaded_end = 64;
+                __syncwarp();
+            }
+
+            float acc = 0.0f;
+            bool touched = false, done = !active, pending = false;
+            uint2 ahead = make_uint2(kNoKey, 0u);
+            for (uint32_t fbase = eb;; fbase += UN) {
+                if (pending) {  // the positions fetched one step ago enter the ring
+                    __syncwarp();
+                    ring[(loaded_end + lane) & (kRing - 1)] = ahead;
+                    loaded_end += 32;
+                    pending = false;
+                    __syncwarp();
+                }
+                // the next step reads up to position fbase + UN + (EPW-1) + (UN-1)
+                if (loaded_end <= fbase + 2 * UN + EPW - 2) {
+                    ahead = fetch(loaded_end + lane);
+                    pending = true;
+                }
+                uint2 kv[UN];
 #pragma unroll
-        for (int t = 0; t < PF; ++t) {
-            ok[t] = false;
-            if (ii + t < run_end) ok[t] = block_term<SIGN>(a, bag_of, V[ii + t], j - K[ii + t], term[t]);
-        }
+                for (int t = 0; t < UN; ++t) kv[t] = ring[(fbase + sub + t) & (kRing - 1)];
+                float term[UN];
+                bool ok[UN];
+                bool in_last = false;
 #pragma unroll
-        for (int t = 0; t < PF; ++t)
-            if (ok[t]) {
-                acc = __fadd_rn(acc, term[t]);
-                touched = true;
+                for (int t = 0; t < UN; ++t) {
+                    const bool in = !done && kv[t].x <= j;  // sorted: true on a prefix
+                    ok[t] = false;
+                    if (in) ok[t] = block_term<SIGN, SHORT>(a, bag_of, kv[t].y, j - kv[t].x, term[t]);
+                    if (t == UN - 1) in_last = in;
+                }
+#pragma unroll
+                for (int t = 0; t < UN; ++t)
+                    if (ok[t]) {
+                        acc = __fadd_rn(acc, term[t]);
+                        touched = true;
+                    }
+                done = done || !in_last;
+                if (__ballot_sync(0xFFFFFFFFu, !done) == 0) break;
             }
+            if (touched) a.target[j] = SGD ? __fmaf_rn(-a.lr, acc, old) : __fadd_rn(old, acc);
+        }
     }
-    if (touched) commit_slot<SGD>(a.target, j, acc, a.lr);
 }
 
 // Slots j in [0, Z-1): plain blocks with key <= j first, then the wrapped tails of blocks
 // whose key lies in [m + j - (Z-1), m-1] (o = j + m - key).
-template <bool SIGN, bool SGD>
+template <bool SIGN, bool SGD, bool SHORT>
 __global__ void __launch_bounds__(128)
 det_apply_low_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint32_t* __restrict__ V,
                      const uint32_t* __restrict__ bag_of) {
@@ -316,7 +411,7 @@ det_apply_low_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint32_t
         float acc = 0.0f, term;
         bool touched = false;
         for (uint64_t ii = 0; ii < a.nb && K[ii] <= j; ++ii)
-            if (block_term<SIGN>(a, bag_of, V[ii], j - K[ii], term)) {
+            if (block_term<SIGN, SHORT>(a, bag_of, V[ii], j - K[ii], term)) {
                 acc = __fadd_rn(acc, term);
                 touched = true;
             }
@@ -327,7 +422,7 @@ det_apply_low_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint32_t
             if (K[mid] >= lowkey) hi = mid; else lo = mid + 1;
         }
         for (uint64_t ii = lo; ii < a.nb; ++ii)
-            if (block_term<SIGN>(a, bag_of, V[ii], j + (mp.m - K[ii]), term)) {
+            if (block_term<SIGN, SHORT>(a, bag_of, V[ii], j + (mp.m - K[ii]), term)) {
                 acc = __fadd_rn(acc, term);
                 touched = true;
             }
@@ -342,7 +437,7 @@ uint32_t bits_for(uint32_t m) {  // bits needed for keys in [0, m)
 }
 
 struct Layout {
-    size_t keysA, keysB, valsA, valsB, bag_of, counts, total;
+    size_t keysA, keysB, valsA, valsB, bag_of, counts, totals, total;
 };
 
 Layout make_layout(uint64_t nb, int64_t nnz, bool bags) {
@@ -355,8 +450,25 @@ Layout make_layout(uint64_t nb, int64_t nnz, bool bags) {
     L.valsB = off; off += kb;
     L.bag_of = off; off += bags ? align256((size_t)(nnz ? nnz : 1) * sizeof(uint32_t)) : 0;
     L.counts = off; off += align256((size_t)kRadix * kSortMaxGrid * sizeof(uint32_t));
+    L.totals = off; off += align256((size_t)kRadix * sizeof(uint32_t));
     L.total = off;
     return L;
+}
+
+template <bool SIGN, bool SGD>
+void launch_apply(const ApplyArgs& aa, const uint32_t* K, const uint32_t* V, const uint32_t* bag_of,
+                  cudaStream_t st) {
+    const MapParams& mp = aa.mp;
+    uint32_t log2Zp = 0;
+    while ((1u << log2Zp) < mp.Z) ++log2Zp;
+    const unsigned blocks = (unsigned)((aa.nb + 255) / 256);  // one warp per 32 sorted positions
+    if (mp.d % mp.Z != 0) {
+        det_apply_kernel<SIGN, SGD, true><<<blocks, 256, 0, st>>>(aa, K, V, bag_of, log2Zp);
+        if (mp.Z > 1) det_apply_low_kernel<SIGN, SGD, true><<<1, 128, 0, st>>>(aa, K, V, bag_of);
+    } else {
+        det_apply_kernel<SIGN, SGD, false><<<blocks, 256, 0, st>>>(aa, K, V, bag_of, log2Zp);
+        if (mp.Z > 1) det_apply_low_kernel<SIGN, SGD, false><<<1, 128, 0, st>>>(aa, K, V, bag_of);
+    }
 }
 
 }  // namespace
@@ -376,6 +488,8 @@ cudaError_t launch_backward_det(const Problem& pb, const float* grad_out, float*
     const uint64_t nb = (uint64_t)pb.nnz * mp.C;
     const Layout L = make_layout(nb, pb.nnz, bags);
     if (workspace == nullptr || workspace_bytes < L.total) return cudaErrorInvalidValue;
+    // the payload of a block is a 32-bit position in grad_out
+    if ((uint64_t)pb.nbags * mp.d > (1ull << 32)) return cudaErrorInvalidValue;
     char* ws = (char*)workspace;
     uint32_t* kA = (uint32_t*)(ws + L.keysA);
     uint32_t* kB = (uint32_t*)(ws + L.keysB);
@@ -383,6 +497,7 @@ cudaError_t launch_backward_det(const Problem& pb, const float* grad_out, float*
     uint32_t* vB = (uint32_t*)(ws + L.valsB);
     uint32_t* bag_of = bags ? (uint32_t*)(ws + L.bag_of) : nullptr;
     uint32_t* counts = (uint32_t*)(ws + L.counts);
+    uint32_t* totals = (uint32_t*)(ws + L.totals);
 
     KeyArgs ka{mp, pb.indices, pb.offsets, pb.nbags, pb.nnz, pb.status};
     if (bags) {
@@ -390,7 +505,10 @@ cudaError_t launch_backward_det(const Problem& pb, const float* grad_out, float*
         cudaMemsetAsync(bag_of, 0, (size_t)pb.nnz * sizeof(uint32_t), st);
         det_bag_of_kernel<<<(unsigned)((pb.nbags + 7) / 8), 256, 0, st>>>(ka, bag_of);
     }
-    det_keys_kernel<<<(unsigned)((nb + 255) / 256), 256, 0, st>>>(ka, bag_of, kA, vA, nb);
+    if (pb.sign)
+        det_keys_kernel<true><<<(unsigned)((nb + 255) / 256), 256, 0, st>>>(ka, bag_of, kA, vA, nb);
+    else
+        det_keys_kernel<false><<<(unsigned)((nb + 255) / 256), 256, 0, st>>>(ka, bag_of, kA, vA, nb);
 
     const SortPlan sp = make_plan(nb);
     const uint32_t bits = bits_for(mp.m);
@@ -401,29 +519,21 @@ cudaError_t launch_backward_det(const Problem& pb, const float* grad_out, float*
         const uint32_t width = bits - shift < bpp ? bits - shift : bpp;
         const uint32_t mask = (1u << width) - 1u;
         sort_count_kernel<<<sp.grid, kSortThreads, 0, st>>>(kA, counts, nb, sp.tiles, shift, mask);
-        sort_scan_kernel<<<1, 1024, 0, st>>>(counts, (uint32_t)kRadix * sp.grid);
-        sort_scatter_kernel<<<sp.grid, kSortThreads, 0, st>>>(kA, vA, kB, vB, counts, nb, sp.tiles,
-                                                             shift, mask);
+        sort_scan_kernel<<<kRadix, kSortThreads, 0, st>>>(counts, totals, sp.grid);
+        sort_scatter_kernel<<<sp.grid, kSortThreads, 0, st>>>(kA, vA, kB, vB, counts, totals, nb,
+                                                             sp.tiles, shift, mask);
         uint32_t* t = kA; kA = kB; kB = t;
         t = vA; vA = vB; vB = t;
     }
 
     ApplyArgs aa{mp, grad_out, pb.indices, target, lr, nb, pb.status};
-    uint32_t log2Zp = 0;
-    while ((1u << log2Zp) < mp.Z) ++log2Zp;
-    const uint64_t threads = nb << log2Zp;
-    const unsigned blocks = (unsigned)((threads + 255) / 256);
-#define ROBE_DET_LAUNCH(SIGN, SGD)                                                        \
-    do {                                                                                  \
-        det_apply_kernel<SIGN, SGD><<<blocks, 256, 0, st>>>(aa, kA, vA, bag_of, log2Zp);   \
-        if (mp.Z > 1) det_apply_low_kernel<SIGN, SGD><<<1, 128, 0, st>>>(aa, kA, vA, bag_of); \
-    } while (0)
     if (pb.sign) {
-        if (sgd) ROBE_DET_LAUNCH(true, true); else ROBE_DET_LAUNCH(true, false);
+        if (sgd) launch_apply<true, true>(aa, kA, vA, bag_of, st);
+        else launch_apply<true, false>(aa, kA, vA, bag_of, st);
     } else {
-        if (sgd) ROBE_DET_LAUNCH(false, true); else ROBE_DET_LAUNCH(false, false);
+        if (sgd) launch_apply<false, true>(aa, kA, vA, bag_of, st);
+        else launch_apply<false, false>(aa, kA, vA, bag_of, st);
     }
-#undef ROBE_DET_LAUNCH
     return cudaGetLastError();
 }
 
