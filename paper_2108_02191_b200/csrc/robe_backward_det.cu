@@ -289,40 +289,173 @@ __device__ __forceinline__ void commit_slot(float* target, uint32_t j, float acc
 // cover (position, offset) pairs: G = min(Zp, 32) lanes per position (Zp = Z rounded up to a
 // power of two), 32/G positions at a time, Zp/G offset chunks per position.  For the pairs that
 // serve a slot, all lanes step through the ring together, UN positions per step: ring reads,
-// then the UN gradient loads, then the adds in sorted order; the next 32 positions are fetched
-// one step ahead of their first use.
+// then the gradient loads, then the adds in sorted order; the next 32 positions are fetched one
+// step ahead of their first use.  A walk that is still going after 64 positions (an id that
+// occurs many times in the batch) goes on 32 positions per step, with the gradient rows of the
+// positions after those asked into L2 ahead of time, so that its chain of dependent adds waits
+// for memory once per 32 terms.
+#ifndef ROBE_DEEP_UN
+#define ROBE_DEEP_UN 16
+#endif
+constexpr uint32_t kRing = 128;
+constexpr uint32_t kNoKey = 0xFFFFFFFFu;  // above every slot number (m + d <= 2^32)
+
+struct ApplyTile {
+    const uint32_t* K;
+    const uint32_t* V;
+    uint64_t nb;
+    uint64_t i0;          // first sorted position of the tile
+    uint2* ring;          // warp-private, kRing entries
+    uint32_t loaded_end;  // the ring holds tile-relative positions [loaded_end - kRing, loaded_end)
+    // (key, payload) of tile-relative position r, or a key above every slot past the end
+    __device__ __forceinline__ uint2 fetch(uint32_t r) const {
+        const uint64_t idx = i0 + r;
+        if (idx >= nb) return make_uint2(kNoKey, 0u);
+        return make_uint2(__ldg(K + idx), __ldg(V + idx));
+    }
+};
+
+struct ApplyWalk {
+    float acc;
+    bool touched, done, pending;
+    uint2 ahead;     // positions [loaded_end, loaded_end + 32), fetched but not yet in the ring
+    uint32_t fbase;  // the next step starts at tile-relative position fbase + sub
+};
+
+// The positions fetched last enter the ring.  pf != nullptr: their gradient rows are asked
+// into L2 (pf = grad_out + the first offset of the lanes' chunk).
+__device__ __forceinline__ void walk_commit(ApplyTile& tl, ApplyWalk& wk, uint32_t lane,
+                                            const float* pf) {
+    __syncwarp();
+    tl.ring[(tl.loaded_end + lane) & (kRing - 1)] = wk.ahead;
+    if (pf != nullptr && wk.ahead.x != kNoKey)
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(pf + wk.ahead.y));
+    tl.loaded_end += 32;
+    wk.pending = false;
+    __syncwarp();
+}
+
+// Start of a step of UN positions: the positions fetched one step ago enter the ring, and the
+// ones the step after this one will read are fetched.
+template <int UN>
+__device__ __forceinline__ void walk_advance(ApplyTile& tl, ApplyWalk& wk, uint32_t EPW,
+                                             uint32_t lane, const float* pf) {
+    if (wk.pending) walk_commit(tl, wk, lane, pf);
+    // the next step reads up to position fbase + UN + (EPW-1) + (UN-1)
+    if (tl.loaded_end <= wk.fbase + 2 * UN + EPW - 2) {
+        wk.ahead = tl.fetch(tl.loaded_end + lane);
+        wk.pending = true;
+    }
+}
+
+// Steps of UN positions until no lane goes on, or (limit != 0) until fbase reaches limit.
+// Returns whether every lane is done.
+template <bool SIGN, bool SHORT, int UN>
+__device__ __forceinline__ bool walk_steps(const ApplyArgs& a, const uint32_t* bag_of, ApplyTile& tl,
+                                           ApplyWalk& wk, uint32_t j, uint32_t sub, uint32_t EPW,
+                                           uint32_t lane, uint32_t limit) {
+    for (;; wk.fbase += UN) {
+        if (limit != 0 && wk.fbase >= limit) return false;
+        walk_advance<UN>(tl, wk, EPW, lane, nullptr);
+        uint2 kv[UN];
+#pragma unroll
+        for (int t = 0; t < UN; ++t) kv[t] = tl.ring[(wk.fbase + sub + t) & (kRing - 1)];
+        float term[UN];
+        bool ok[UN];
+        bool in_last = false;
+#pragma unroll
+        for (int t = 0; t < UN; ++t) {
+            const bool in = !wk.done && kv[t].x <= j;  // sorted: true on a prefix
+            ok[t] = false;
+            if (in) ok[t] = block_term<SIGN, SHORT>(a, bag_of, kv[t].y, j - kv[t].x, term[t]);
+            if (t == UN - 1) in_last = in;
+        }
+#pragma unroll
+        for (int t = 0; t < UN; ++t)
+            if (ok[t]) {
+                wk.acc = __fadd_rn(wk.acc, term[t]);
+                wk.touched = true;
+            }
+        wk.done = wk.done || !in_last;
+        if (__ballot_sync(0xFFFFFFFFu, !wk.done) == 0) {
+            wk.fbase += UN;
+            return true;
+        }
+    }
+}
+
+// The same for a long walk of plain blocks (sign off, no short last block): more positions per
+// step, each term's place in grad_out computed while its key is compared.
+__device__ __forceinline__ void walk_deep(const ApplyArgs& a, ApplyTile& tl, ApplyWalk& wk, uint32_t j,
+                                          uint32_t sub, uint32_t EPW, uint32_t lane,
+                                          uint32_t chunk_off) {
+    constexpr int UN = ROBE_DEEP_UN;
+    const float* pf = a.grad_out + chunk_off;
+    // the ring has to reach the end of the first step before the one-step-ahead fetches take over
+    if (wk.pending) walk_commit(tl, wk, lane, pf);
+    while (tl.loaded_end < wk.fbase + EPW + UN - 1) {
+        wk.ahead = tl.fetch(tl.loaded_end + lane);
+        walk_commit(tl, wk, lane, pf);
+    }
+    for (;; wk.fbase += UN) {
+        walk_advance<UN>(tl, wk, EPW, lane, pf);
+        uint32_t at[UN];
+        uint32_t n_in = 0;
+#pragma unroll
+        for (int t = 0; t < UN; ++t) {
+            const uint2 e = tl.ring[(wk.fbase + sub + t) & (kRing - 1)];
+            n_in += (!wk.done && e.x <= j) ? 1u : 0u;  // sorted: a prefix of the step
+            at[t] = e.y + (j - e.x);
+        }
+        const uint32_t n_max = __reduce_max_sync(0xFFFFFFFFu, n_in);  // warp-uniform
+        float term[UN];
+#pragma unroll
+        for (int t = 0; t < UN; ++t) {
+            term[t] = 0.0f;
+            if ((uint32_t)t < n_max) {
+                if ((uint32_t)t < n_in) term[t] = __ldg(a.grad_out + at[t]);
+            }
+        }
+#pragma unroll
+        for (int t = 0; t < UN; ++t) {
+            if ((uint32_t)t < n_max) {
+                if ((uint32_t)t < n_in) wk.acc = __fadd_rn(wk.acc, term[t]);
+            }
+        }
+        if (n_in != 0) wk.touched = true;
+        wk.done = wk.done || n_in < (uint32_t)UN;
+        if (n_max < (uint32_t)UN) return;  // no lane goes on
+    }
+}
+
 template <bool SIGN, bool SGD, bool SHORT>
 __global__ void __launch_bounds__(256)
 det_apply_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint32_t* __restrict__ V,
                  const uint32_t* __restrict__ bag_of, uint32_t log2Zp) {
     constexpr int UN = 8;
-    constexpr uint32_t kRing = 128;
-    constexpr uint32_t kNoKey = 0xFFFFFFFFu;  // above every slot number (m + d <= 2^32)
+    constexpr uint32_t kDeepAfter = 64;  // positions after which a walk counts as long
     __shared__ uint2 ring_s[8][kRing];
     if (a.status != nullptr && *a.status != 0) return;
     const MapParams& mp = a.mp;
     const uint32_t lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-    const uint64_t i0 = ((uint64_t)blockIdx.x * 8 + w) * 32;  // first position of the tile
-    if (i0 >= a.nb) return;                                   // whole warp
-    uint2* ring = ring_s[w];
-
-    // (key, payload) of tile-relative position r, or a key above every slot past the end
-    auto fetch = [&](uint32_t r) -> uint2 {
-        const uint64_t idx = i0 + r;
-        if (idx >= a.nb) return make_uint2(kNoKey, 0u);
-        return make_uint2(__ldg(K + idx), __ldg(V + idx));
-    };
-    const uint2 mine = fetch(lane);
-    ring[lane] = mine;
-    ring[32 + lane] = fetch(32 + lane);
-    uint32_t loaded_end = 64;  // the ring holds positions [loaded_end - 128, loaded_end)
+    ApplyTile tl;
+    tl.K = K;
+    tl.V = V;
+    tl.nb = a.nb;
+    tl.i0 = ((uint64_t)blockIdx.x * 8 + w) * 32;
+    if (tl.i0 >= a.nb) return;  // whole warp
+    tl.ring = ring_s[w];
+    const uint2 mine = tl.fetch(lane);
+    tl.ring[lane] = mine;
+    tl.ring[32 + lane] = tl.fetch(32 + lane);
+    tl.loaded_end = 64;
 
     // first offset served from this lane's position (Z = none)
     uint32_t kprev = __shfl_up_sync(0xFFFFFFFFu, mine.x, 1);
-    if (lane == 0 && i0 > 0) kprev = __ldg(K + i0 - 1);
+    if (lane == 0 && tl.i0 > 0) kprev = __ldg(K + tl.i0 - 1);
     uint32_t own_lo = mp.Z;
-    if (i0 + lane < a.nb) {
-        if (i0 + lane == 0) own_lo = 0;
+    if (tl.i0 + lane < a.nb) {
+        if (tl.i0 + lane == 0) own_lo = 0;
         else if (kprev != mine.x) {
             const uint32_t gap = mine.x - kprev;
             own_lo = gap >= mp.Z ? 0u : mp.Z - gap;
@@ -348,53 +481,28 @@ det_apply_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint32_t* __
             float old = 0.0f;
             if (active) old = a.target[j];
 
-            if (loaded_end > eb + kRing) {  // an earlier long walk moved the ring past this tile
+            if (tl.loaded_end > eb + kRing) {  // an earlier long walk moved the ring past this tile
                 __syncwarp();
-                ring[lane] = mine;
-                ring[32 + lane] = fetch(32 + lane);
-                loaded_end = 64;
+                tl.ring[lane] = mine;
+                tl.ring[32 + lane] = tl.fetch(32 + lane);
+                tl.loaded_end = 64;
                 __syncwarp();
             }
 
-            float acc = 0.0f;
-            bool touched = false, done = !active, pending = false;
-            uint2 ahead = make_uint2(kNoKey, 0u);
-            for (uint32_t fbase = eb;; fbase += UN) {
-                if (pending) {  // the positions fetched one step ago enter the ring
-                    __syncwarp();
-                    ring[(loaded_end + lane) & (kRing - 1)] = ahead;
-                    loaded_end += 32;
-                    pending = false;
-                    __syncwarp();
-                }
-                // the next step reads up to position fbase + UN + (EPW-1) + (UN-1)
-                if (loaded_end <= fbase + 2 * UN + EPW - 2) {
-                    ahead = fetch(loaded_end + lane);
-                    pending = true;
-                }
-                uint2 kv[UN];
-#pragma unroll
-                for (int t = 0; t < UN; ++t) kv[t] = ring[(fbase + sub + t) & (kRing - 1)];
-                float term[UN];
-                bool ok[UN];
-                bool in_last = false;
-#pragma unroll
-                for (int t = 0; t < UN; ++t) {
-                    const bool in = !done && kv[t].x <= j;  // sorted: true on a prefix
-                    ok[t] = false;
-                    if (in) ok[t] = block_term<SIGN, SHORT>(a, bag_of, kv[t].y, j - kv[t].x, term[t]);
-                    if (t == UN - 1) in_last = in;
-                }
-#pragma unroll
-                for (int t = 0; t < UN; ++t)
-                    if (ok[t]) {
-                        acc = __fadd_rn(acc, term[t]);
-                        touched = true;
-                    }
-                done = done || !in_last;
-                if (__ballot_sync(0xFFFFFFFFu, !done) == 0) break;
+            ApplyWalk wk;
+            wk.acc = 0.0f;
+            wk.touched = false;
+            wk.done = !active;
+            wk.pending = false;
+            wk.ahead = make_uint2(kNoKey, 0u);
+            wk.fbase = eb;
+            if (!SIGN && !SHORT) {
+                if (!walk_steps<SIGN, SHORT, UN>(a, bag_of, tl, wk, j, sub, EPW, lane, eb + kDeepAfter))
+                    walk_deep(a, tl, wk, j, sub, EPW, lane, ch * G);
+            } else {
+                walk_steps<SIGN, SHORT, UN>(a, bag_of, tl, wk, j, sub, EPW, lane, 0);
             }
-            if (touched) a.target[j] = SGD ? __fmaf_rn(-a.lr, acc, old) : __fadd_rn(old, acc);
+            if (wk.touched) a.target[j] = SGD ? __fmaf_rn(-a.lr, wk.acc, old) : __fadd_rn(old, wk.acc);
         }
     }
 }
