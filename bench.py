@@ -130,6 +130,24 @@ def visible_gpu_index(local_rank: int) -> int:
     return local_rank
 
 
+def rank_batch_variants(rank: int, nb: int):
+    """Seeds of the id batches of one rank: every rank draws its own shard of the global batch
+    (data parallel by sample), so no two ranks ever share a variant number."""
+    return [1000 * rank + v for v in range(nb)]
+
+
+def aggregate_over_ranks(dist, device, times_ms, units):
+    """Whole-job figures from per-rank ones: every time becomes the MAXIMUM over ranks, the units
+    of work (ids) the SUM over ranks.  `dist` is torch.distributed or None for one process; the
+    reductions are the only communication of the benchmark (the data path has none)."""
+    t = torch.tensor([float(v) for v in times_ms], dtype=torch.float64, device=device)
+    u = torch.tensor([float(v) for v in units], dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return [float(v) for v in t.tolist()], [float(v) for v in u.tolist()]
+
+
 def pick_workload(name: str):
     table = {
         "cfg2": synth.workload(2), "cfg3_z1": synth.workload(3, Z=1), "cfg3_z128": synth.workload(3, Z=128),
@@ -211,9 +229,8 @@ def run_ours(args, w):
     B, T, d = w.batch, w.num_tables, w.d
     nbags = B * T
     batches = []
-    for v in range(NB):
-        ids, offs = synth.make_ids(w, B, variant=1000 * rank + v)
-        batches.append((ids, offs))
+    for v in rank_batch_variants(rank, NB):
+        batches.append(synth.make_ids(w, B, variant=v))
     array = synth.make_array(w, dev)
     gen = torch.Generator(device=dev)
     gen.manual_seed(w.data_seed + 17 * rank)
@@ -299,10 +316,9 @@ def run_ours(args, w):
     d2h = int(4 * nbags * d)
 
     # ---- max over ranks --------------------------------------------------------------------
-    times = torch.tensor([total_ms, e2e_ms, fwd_ms, bwd_ms], dtype=torch.float64, device=dev)
-    if dist is not None:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    total_ms, e2e_ms, fwd_ms, bwd_ms = [float(v) for v in times.tolist()]
+    (total_ms, e2e_ms, fwd_ms, bwd_ms), (job_ids, job_e2e_ids) = aggregate_over_ranks(
+        dist, dev, [total_ms, e2e_ms, fwd_ms, bwd_ms],
+        [nnz_per_step * args.steps, e2e_nnz * e2e_steps])
 
     robe.robe_destroy(h)
     if rank != 0:
@@ -322,7 +338,7 @@ def run_ours(args, w):
                 "frac": ach / peak, "peak_kind": f"of {peak_kind}", "traffic": traffic.get(which),
                 "ms_per_launch": ms, "algorithmic_bytes": int(nbytes)}
 
-    value = world * nnz_per_step * args.steps / (total_ms * 1e-3)
+    value = job_ids / (total_ms * 1e-3)
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
@@ -332,7 +348,7 @@ def run_ours(args, w):
                    "l2": "1 GB array and 4 rotated id batches exceed L2; no flush",
                    "parallelism": f"dp{world} replicas, no collective"},
         "clocks": clocks,
-        "e2e": {"value": world * e2e_nnz * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT,
+        "e2e": {"value": job_e2e_ids / (e2e_ms * 1e-3), "unit": UNIT,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
                 "ms_per_step": e2e_ms / e2e_steps},
         "gpu_launches": 2 * args.steps,
@@ -343,11 +359,11 @@ def run_ours(args, w):
                          "bags_per_s": world * nbags / (fwd_ms * 1e-3), "ms": fwd_ms},
     }
     if not args.no_cpu_baseline and world == 1:
-        sample_batch = max(1, w.batch // 8)
+        sample_batch = w.batch  # about 10 s of host work on the default workload
         rate, n, threads, dt = oracle_step_rate(w, sample_batch, synth.array_to_numpy(array), variant=7)
         line["cpu_baseline"] = {"value": rate, "unit": UNIT, "cores": threads, "kind": "oracle",
-                                "sample": f"{sample_batch} of {w.batch} samples ({n} ids), forward + "
-                                          f"fp64 backward, {dt:.1f} s"}
+                                "sample": f"{sample_batch} of {w.batch} samples ({n} ids), forward "
+                                          f"({threads} threads) + fp64 backward (1 thread), {dt:.1f} s"}
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()

@@ -94,7 +94,7 @@ def assert_bits_equal(a: np.ndarray, b: np.ndarray, what=""):
 
 
 def assert_within_l1(got: np.ndarray, delta64: np.ndarray, l1: np.ndarray, scale=1.0, what=""):
-    """spec tolerance: |got - ref| <= 1e-5 * scale * L1 mass per slot (exactly equal
+    """Tolerance of the atomic backward: |got - ref| <= 1e-5 * scale * L1 mass per slot (exactly equal
     where no gradient landed)."""
     err = np.abs(got.astype(np.float64) - delta64)
     tol = 1e-5 * scale * l1
