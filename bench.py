@@ -35,10 +35,12 @@ from paper_2108_02191_b200 import synth  # noqa: E402
 METRIC = "robe_lookups_per_s_fwd_bwd"
 UNIT = "ids/s"
 
-# DRAM bytes per launch of the dominant kernel of the default workload, from the ncu capture
-# summarised under profiles/ (dram__bytes_read.sum + dram__bytes_write.sum); None = not captured.
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu capture of the
+# full-size default workload that profiles/dram_traffic_cfg4_multihot.md summarises; None = not
+# captured for that workload or backward variant.
 NCU_TRAFFIC_BYTES = {
-    "cfg4_multihot": {"forward": None, "backward": None},
+    ("cfg4_multihot", "atomic"): {"forward": 4_155_085_568, "backward": 7_510_767_360},
+    ("cfg4_multihot", "det"): {"forward": 4_155_085_568, "backward": None},
 }
 
 
@@ -148,12 +150,31 @@ def aggregate_over_ranks(dist, device, times_ms, units):
     return [float(v) for v in t.tolist()], [float(v) for v in u.tolist()]
 
 
+WORKLOAD_HELP = ("cfg2 | cfg3_z<Z> | cfg4 | cfg5_<1m|100m|10g>_z<Z>[_bf16]  (cfg5 = cfg5_100m_z32); "
+                 "cfg4 is the headline workload, the others are the parity-test shapes")
+
+
 def pick_workload(name: str):
-    table = {
-        "cfg2": synth.workload(2), "cfg3_z1": synth.workload(3, Z=1), "cfg3_z128": synth.workload(3, Z=128),
-        "cfg4": synth.workload(4), "cfg5": synth.workload(5),
-    }
-    return table[name]
+    """A workload by name, see WORKLOAD_HELP."""
+    if name == "cfg2":
+        return synth.workload(2)
+    if name == "cfg4":
+        return synth.workload(4)
+    if name == "cfg5":
+        return synth.workload(5)
+    parts = name.split("_")
+    if parts[0] == "cfg3" and len(parts) == 2 and parts[1].startswith("z"):
+        return synth.workload(3, Z=int(parts[1][1:])).with_(name=name)
+    if parts[0] == "cfg5" and len(parts) in (3, 4) and parts[2].startswith("z"):
+        M = {"1m": 262_144, "100m": 25_000_000, "10g": 2_500_000_000}[parts[1]]
+        kw = dict(M=M, Z=int(parts[2][1:]))
+        if len(parts) == 4:
+            if parts[3] != "bf16":
+                raise ValueError(name)
+            kw["array_dtype"] = "bf16"
+        w = synth.workload(5, **kw)
+        return w.with_(name=name)
+    raise ValueError(f"unknown workload {name!r}: {WORKLOAD_HELP}")
 
 
 # -------------------------------------------------------------------------------------------
@@ -242,6 +263,18 @@ def run_ours(args, w):
     h = robe.robe_create(w.M, w.Z, w.d, T, w.hash_seed)
     robe.robe_attach_array(h, array)
     lr = 1.0  # the paper trains its DLRM with plain SGD at learning rate 1.0 (Section 5)
+    ws = None
+    bwd_launches = 1
+    # a bf16 array is read-only for the library: its gradient goes to a dense fp32 array instead
+    # of the fused SGD step (the array stays as it is)
+    dense = torch.zeros(w.M, dtype=torch.float32, device=dev) if w.array_dtype != "f32" else None
+    if args.backward == "det":
+        robe.robe_set_option(h, robe.ROBE_OPT_BWD_MODE, robe.ROBE_BWD_DETERMINISTIC)
+        ws = torch.empty(robe.robe_backward_workspace_bytes(h, B, max(len(b[0]) for b in batches)),
+                         dtype=torch.uint8, device=dev)
+        # keys (+ bag numbers), three kernels per 8-bit sort pass, apply (+ the low-slot kernel)
+        npass = -(-max(1, (w.M - 1).bit_length()) // 8)
+        bwd_launches = (1 if bags else 0) + 1 + 3 * npass + 1 + (1 if w.Z > 1 else 0)
 
     def step(i, events=None):
         k = i % NB
@@ -250,7 +283,7 @@ def run_ours(args, w):
         robe.robe_forward(h, d_ids[k], d_offs[k], B, out)
         if events is not None:
             events[1].record()
-        robe.robe_backward(h, grad_out, d_ids[k], d_offs[k], B, None, lr, None)
+        robe.robe_backward(h, grad_out, d_ids[k], d_offs[k], B, dense, lr, ws)
         if events is not None:
             events[2].record()
 
@@ -297,7 +330,7 @@ def run_ours(args, w):
             e_offs.copy_(h_offs[k], non_blocking=True)
         e_grad.copy_(h_grad, non_blocking=True)
         robe.robe_forward(h, ids_d, e_offs, B, out)
-        robe.robe_backward(h, e_grad, ids_d, e_offs, B, None, lr, None)
+        robe.robe_backward(h, e_grad, ids_d, e_offs, B, dense, lr, ws)
         h_out.copy_(out, non_blocking=True)
 
     e2e_steps = max(3, min(args.steps, 10))
@@ -330,7 +363,7 @@ def run_ours(args, w):
     fwd_bytes, bwd_bytes = algorithmic_bytes(w, nbags, nnz_per_step, bags)
     dominant = "backward" if bwd_ms >= fwd_ms else "forward"
     dom_bytes, dom_ms = (bwd_bytes, bwd_ms) if dominant == "backward" else (fwd_bytes, fwd_ms)
-    traffic = NCU_TRAFFIC_BYTES.get(w.name, {})
+    traffic = NCU_TRAFFIC_BYTES.get((w.name, args.backward), {})
 
     def roof(nbytes, ms, which):
         ach = nbytes / (ms * 1e-3) / 1e9
@@ -339,19 +372,27 @@ def run_ours(args, w):
                 "ms_per_launch": ms, "algorithmic_bytes": int(nbytes)}
 
     value = job_ids / (total_ms * 1e-3)
+    array_mb = w.M * (4 if w.array_dtype == "f32" else 2) / 1e6
+    stream_mb = (2 * 4 * nbags * d + 8 * nnz_per_step) / 1e6
+    if array_mb > 2 * 126:
+        l2_note = f"{array_mb:.0f} MB array and 4 rotated id batches exceed L2; no flush"
+    else:
+        l2_note = (f"{array_mb:.0f} MB array stays L2-warm on purpose (steady state of a model that fits L2); "
+                   f"the {stream_mb:.0f} MB of ids, output and gradient streamed per step exceed L2; no flush")
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": w.name, "num_tables": T, "d": d, "Z": w.Z, "M": w.M, "batch_per_gpu": B,
-                   "ids_per_step_per_gpu": nnz_per_step, "bags": bags, "backward": "atomic, SGD fused",
-                   "l2": "1 GB array and 4 rotated id batches exceed L2; no flush",
+                   "ids_per_step_per_gpu": nnz_per_step, "bags": bags, "backward": ("atomic" if args.backward == "atomic" else "deterministic") +
+                   (", SGD fused" if dense is None else ", dense fp32 gradient"),
+                   "l2": l2_note,
                    "parallelism": f"dp{world} replicas, no collective"},
         "clocks": clocks,
         "e2e": {"value": job_e2e_ids / (e2e_ms * 1e-3), "unit": UNIT,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
                 "ms_per_step": e2e_ms / e2e_steps},
-        "gpu_launches": 2 * args.steps,
+        "gpu_launches": (1 + bwd_launches) * args.steps,
         "roofline": roof(dom_bytes, dom_ms, dominant),
         "roofline_forward": roof(fwd_bytes, fwd_ms, "forward"),
         "roofline_backward": roof(bwd_bytes, bwd_ms, "backward"),
@@ -376,7 +417,9 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg4", choices=["cfg2", "cfg3_z1", "cfg3_z128", "cfg4", "cfg5"])
+    ap.add_argument("--workload", default="cfg4", help=WORKLOAD_HELP)
+    ap.add_argument("--backward", default="atomic", choices=["atomic", "det"],
+                    help="backward variant of the step (default: atomic red.global adds)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=0,
                     help="samples per GPU instead of the workload's own batch (small profiler captures)")
