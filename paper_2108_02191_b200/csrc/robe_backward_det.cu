@@ -285,15 +285,15 @@ __device__ __forceinline__ void commit_slot(float* target, uint32_t j, float acc
 // server then only walks forward through the sorted list, adding terms while the key stays <= j.
 //
 // One warp takes 32 consecutive sorted positions (a tile).  Keys and payloads live in a
-// warp-private ring of 128 positions in shared memory, filled by coalesced loads.  The lanes
-// cover (position, offset) pairs: G = min(Zp, 32) lanes per position (Zp = Z rounded up to a
-// power of two), 32/G positions at a time, Zp/G offset chunks per position.  For the pairs that
-// serve a slot, all lanes step through the ring together, UN positions per step: ring reads,
-// then the gradient loads, then the adds in sorted order; the next 32 positions are fetched one
-// step ahead of their first use.  A walk that is still going after 64 positions (an id that
-// occurs many times in the batch) goes on 32 positions per step, with the gradient rows of the
-// positions after those asked into L2 ahead of time, so that its chain of dependent adds waits
-// for memory once per 32 terms.
+// warp-private ring of 128 positions in shared memory, filled by coalesced loads.  The
+// (position, offset) pairs of the tile that serve a slot are numbered through and dealt out one
+// per lane, 32 per round.  In a round all lanes step through the ring together, each from its own
+// position, UN positions per step (4 in the first step, then 8): ring reads, then the gradient
+// loads, then the adds in sorted order; the next 32 positions are fetched one step ahead of
+// their first use.  A walk that is still going after 64 positions (an id that occurs many
+// times in the batch) goes on 16 positions per step, with the gradient rows of the positions
+// after those asked into L2 ahead of time, so that its chain of dependent adds waits for memory
+// once per 16 terms.
 #ifndef ROBE_DEEP_UN
 #define ROBE_DEEP_UN 16
 #endif
@@ -431,7 +431,7 @@ __device__ __forceinline__ void walk_deep(const ApplyArgs& a, ApplyTile& tl, App
 template <bool SIGN, bool SGD, bool SHORT>
 __global__ void __launch_bounds__(256)
 det_apply_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint32_t* __restrict__ V,
-                 const uint32_t* __restrict__ bag_of, uint32_t log2Zp) {
+                 const uint32_t* __restrict__ bag_of) {
     constexpr int UN = 8;
     constexpr uint32_t kDeepAfter = 64;  // positions after which a walk counts as long
     __shared__ uint2 ring_s[8][kRing];
@@ -463,47 +463,65 @@ det_apply_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint32_t* __
     }
     __syncwarp();
 
-    const uint32_t log2G = log2Zp < 5 ? log2Zp : 5;
-    const uint32_t G = 1u << log2G, EPW = 32u >> log2G, CH = 1u << (log2Zp - log2G);
-    const uint32_t sub = lane >> log2G, ul = lane & (G - 1);
+    // Served (position, offset) pairs are numbered tile-wide - position after position, offsets
+    // ascending - and dealt out 32 per round, one pair per lane, so that no lane idles on a pair
+    // that serves nothing.
+    const uint32_t cnt = mp.Z - own_lo;
+    uint32_t incl = cnt;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t n = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if (lane >= (uint32_t)o) incl += n;
+    }
+    const uint32_t total = __shfl_sync(0xFFFFFFFFu, incl, 31);
 
-    for (uint32_t eb = 0; eb < 32; eb += EPW) {
-        const uint32_t e = eb + sub;
+    for (uint32_t r0 = 0; r0 < total; r0 += 32) {
+        const uint32_t idx = r0 + lane;
+        // position e of pair idx: the first lane whose inclusive count exceeds idx
+        uint32_t e = 0;
+#pragma unroll
+        for (int step = 16; step >= 1; step >>= 1) {
+            const uint32_t v = __shfl_sync(0xFFFFFFFFu, incl, e + step - 1);
+            if (v <= idx) e += step;
+        }
+        if (e > 31) e = 31;  // idx >= total: no pair
+        const uint32_t incl_e = __shfl_sync(0xFFFFFFFFu, incl, e);
         const uint32_t lo_e = __shfl_sync(0xFFFFFFFFu, own_lo, e);
         const uint32_t s = __shfl_sync(0xFFFFFFFFu, mine.x, e);
-        for (uint32_t ch = 0; ch < CH; ++ch) {
-            const uint32_t u = ch * G + ul;
-            const uint64_t j64 = (uint64_t)s + u;
-            // j64 >= m: wrapped part, j64 < Z-1: low slots - both belong to the other kernel
-            const bool active = u >= lo_e && u < mp.Z && j64 < mp.m && j64 + 1 >= mp.Z;
-            if (__ballot_sync(0xFFFFFFFFu, active) == 0) continue;
-            const uint32_t j = (uint32_t)j64;
-            float old = 0.0f;
-            if (active) old = a.target[j];
+        const uint32_t u = mp.Z - (incl_e - idx);  // lo_e <= u < Z for a real pair
+        const uint64_t j64 = (uint64_t)s + u;
+        // j64 >= m: wrapped part, j64 < Z-1: low slots - both belong to the other kernel
+        const bool active = idx < total && u >= lo_e && u < mp.Z && j64 < mp.m && j64 + 1 >= mp.Z;
+        if (__ballot_sync(0xFFFFFFFFu, active) == 0) continue;
+        const uint32_t j = (uint32_t)j64;
+        float old = 0.0f;
+        if (active) old = a.target[j];
 
-            if (tl.loaded_end > eb + kRing) {  // an earlier long walk moved the ring past this tile
-                __syncwarp();
-                tl.ring[lane] = mine;
-                tl.ring[32 + lane] = tl.fetch(32 + lane);
-                tl.loaded_end = 64;
-                __syncwarp();
-            }
-
-            ApplyWalk wk;
-            wk.acc = 0.0f;
-            wk.touched = false;
-            wk.done = !active;
-            wk.pending = false;
-            wk.ahead = make_uint2(kNoKey, 0u);
-            wk.fbase = eb;
-            if (!SIGN && !SHORT) {
-                if (!walk_steps<SIGN, SHORT, UN>(a, bag_of, tl, wk, j, sub, EPW, lane, eb + kDeepAfter))
-                    walk_deep(a, tl, wk, j, sub, EPW, lane, ch * G);
-            } else {
-                walk_steps<SIGN, SHORT, UN>(a, bag_of, tl, wk, j, sub, EPW, lane, 0);
-            }
-            if (wk.touched) a.target[j] = SGD ? __fmaf_rn(-a.lr, wk.acc, old) : __fadd_rn(old, wk.acc);
+        if (tl.loaded_end > kRing) {  // an earlier long walk moved the ring past the tile's start
+            __syncwarp();
+            tl.ring[lane] = mine;
+            tl.ring[32 + lane] = tl.fetch(32 + lane);
+            tl.loaded_end = 64;
+            __syncwarp();
         }
+
+        // the lane walks from its own position e: step n reads positions fbase + e + t
+        ApplyWalk wk;
+        wk.acc = 0.0f;
+        wk.touched = false;
+        wk.done = !active;
+        wk.pending = false;
+        wk.ahead = make_uint2(kNoKey, 0u);
+        wk.fbase = 0;
+        if (!walk_steps<SIGN, SHORT, 4>(a, bag_of, tl, wk, j, e, 32u, lane, 4)) {
+            if (!SIGN && !SHORT) {
+                if (!walk_steps<SIGN, SHORT, UN>(a, bag_of, tl, wk, j, e, 32u, lane, kDeepAfter))
+                    walk_deep(a, tl, wk, j, e, 32u, lane, u & ~31u);
+            } else {
+                walk_steps<SIGN, SHORT, UN>(a, bag_of, tl, wk, j, e, 32u, lane, 0);
+            }
+        }
+        if (wk.touched) a.target[j] = SGD ? __fmaf_rn(-a.lr, wk.acc, old) : __fadd_rn(old, wk.acc);
     }
 }
 
@@ -567,14 +585,12 @@ template <bool SIGN, bool SGD>
 void launch_apply(const ApplyArgs& aa, const uint32_t* K, const uint32_t* V, const uint32_t* bag_of,
                   cudaStream_t st) {
     const MapParams& mp = aa.mp;
-    uint32_t log2Zp = 0;
-    while ((1u << log2Zp) < mp.Z) ++log2Zp;
     const unsigned blocks = (unsigned)((aa.nb + 255) / 256);  // one warp per 32 sorted positions
     if (mp.d % mp.Z != 0) {
-        det_apply_kernel<SIGN, SGD, true><<<blocks, 256, 0, st>>>(aa, K, V, bag_of, log2Zp);
+        det_apply_kernel<SIGN, SGD, true><<<blocks, 256, 0, st>>>(aa, K, V, bag_of);
         if (mp.Z > 1) det_apply_low_kernel<SIGN, SGD, true><<<1, 128, 0, st>>>(aa, K, V, bag_of);
     } else {
-        det_apply_kernel<SIGN, SGD, false><<<blocks, 256, 0, st>>>(aa, K, V, bag_of, log2Zp);
+        det_apply_kernel<SIGN, SGD, false><<<blocks, 256, 0, st>>>(aa, K, V, bag_of);
         if (mp.Z > 1) det_apply_low_kernel<SIGN, SGD, false><<<1, 128, 0, st>>>(aa, K, V, bag_of);
     }
 }
