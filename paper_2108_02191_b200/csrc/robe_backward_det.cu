@@ -13,6 +13,8 @@
 //                      ever walks forward through the sorted list.  Slots [0, Z-1), which also
 //                      receive the wrapped tails of blocks near the end of the array, are handled
 //                      by a small second kernel (those terms come last: their keys are the largest).
+//                      Walks over hundreds of blocks (an id repeated many times in the batch)
+//                      are finished by a third kernel that keeps a whole step of terms in flight.
 // No atomics on floating-point data and no waits between CTAs: the result is bit-reproducible.
 #include "robe_internal.h"
 
@@ -237,6 +239,18 @@ sort_scatter_kernel(const uint32_t* __restrict__ kin, const uint32_t* __restrict
     }
 }
 
+// A round of the apply kernel whose walks got long, handed over to the long-walk kernel: where
+// the tile starts, how far the lanes have come, and per lane its slot, its sum so far and its
+// position in the tile.
+struct LongWalk {
+    uint64_t i0;
+    uint32_t fbase;         // lane l goes on at sorted position i0 + fbase + e(l)
+    uint32_t pad;
+    uint32_t j[32];
+    float acc[32];
+    uint32_t state[32];     // e | going << 8 | touched << 9
+};
+
 struct ApplyArgs {
     MapParams mp;
     const float* grad_out;
@@ -245,6 +259,9 @@ struct ApplyArgs {
     float lr;
     uint64_t nb;
     const int32_t* status;
+    uint32_t* long_count;    // number of handed-over rounds (may run past long_cap)
+    LongWalk* long_walks;
+    uint32_t long_cap;
 };
 
 // The term that the sorted block with payload v contributes to the slot at in-block offset o
@@ -292,8 +309,9 @@ __device__ __forceinline__ void commit_slot(float* target, uint32_t j, float acc
 // loads, then the adds in sorted order; the next 32 positions are fetched one step ahead of
 // their first use.  A walk that is still going after 64 positions (an id that occurs many
 // times in the batch) goes on 16 positions per step, with the gradient rows of the positions
-// after those asked into L2 ahead of time, so that its chain of dependent adds waits for memory
-// once per 16 terms.
+// after those asked into L2 ahead of time; one that is still going after 256 positions is
+// handed, with its sums so far, to the long-walk kernel below (or finished here if the list of
+// handed-over rounds is full).
 #ifndef ROBE_DEEP_UN
 #define ROBE_DEEP_UN 16
 #endif
@@ -386,9 +404,9 @@ __device__ __forceinline__ bool walk_steps(const ApplyArgs& a, const uint32_t* b
 
 // The same for a long walk of plain blocks (sign off, no short last block): more positions per
 // step, each term's place in grad_out computed while its key is compared.
-__device__ __forceinline__ void walk_deep(const ApplyArgs& a, ApplyTile& tl, ApplyWalk& wk, uint32_t j,
+__device__ __forceinline__ bool walk_deep(const ApplyArgs& a, ApplyTile& tl, ApplyWalk& wk, uint32_t j,
                                           uint32_t sub, uint32_t EPW, uint32_t lane,
-                                          uint32_t chunk_off) {
+                                          uint32_t chunk_off, uint32_t limit) {
     constexpr int UN = ROBE_DEEP_UN;
     const float* pf = a.grad_out + chunk_off;
     // the ring has to reach the end of the first step before the one-step-ahead fetches take over
@@ -398,6 +416,7 @@ __device__ __forceinline__ void walk_deep(const ApplyArgs& a, ApplyTile& tl, App
         walk_commit(tl, wk, lane, pf);
     }
     for (;; wk.fbase += UN) {
+        if (limit != 0 && wk.fbase >= limit) return false;
         walk_advance<UN>(tl, wk, EPW, lane, pf);
         uint32_t at[UN];
         uint32_t n_in = 0;
@@ -424,7 +443,10 @@ __device__ __forceinline__ void walk_deep(const ApplyArgs& a, ApplyTile& tl, App
         }
         if (n_in != 0) wk.touched = true;
         wk.done = wk.done || n_in < (uint32_t)UN;
-        if (n_max < (uint32_t)UN) return;  // no lane goes on
+        if (n_max < (uint32_t)UN) {  // no lane goes on
+            wk.fbase += UN;
+            return true;
+        }
     }
 }
 
@@ -433,7 +455,8 @@ __global__ void __launch_bounds__(256)
 det_apply_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint32_t* __restrict__ V,
                  const uint32_t* __restrict__ bag_of) {
     constexpr int UN = 8;
-    constexpr uint32_t kDeepAfter = 64;  // positions after which a walk counts as long
+    constexpr uint32_t kDeepAfter = 64;       // positions after which a walk takes 16 per step
+    constexpr uint32_t kHandOverAfter = 256;  // ... and after which it goes to the long-walk kernel
     __shared__ uint2 ring_s[8][kRing];
     if (a.status != nullptr && *a.status != 0) return;
     const MapParams& mp = a.mp;
@@ -515,13 +538,129 @@ det_apply_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint32_t* __
         wk.fbase = 0;
         if (!walk_steps<SIGN, SHORT, 4>(a, bag_of, tl, wk, j, e, 32u, lane, 4)) {
             if (!SIGN && !SHORT) {
-                if (!walk_steps<SIGN, SHORT, UN>(a, bag_of, tl, wk, j, e, 32u, lane, kDeepAfter))
-                    walk_deep(a, tl, wk, j, e, 32u, lane, u & ~31u);
+                if (!walk_steps<SIGN, SHORT, UN>(a, bag_of, tl, wk, j, e, 32u, lane, kDeepAfter) &&
+                    !walk_deep(a, tl, wk, j, e, 32u, lane, u & ~31u, kHandOverAfter)) {
+                    // long walks: hand the round over if the list has room, else go on here
+                    uint32_t rec = a.long_cap;
+                    if (a.long_cap != 0) {
+                        if (lane == 0) rec = atomicAdd(a.long_count, 1u);
+                        rec = __shfl_sync(0xFFFFFFFFu, rec, 0);
+                    }
+                    if (rec < a.long_cap) {
+                        LongWalk* lw = a.long_walks + rec;
+                        if (lane == 0) {
+                            lw->i0 = tl.i0;
+                            lw->fbase = wk.fbase;
+                        }
+                        lw->j[lane] = j;
+                        lw->acc[lane] = wk.acc;
+                        lw->state[lane] = e | (wk.done ? 0u : 1u << 8) | (wk.touched ? 1u << 9 : 0u);
+                        if (!wk.done) wk.touched = false;  // finished (and stored) by the other kernel
+                    } else {
+                        walk_deep(a, tl, wk, j, e, 32u, lane, u & ~31u, 0);
+                    }
+                }
             } else {
                 walk_steps<SIGN, SHORT, UN>(a, bag_of, tl, wk, j, e, 32u, lane, 0);
             }
         }
         if (wk.touched) a.target[j] = SGD ? __fmaf_rn(-a.lr, wk.acc, old) : __fadd_rn(old, wk.acc);
+    }
+}
+
+// Long walks (plain blocks only).  One warp per handed-over round, in steps of kLongStep
+// positions.  The keys come from a warp-private ring of 256 positions; every lane copies the
+// gradient terms of its slot with cp.async into its own column of a shared-memory buffer, so a
+// whole step is in flight at once without a register per term.  Two buffers: the copies of step
+// n+1 are issued before the terms of step n are added (in sorted order), and the keys two
+// steps ahead are fetched meanwhile.
+constexpr int kLongStep = 64;
+constexpr uint32_t kLongRing = 256;
+
+template <bool SGD>
+__global__ void __launch_bounds__(64)
+det_apply_long_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint32_t* __restrict__ V) {
+    __shared__ float terms_s[2][2][kLongStep][32];
+    __shared__ uint2 ring_s[2][kLongRing];
+    if (a.status != nullptr && *a.status != 0) return;
+    const uint32_t lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const uint32_t n_rec = *a.long_count < a.long_cap ? *a.long_count : a.long_cap;
+    uint2* ring = ring_s[w];
+    const uint32_t dst0 = (uint32_t)__cvta_generic_to_shared(&terms_s[w][0][0][lane]);
+    constexpr uint32_t kBufBytes = kLongStep * 32 * sizeof(float);
+    for (uint32_t rec = blockIdx.x * 2 + w; rec < n_rec; rec += gridDim.x * 2) {
+        const LongWalk* lw = a.long_walks + rec;
+        const uint64_t i0 = lw->i0;
+        const uint32_t j = lw->j[lane];
+        float acc = lw->acc[lane];
+        const uint32_t st = lw->state[lane];
+        const uint32_t e = st & 0xFFu;
+        const bool mine = (st >> 8) & 1u;  // this lane's walk was handed over
+        bool going = mine, touched = (st >> 9) & 1u;
+        auto fetch = [&](uint32_t r) -> uint2 {
+            const uint64_t idx = i0 + r;
+            if (idx >= a.nb) return make_uint2(kNoKey, 0u);
+            return make_uint2(__ldg(K + idx), __ldg(V + idx));
+        };
+        // Issues the copies of the step that starts at tile-relative position `base` into buffer
+        // `buf`; returns how many positions of the step reach slot j (sorted keys: a prefix).
+        auto issue = [&](uint32_t base, uint32_t buf) -> uint32_t {
+            uint32_t n = 0;
+            const uint32_t dst = dst0 + buf * kBufBytes;
+#pragma unroll 8
+            for (int t = 0; t < kLongStep; ++t) {
+                const uint2 kv = ring[(base + e + t) & (kLongRing - 1)];
+                if (going && kv.x <= j) {
+                    const float* src = a.grad_out + (kv.y + (j - kv.x));
+                    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst + (uint32_t)t * 128u),
+                                 "l"(src));
+                    ++n;
+                }
+            }
+            asm volatile("cp.async.commit_group;");
+            going = going && n == (uint32_t)kLongStep;
+            return n;
+        };
+        // a step reads positions base + e + t, e < 32, t < kLongStep: [base, base + 96)
+        uint32_t base = lw->fbase;
+        uint32_t ring_end = base + 160;
+        __syncwarp();
+#pragma unroll
+        for (int q = 0; q < 5; ++q) ring[(base + 32 * q + lane) & (kLongRing - 1)] = fetch(base + 32 * q + lane);
+        __syncwarp();
+        uint32_t n_cur = issue(base, 0);
+        for (uint32_t step = 0;; ++step) {
+            // step+1: its keys [base + 64, base + 160) are in the ring (ring_end = base + 160)
+            const uint32_t n_nxt = issue(base + kLongStep, (step + 1) & 1u);
+            const uint2 f0 = fetch(ring_end + lane), f1 = fetch(ring_end + 32 + lane);
+            asm volatile("cp.async.wait_group 1;" ::: "memory");  // the copies of `step` are in
+            const float(*buf)[32] = terms_s[w][step & 1u];
+            const uint32_t n_max = __reduce_max_sync(0xFFFFFFFFu, n_cur);
+            for (uint32_t t0 = 0; t0 < n_max; t0 += 8) {
+                float x[8];
+#pragma unroll
+                for (int q = 0; q < 8; ++q) x[q] = buf[t0 + q][lane];
+#pragma unroll
+                for (int q = 0; q < 8; ++q)
+                    if (t0 + q < n_cur) acc = __fadd_rn(acc, x[q]);
+            }
+            if (n_cur != 0) touched = true;
+            const bool any_next = __ballot_sync(0xFFFFFFFFu, n_nxt != 0) != 0;
+            if (!any_next) break;
+            __syncwarp();  // every lane is past its ring reads of step+1: the keys of step+2 may enter
+            ring[(ring_end + lane) & (kLongRing - 1)] = f0;
+            ring[(ring_end + 32 + lane) & (kLongRing - 1)] = f1;
+            ring_end += 64;
+            __syncwarp();
+            n_cur = n_nxt;
+            base += kLongStep;
+        }
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        if (mine && touched) {
+            const float old = a.target[j];
+            a.target[j] = SGD ? __fmaf_rn(-a.lr, acc, old) : __fadd_rn(old, acc);
+        }
+        __syncwarp();  // the buffers and the ring are reused by the warp's next round
     }
 }
 
@@ -563,7 +702,8 @@ uint32_t bits_for(uint32_t m) {  // bits needed for keys in [0, m)
 }
 
 struct Layout {
-    size_t keysA, keysB, valsA, valsB, bag_of, counts, totals, total;
+    size_t keysA, keysB, valsA, valsB, bag_of, counts, totals, long_count, long_walks, total;
+    uint32_t long_cap;
 };
 
 Layout make_layout(uint64_t nb, int64_t nnz, bool bags) {
@@ -577,6 +717,12 @@ Layout make_layout(uint64_t nb, int64_t nnz, bool bags) {
     L.bag_of = off; off += bags ? align256((size_t)(nnz ? nnz : 1) * sizeof(uint32_t)) : 0;
     L.counts = off; off += align256((size_t)kRadix * kSortMaxGrid * sizeof(uint32_t));
     L.totals = off; off += align256((size_t)kRadix * sizeof(uint32_t));
+    // list of long walks: room for one round per 128 blocks, within 64 .. 2^20 rounds
+    uint64_t cap = nb / 128;
+    cap = cap < 64 ? 64 : (cap > (1u << 20) ? (1u << 20) : cap);
+    L.long_cap = (uint32_t)cap;
+    L.long_count = off; off += 256;
+    L.long_walks = off; off += align256((size_t)cap * sizeof(LongWalk));
     L.total = off;
     return L;
 }
@@ -591,6 +737,11 @@ void launch_apply(const ApplyArgs& aa, const uint32_t* K, const uint32_t* V, con
         if (mp.Z > 1) det_apply_low_kernel<SIGN, SGD, true><<<1, 128, 0, st>>>(aa, K, V, bag_of);
     } else {
         det_apply_kernel<SIGN, SGD, false><<<blocks, 256, 0, st>>>(aa, K, V, bag_of);
+        if (!SIGN) {
+            // the rounds the apply kernel handed over; a grid-stride loop over the list
+            const unsigned lblocks = aa.long_cap / 2 < 148u * 8u ? (aa.long_cap + 1) / 2 : 148u * 8u;
+            det_apply_long_kernel<SGD><<<lblocks, 64, 0, st>>>(aa, K, V);
+        }
         if (mp.Z > 1) det_apply_low_kernel<SIGN, SGD, false><<<1, 128, 0, st>>>(aa, K, V, bag_of);
     }
 }
@@ -650,7 +801,10 @@ cudaError_t launch_backward_det(const Problem& pb, const float* grad_out, float*
         t = vA; vA = vB; vB = t;
     }
 
-    ApplyArgs aa{mp, grad_out, pb.indices, target, lr, nb, pb.status};
+    uint32_t* long_count = (uint32_t*)(ws + L.long_count);
+    cudaMemsetAsync(long_count, 0, sizeof(uint32_t), st);
+    ApplyArgs aa{mp, grad_out, pb.indices, target, lr, nb, pb.status,
+                 long_count, (LongWalk*)(ws + L.long_walks), L.long_cap};
     if (pb.sign) {
         if (sgd) launch_apply<true, true>(aa, kA, vA, bag_of, st);
         else launch_apply<true, false>(aa, kA, vA, bag_of, st);

@@ -79,17 +79,19 @@ def test_fused_sgd_matches_the_workspace_variant():
 
 
 def test_largest_and_too_large_calls():
-    # one-hot, Z = d: one block per id.  The workspace is 16 bytes per block + 4 per id + counters.
+    # one-hot, Z = d: one block per id
     w = _workload(d=32, Z=32, M=100003, bag_rule=None, num_tables=4, vocab_arg=(100, 10**6, 5, 77))
     with Case(w, batch=8) as c:
         robe.robe_set_option(c.h, robe.ROBE_OPT_BWD_MODE, robe.ROBE_BWD_DETERMINISTIC)
         limit = robe.ROBE_STATIC_SCRATCH_BYTES
-        per_sample = (robe.robe_backward_workspace_bytes(c.h, 4096, 4096 * c.T)
-                      - robe.robe_backward_workspace_bytes(c.h, 2048, 2048 * c.T)) / 2048
-        fits = int((limit - robe.robe_backward_workspace_bytes(c.h, 0, 0)) // per_sample) - 8
-        assert robe.robe_backward_workspace_bytes(c.h, fits, fits * c.T) <= limit
-        too_big = fits + 64
-        assert robe.robe_backward_workspace_bytes(c.h, too_big, too_big * c.T) > limit
+        need = lambda b: robe.robe_backward_workspace_bytes(c.h, b, b * c.T)
+        lo, hi = 1, 1 << 22  # the largest batch whose workspace fits, by bisection
+        assert need(lo) <= limit < need(hi)
+        while hi - lo > 1:
+            mid = (lo + hi) // 2
+            lo, hi = (mid, hi) if need(mid) <= limit else (lo, mid)
+        fits, too_big = lo, lo + 64
+        assert need(fits) <= limit < need(too_big)
     with Case(w, batch=too_big) as c:
         g = torch.zeros(c.B, c.T, w.d, device=c.dev)
         ga = torch.zeros(w.M, device=c.dev)
