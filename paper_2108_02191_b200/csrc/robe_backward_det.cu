@@ -153,7 +153,7 @@ sort_scan_kernel(uint32_t* counts, uint32_t* totals, uint32_t grid) {
 }
 
 // ---- kernel 3: stable ranked scatter.  Per tile of 4096 pairs: every warp ranks its 512 pairs
-// by digit (16 rounds of __match_any_sync, earlier rounds and lower lanes first), the ranks are
+// by digit (16 rounds of ballots, earlier rounds and lower lanes first), the ranks are
 // extended over the warps, the pairs are laid out in shared memory in (digit, original order),
 // and then written out so that each digit's pairs go to consecutive addresses.
 __global__ void __launch_bounds__(kSortThreads, 3)
@@ -191,8 +191,16 @@ sort_scatter_kernel(const uint32_t* __restrict__ kin, const uint32_t* __restrict
 #pragma unroll
         for (int r = 0; r < kSortItems; ++r) {
             const bool valid = wbegin + r * 32 + lane < nb;
-            const uint32_t dg = valid ? ((key[r] >> shift) & mask) : (uint32_t)kRadix;
-            const uint32_t peers = __match_any_sync(0xFFFFFFFFu, dg);
+            const uint32_t dg = valid ? ((key[r] >> shift) & mask) : 0u;
+            // lanes holding the same digit: one ballot per digit bit (a fixed cost, where
+            // __match_any_sync takes time in proportion to the number of distinct digits)
+            uint32_t peers = __ballot_sync(0xFFFFFFFFu, valid);
+#pragma unroll
+            for (int b = 0; b < 8; ++b) {
+                const bool bit = (dg >> b) & 1u;
+                const uint32_t bal = __ballot_sync(0xFFFFFFFFu, bit);
+                peers &= bit ? bal : ~bal;
+            }
             uint32_t before = 0;
             if (valid) before = wcnt[w][dg];
             __syncwarp();
