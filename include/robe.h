@@ -176,9 +176,9 @@ int robe_backward(robe_handle_t h, const float* grad_out, const int64_t* indices
  * allocating routine.
  *
  * Limit: the call must fit the fixed array, i.e. the value robe_backward_workspace_bytes
- * reports for it in deterministic mode (about 16 bytes per block, nnz * ceil(d/Z) blocks,
- * plus 4 bytes per id and 0.6 MB of counters) must not exceed ROBE_STATIC_SCRATCH_BYTES;
- * a larger call returns ROBE_ERR_WORKSPACE and launches nothing.
+ * reports for it in deterministic mode (about 19 bytes per block, nnz * ceil(d/Z) blocks,
+ * plus 4 bytes per id and 0.7 MB of counters and lists) must not exceed
+ * ROBE_STATIC_SCRATCH_BYTES; a larger call returns ROBE_ERR_WORKSPACE and launches nothing.
  *
  * First call on a device: the function looks up the device address of the array once per
  * device (with that device current) and remembers it.  Make that first call during

@@ -26,6 +26,11 @@
  *     appendix both say it is not used in practice).
  *   - pooling over a bag is a sequential fp32 sum in bag order (the paper's data
  *     are one-hot, so this part is a definition of this library, not the paper's).
+ *   - Z > d (Section 3.2, last paragraph: "clubbing multiple embeddings together
+ *     in a chunk"; the appendix cuts the row-wise flattened table into chunks of
+ *     Z) is taken for d dividing Z: R = Z/d consecutive rows of a table share one
+ *     block, row x is the piece [(x mod R) d, (x mod R) d + d) of the block that
+ *     starts at h(e, floor(x/R), 0).
  *
  * Parity pins: the hash arithmetic, the idx mapping, the circular wrap, the
  * Z = d and Z = 1 special cases, the sign range, the adjoint identity that ties
@@ -97,11 +102,37 @@ uint64_t robe_oracle_h(const uint64_t k[9], uint64_t m, uint64_t e, uint64_t x, 
     return r % m;
 }
 
-uint64_t robe_oracle_idx(const uint64_t k[9], uint64_t m, uint64_t Z, uint64_t e, uint64_t x,
-                         uint64_t i) {
+uint64_t robe_oracle_idx(const uint64_t k[9], uint64_t m, uint64_t Z, uint64_t d, uint64_t e,
+                         uint64_t x, uint64_t i) {
+    if (Z > d) { /* rows clubbed into one chunk of Z: position x d + i of the flattened table */
+        uint64_t R = Z / d;
+        return (robe_oracle_h(k, m, e, x / R, 0) + (x % R) * d + i) % m;
+    }
     uint64_t c = i / Z; /* chunk id    */
     uint64_t o = i % Z; /* offset in it */
     return (robe_oracle_h(k, m, e, x, c) + o) % m;
+}
+
+/* The blocks of one embedding, for any Z.  Z <= d: ceil(d/Z) blocks, block c holds elements
+   [cZ, min(cZ+Z, d)) and starts at h(e,x,c).  Z > d (d divides Z): ONE block holding all d
+   elements; it is the piece of the shared Z-block of rows floor(x/R)R .. +R-1 (R = Z/d) that
+   belongs to row x, so it starts (x mod R) d slots after h(e, floor(x/R), 0). */
+static uint64_t blocks_per_id(uint64_t Z, uint64_t d) { return Z > d ? 1 : (d + Z - 1) / Z; }
+
+static uint64_t block_len(uint64_t Z, uint64_t d, uint64_t c) {
+    if (Z > d) return d;
+    return c * Z + Z <= d ? Z : d - c * Z;
+}
+
+static uint64_t block_first_elem(uint64_t Z, uint64_t d, uint64_t c) { return Z > d ? 0 : c * Z; }
+
+uint64_t robe_oracle_block_start(const uint64_t k[9], uint64_t m, uint64_t Z, uint64_t d,
+                                 uint64_t e, uint64_t x, uint64_t c) {
+    if (Z > d) {
+        uint64_t R = Z / d;
+        return (robe_oracle_h(k, m, e, x / R, 0) + (x % R) * d) % m;
+    }
+    return robe_oracle_h(k, m, e, x, c);
 }
 
 /* sign hash (Section 3.1, g equation): +1 or -1 */
@@ -144,11 +175,11 @@ static void forward_one_bag(const uint64_t k[9], uint64_t m, uint64_t Z, uint64_
     for (uint64_t i = 0; i < d; ++i) row[i] = 0.0f;
     for (int64_t p = lo; p < hi; ++p) {
         uint64_t x = (uint64_t)indices[p];
-        uint64_t nchunks = (d + Z - 1) / Z;
+        uint64_t nchunks = blocks_per_id(Z, d);
         for (uint64_t c = 0; c < nchunks; ++c) {
-            uint64_t h = robe_oracle_h(k, m, e, x, c);
-            for (uint64_t o = 0; o < Z && c * Z + o < d; ++o) {
-                uint64_t i = c * Z + o;
+            uint64_t h = robe_oracle_block_start(k, m, Z, d, e, x, c);
+            for (uint64_t o = 0; o < block_len(Z, d, c); ++o) {
+                uint64_t i = block_first_elem(Z, d, c) + o;
                 float v = array_at(array, dtype, (h + o) % m);
                 if (sign) v = (float)robe_oracle_g(k, e, x, i) * v;
                 row[i] = (p == lo) ? v : row[i] + v;
@@ -180,7 +211,11 @@ void robe_oracle_forward_bags(const uint64_t k[9], uint64_t m, uint64_t Z, uint6
 /* The slots idx(e,x,i) of one embedding, for tests that need the mapping itself. */
 void robe_oracle_locate(const uint64_t k[9], uint64_t m, uint64_t Z, uint64_t d, uint64_t e,
                         uint64_t x, uint64_t *slots) {
-    for (uint64_t i = 0; i < d; ++i) slots[i] = robe_oracle_idx(k, m, Z, e, x, i);
+    for (uint64_t c = 0; c < blocks_per_id(Z, d); ++c) {
+        uint64_t h = robe_oracle_block_start(k, m, Z, d, e, x, c);
+        for (uint64_t o = 0; o < block_len(Z, d, c); ++o)
+            slots[block_first_elem(Z, d, c) + o] = (h + o) % m;
+    }
 }
 
 /* ---- backward (Section 3.1 backward equation): delta[j] = sum over idx(e,x,i)=j of g * dE ---- */
@@ -192,7 +227,7 @@ void robe_oracle_backward_f64(const uint64_t k[9], uint64_t m, uint64_t Z, uint6
                               const int64_t *offsets, int64_t batch, uint64_t j0, uint64_t jn,
                               double *delta64, double *l1) {
     int64_t nbags = batch * (int64_t)T;
-    uint64_t nchunks = (d + Z - 1) / Z;
+    uint64_t nchunks = blocks_per_id(Z, d);
     for (int64_t bag = 0; bag < nbags; ++bag) {
         int64_t lo, hi;
         bag_bounds(offsets, bag, &lo, &hi);
@@ -201,9 +236,9 @@ void robe_oracle_backward_f64(const uint64_t k[9], uint64_t m, uint64_t Z, uint6
         for (int64_t p = lo; p < hi; ++p) {
             uint64_t x = (uint64_t)indices[p];
             for (uint64_t c = 0; c < nchunks; ++c) {
-                uint64_t h = robe_oracle_h(k, m, e, x, c);
-                for (uint64_t o = 0; o < Z && c * Z + o < d; ++o) {
-                    uint64_t i = c * Z + o;
+                uint64_t h = robe_oracle_block_start(k, m, Z, d, e, x, c);
+                for (uint64_t o = 0; o < block_len(Z, d, c); ++o) {
+                    uint64_t i = block_first_elem(Z, d, c) + o;
                     uint64_t j = (h + o) % m;
                     if (j < j0 || j - j0 >= jn) continue;
                     double gsign = sign ? (double)robe_oracle_g(k, e, x, i) : 1.0;
@@ -238,7 +273,7 @@ int robe_oracle_backward_canonical(const uint64_t k[9], uint64_t m, uint64_t Z, 
                                    const int64_t *indices, const int64_t *offsets, int64_t batch,
                                    uint64_t j0, uint64_t jn, float *delta, uint8_t *touched) {
     int64_t nbags = batch * (int64_t)T;
-    uint64_t nchunks = (d + Z - 1) / Z;
+    uint64_t nchunks = blocks_per_id(Z, d);
     int64_t nnz = offsets ? offsets[nbags] : nbags;
     uint64_t nblocks = (uint64_t)nnz * nchunks;
     block_key *keys = (block_key *)malloc((nblocks ? nblocks : 1) * sizeof(block_key));
@@ -255,7 +290,8 @@ int robe_oracle_backward_canonical(const uint64_t k[9], uint64_t m, uint64_t Z, 
         for (int64_t p = lo; p < hi; ++p) {
             bag_of[p] = bag;
             for (uint64_t c = 0; c < nchunks; ++c) {
-                keys[(uint64_t)p * nchunks + c].s = robe_oracle_h(k, m, e, (uint64_t)indices[p], c);
+                keys[(uint64_t)p * nchunks + c].s =
+                    robe_oracle_block_start(k, m, Z, d, e, (uint64_t)indices[p], c);
                 keys[(uint64_t)p * nchunks + c].q = (uint64_t)p * nchunks + c;
             }
         }
@@ -271,8 +307,8 @@ int robe_oracle_backward_canonical(const uint64_t k[9], uint64_t m, uint64_t Z, 
         uint64_t e = (uint64_t)bag % T;
         uint64_t x = (uint64_t)indices[p];
         const float *grow = grad_out + bag * (int64_t)d;
-        for (uint64_t o = 0; o < Z && c * Z + o < d; ++o) {
-            uint64_t i = c * Z + o;
+        for (uint64_t o = 0; o < block_len(Z, d, c); ++o) {
+            uint64_t i = block_first_elem(Z, d, c) + o;
             uint64_t j = (keys[b].s + o) % m;
             if (j < j0 || j - j0 >= jn) continue;
             float term = grow[i];

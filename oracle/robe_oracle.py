@@ -42,7 +42,7 @@ def lib() -> C.CDLL:
         _lib.robe_oracle_num_threads.restype = C.c_int
         _lib.robe_oracle_h.argtypes = [p, u64, u64, u64, u64]
         _lib.robe_oracle_h.restype = u64
-        _lib.robe_oracle_idx.argtypes = [p, u64, u64, u64, u64, u64]
+        _lib.robe_oracle_idx.argtypes = [p, u64, u64, u64, u64, u64, u64]
         _lib.robe_oracle_idx.restype = u64
         _lib.robe_oracle_g.argtypes = [p, u64, u64, u64]
         _lib.robe_oracle_g.restype = C.c_int
@@ -95,7 +95,7 @@ class Oracle:
         return int(lib().robe_oracle_h(_ptr(self.k), self.M, e, x, c))
 
     def idx(self, e, x, i) -> int:
-        return int(lib().robe_oracle_idx(_ptr(self.k), self.M, self.Z, e, x, i))
+        return int(lib().robe_oracle_idx(_ptr(self.k), self.M, self.Z, self.d, e, x, i))
 
     def g(self, e, x, i) -> int:
         return int(lib().robe_oracle_g(_ptr(self.k), e, x, i))

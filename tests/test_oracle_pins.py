@@ -195,6 +195,66 @@ def test_forward_equals_brute_force_table(m, Z, d):
             np.testing.assert_array_equal(o.locate(e, x), np.array(loc[e][x], dtype=np.uint64))
 
 
+def brute_force_locations_clubbed(kk, m, Z, d, vocab):
+    """Z > d by the appendix's procedure taken literally: flatten the table row-wise into one
+    vector of V*d parameters, cut THAT into chunks of Z (the last may be short), hash chunk number
+    X of table e with (e, X, 0), lay it down circularly.  loc[e][x][i] = slot of flat position
+    x*d + i.  Python integers only; no division of x by Z/d anywhere."""
+    loc = []
+    for e, V in enumerate(vocab):
+        flat = [None] * (V * d)
+        for X in range((V * d + Z - 1) // Z):
+            start = ((kk[1] * e + kk[2] * X + kk[3] * 0 + kk[4]) % kk[0]) % m
+            for within in range(min(Z, V * d - X * Z)):
+                flat[X * Z + within] = (start + within) % m
+        loc.append([flat[x * d:(x + 1) * d] for x in range(V)])
+    return loc
+
+
+@pytest.mark.parametrize("m,Z,d", [(4096, 64, 16), (101, 32, 16), (50, 48, 16), (97, 24, 8), (40, 36, 12)])
+def test_z_above_d_equals_flattened_table_chunks(m, Z, d):
+    # Section 3.2, last paragraph, with the appendix's parameter-vector construction
+    vocab = [1000, 37, 5] if m == 4096 else [40, 7, 19]
+    T = len(vocab)
+    k = orc.hash_constants(0x0B0E + 9)
+    loc = brute_force_locations_clubbed([int(v) for v in k], m, Z, d, vocab)
+    o = orc.Oracle(m, Z, d, T, k)
+    arr = np.random.default_rng(2).standard_normal(m).astype(np.float32)
+    Vmax = max(vocab)
+    ids = np.stack([np.arange(Vmax) % V for V in vocab], axis=1)
+    out = o.forward(arr, ids.reshape(-1), None, Vmax)
+    for e, V in enumerate(vocab):
+        for x in range(V):
+            np.testing.assert_array_equal(out[x, e], arr[np.array(loc[e][x])])
+            np.testing.assert_array_equal(o.locate(e, x), np.array(loc[e][x], dtype=np.uint64))
+            assert [o.idx(e, x, i) for i in range(d)] == loc[e][x]
+    # rows of one chunk sit side by side (mod m): that is the point of Z > d
+    R = Z // d
+    a, b = o.locate(0, R * 3), o.locate(0, R * 3 + 1)
+    assert (int(a[-1]) + 1) % m == int(b[0])
+
+
+def test_z_above_d_backward_adjoint_mass_and_canonical():
+    m, Z, d, T, B = 211, 32, 8, 3, 50
+    k = orc.hash_constants(5)
+    o = orc.Oracle(m, Z, d, T, k)
+    rng = np.random.default_rng(3)
+    ids = rng.integers(0, 30, size=B * T)
+    arr = rng.standard_normal(m)
+    g = rng.standard_normal((B, T, d)).astype(np.float32)
+    out = o.forward(arr.astype(np.float32), ids, None, B).astype(np.float64)
+    delta, l1 = o.backward_f64(g, ids, None, B)
+    lhs = float((out * g).sum())
+    rhs = float((arr.astype(np.float32).astype(np.float64) * delta).sum())
+    assert abs(lhs - rhs) <= 1e-9 * (abs(lhs) + 1)
+    assert abs(delta.sum() - g.astype(np.float64).sum()) < 1e-9 * l1.sum()
+    gi = rng.integers(-3, 4, size=(B, T, d)).astype(np.float32)
+    di, _ = o.backward_f64(gi, ids, None, B)
+    can, touched = o.backward_canonical(gi, ids, None, B)
+    np.testing.assert_array_equal(can, di.astype(np.float32))
+    assert touched.sum() == (di != 0).sum() + ((di == 0) & (touched == 1)).sum()
+
+
 def test_blocks_are_consecutive_and_collision_free():
     # Section 4.1 intuition: elements inside one block never collide; slots are consecutive mod m
     k = orc.hash_constants(21)
