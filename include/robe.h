@@ -40,7 +40,7 @@ typedef struct robe_ctx* robe_handle_t; /* opaque; host memory owned by the libr
 
 typedef enum {
     ROBE_OK = 0,
-    ROBE_ERR_INVALID_ARG = -1, /* null pointer, zero size, Z > d, d > M, M + d > 2^32, ... */
+    ROBE_ERR_INVALID_ARG = -1, /* null pointer, zero size, d > M, Z > d not a multiple of d, M + d > 2^32, ... */
     ROBE_ERR_NO_ARRAY = -2,    /* forward/backward before robe_attach_array            */
     ROBE_ERR_WORKSPACE = -3,   /* deterministic backward: workspace missing/too small  */
     ROBE_ERR_CUDA = -4,        /* the CUDA runtime reported an error at launch         */
@@ -73,9 +73,13 @@ typedef enum {
  * robe_create - make a handle for one ROBE array shape (Section 3.2).
  *   out         host pointer receiving the handle.
  *   M           array length m = |M| in elements; 1 <= d <= M and M + d <= 2^32.
- *   Z           block size, 1 <= Z <= d.  Z = d is ROBE-D (one block per
- *               embedding, Section 3.1); Z = 1 hashes every element on its own
- *               (Section 3.3).  If Z does not divide d the last block is short.
+ *   Z           block size.  1 <= Z <= d: Z = d is ROBE-D (one block per embedding,
+ *               Section 3.1); Z = 1 hashes every element on its own (Section 3.3); if Z
+ *               does not divide d the last block is short.  Z > d (Section 3.2, last
+ *               paragraph: several embeddings clubbed into one chunk): Z must be a
+ *               multiple of d and <= M; rows floor(x/R) R .. + R-1 of a table, R = Z/d,
+ *               then share the block that starts at h(e, floor(x/R), 0), row x being the
+ *               piece [(x mod R) d, (x mod R) d + d) of it.
  *   d           embedding dimension (one d per handle; several handles may share
  *               one array, Section 3.1 "Multiple embedding tables").
  *   num_tables  T >= 1; the table id e of bag k is k mod T.

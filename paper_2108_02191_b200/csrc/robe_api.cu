@@ -111,7 +111,8 @@ int robe_create(robe_handle_t* out, uint64_t M, uint32_t Z, uint32_t d, uint32_t
     if (out == nullptr) return ROBE_ERR_INVALID_ARG;
     *out = nullptr;
     if (M == 0 || Z == 0 || d == 0 || num_tables == 0) return ROBE_ERR_INVALID_ARG;
-    if (Z > d || (uint64_t)d > M) return ROBE_ERR_INVALID_ARG;
+    if ((uint64_t)d > M) return ROBE_ERR_INVALID_ARG;
+    if (Z > d && (Z % d != 0 || (uint64_t)Z > M)) return ROBE_ERR_INVALID_ARG;
     if (d > 32768u) return ROBE_ERR_INVALID_ARG;
     if (M + (uint64_t)d > (1ull << 32)) return ROBE_ERR_INVALID_ARG;
     robe_ctx* h = new (std::nothrow) robe_ctx();
@@ -128,12 +129,15 @@ int robe_create(robe_handle_t* out, uint64_t M, uint32_t Z, uint32_t d, uint32_t
     mp.mu = (M == 1) ? ~0ull : (uint64_t)((((unsigned __int128)1) << 64) / M);
     mp.T = num_tables;
     mp.d = d;
-    mp.Z = Z;
-    mp.C = (d + Z - 1) / Z;
+    // Z > d: Z/d rows share one block; every kernel then sees one block of d elements per id
+    const uint32_t Zb = Z > d ? d : Z;
+    mp.Z = Zb;
+    mp.R = Z > d ? Z / d : 1;
+    mp.C = (d + Zb - 1) / Zb;
     mp.log2Z = 0xFFFFFFFFu;
-    if ((Z & (Z - 1)) == 0) {
+    if ((Zb & (Zb - 1)) == 0) {
         uint32_t l = 0;
-        while ((1u << l) < Z) ++l;
+        while ((1u << l) < Zb) ++l;
         mp.log2Z = l;
     }
     mp.tmagic = 0xFFFFFFFFFFFFFFFFull / num_tables + 1;

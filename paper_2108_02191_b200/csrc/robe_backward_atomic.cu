@@ -40,7 +40,7 @@ __global__ void __launch_bounds__(256) bwd_atomic_direct_kernel(BwdArgs a) {
         const float gv = __ldcs(a.grad_out + k * mp.d + i) * a.scale;
         for (int64_t p = lo; p < hi; ++p) {
             const uint64_t x = (uint64_t)__ldg(a.indices + p);
-            uint32_t j = block_start(mp, hash_base(mp.h, e, x), c) + o;
+            uint32_t j = id_block_start(mp, e, x, c) + o;
             if (j >= mp.m) j -= mp.m;
             float t = gv;
             if (SIGN) t = sign_of(mp, hash_base(mp.g, e, x), i) * t;

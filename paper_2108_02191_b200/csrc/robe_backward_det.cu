@@ -87,7 +87,7 @@ det_keys_kernel(KeyArgs a, const uint32_t* bag_of, uint32_t* keys, uint32_t* val
     const uint64_t bag = bag_of ? (uint64_t)bag_of[p] : (uint64_t)p;
     const uint32_t e = table_of_bag(bag, mp);
     const uint64_t x = (uint64_t)__ldg(a.indices + p);
-    keys[q] = block_start(mp, hash_base(mp.h, e, x), c);
+    keys[q] = id_block_start(mp, e, x, c);
     vals[q] = SIGN ? (uint32_t)q : (uint32_t)(bag * mp.d + c * mp.Z);
 }
 

@@ -28,8 +28,9 @@ struct MapParams {
     uint32_t m;        // array length (m + d <= 2^32)
     uint32_t T;        // number of tables
     uint32_t d;        // embedding dimension
-    uint32_t Z;        // block size
-    uint32_t C;        // chunks per embedding = ceil(d / Z)
+    uint32_t Z;        // block length the kernels work with: the block size, or d when rows are clubbed
+    uint32_t R;        // rows clubbed into one block: block size / d when that exceeds 1, else 1
+    uint32_t C;        // blocks per embedding = ceil(d / Z)
     uint32_t log2Z;    // valid when Z is a power of two, else 0xFFFFFFFF
     uint64_t tmagic;   // floor((2^64 - 1) / T) + 1, for k mod T with k < 2^32
 };
@@ -102,6 +103,19 @@ __device__ __forceinline__ uint64_t hash_base(const HashConsts& k, uint32_t e, u
 __device__ __forceinline__ uint32_t block_start(const MapParams& mp, uint64_t base, uint32_t c) {
     uint64_t t = addmod_p61(base, mulmod_p61_u32(mp.h.C, c));
     return mod_m(t, mp.m, mp.mu);
+}
+
+// Start of block c of id x of table e, for every block size.  When R rows share one block
+// (block size above d, Section 3.2 last paragraph) the block is hashed by (e, floor(x/R), 0) and
+// row x is the piece that starts (x mod R) d slots into it.
+__device__ __forceinline__ uint32_t id_block_start(const MapParams& mp, uint32_t e, uint64_t x,
+                                                   uint32_t c) {
+    if (mp.R > 1) {
+        const uint64_t X = x / mp.R;
+        const uint64_t j = (uint64_t)block_start(mp, hash_base(mp.h, e, X), 0) + (x - X * mp.R) * mp.d;
+        return (uint32_t)(j >= mp.m ? j - mp.m : j);  // both terms are below m
+    }
+    return block_start(mp, hash_base(mp.h, e, x), c);
 }
 
 // Sign g(e,x,i) as +1.0f / -1.0f given the sign-hash base of (e,x).

@@ -40,7 +40,7 @@ __global__ void __launch_bounds__(256) fwd_direct_kernel(FwdArgs a) {
         float acc = 0.0f;
         for (int64_t p = lo; p < hi; ++p) {
             const uint64_t x = (uint64_t)__ldg(a.indices + p);
-            uint32_t j = block_start(mp, hash_base(mp.h, e, x), c) + o;  // < m + d <= 2^32
+            uint32_t j = id_block_start(mp, e, x, c) + o;  // < m + d <= 2^32
             if (j >= mp.m) j -= mp.m;
             float v = load_elem<DT>(a.array, j);
             if (SIGN) v = sign_of(mp, hash_base(mp.g, e, x), i) * v;

@@ -31,6 +31,7 @@ struct StageSmem {
     uint64_t cterm[128];               // (C_h * c) mod P, c < C (d <= 128)
     uint64_t base[8][kStageIds];       // per warp: hash base of each staged id
     uint32_t start[8][kStageEntries];  // per warp: block starts, chunk-major
+    uint32_t piece[8][kStageIds];      // per warp, rows clubbed into one block only: (x mod R) d
 };
 
 // ids a warp stages per batch: as many as fit the staging area (and at least one)
@@ -74,13 +75,18 @@ __device__ __forceinline__ bool stage_batch(StageSmem& sm, const MapParams& mp,
     uint32_t* start_s = sm.start[w];
     for (uint32_t t = lane; t < cnt; t += 32) {
         const uint64_t x = (uint64_t)__ldg(indices + p0 + t);
+        uint64_t xh = x;  // what the location hash sees in place of the id
+        if (mp.R > 1) {   // R rows share a block: hashed by floor(x/R), row x starts (x mod R) d in
+            xh = x / mp.R;
+            sm.piece[w][t] = (uint32_t)(x - xh * mp.R) * mp.d;
+        }
         uint64_t tt = tterm, gt = gterm;
         if (!BAGS) {
             const uint32_t e = table_of_bag((uint64_t)(p0 + t), mp);
             tt = table_term(mp.h, e);
             if (SIGN) gt = table_term(mp.g, e);
         }
-        base_s[t] = addmod_p61(tt, mulmod_p61_any(mp.h.B, x));
+        base_s[t] = addmod_p61(tt, mulmod_p61_any(mp.h.B, xh));
         if (SIGN) gbase_s[t] = addmod_p61(gt, mulmod_p61_any(mp.g.B, x));
     }
     __syncwarp();
@@ -90,7 +96,11 @@ __device__ __forceinline__ bool stage_batch(StageSmem& sm, const MapParams& mp,
     for (uint32_t t = lane; t < entries; t += 32) {
         const uint32_t idl = (t * cmagic) >> 20;  // t / C, exact for t < 8192
         const uint32_t c = t - idl * mp.C;
-        const uint32_t s = mod_m(addmod_p61(base_s[idl], sm.cterm[c]), mp.m, mp.mu);
+        uint32_t s = mod_m(addmod_p61(base_s[idl], sm.cterm[c]), mp.m, mp.mu);
+        if (mp.R > 1) {
+            const uint64_t j = (uint64_t)s + sm.piece[w][idl];  // both below m
+            s = (uint32_t)(j >= mp.m ? j - mp.m : j);
+        }
         start_s[c * stride + idl] = s;
         wraps |= s > last_fit;
     }

@@ -38,7 +38,7 @@ def test_binding_has_no_fallback_import():
 
 
 @pytest.mark.parametrize("args", [
-    (0, 1, 1, 1), (10, 0, 4, 1), (10, 4, 0, 1), (10, 4, 4, 0), (10, 8, 4, 1), (3, 2, 4, 1),
+    (0, 1, 1, 1), (10, 0, 4, 1), (10, 4, 0, 1), (10, 4, 4, 0), (10, 6, 4, 1), (10, 12, 4, 1), (3, 2, 4, 1),
     (2**32, 4, 16, 1), (2**32 - 15, 4, 16, 1), (10**6, 4, 40000, 1),
 ])
 def test_create_rejects_bad_shapes(args):

@@ -42,6 +42,9 @@ SHAPES = [
     (128, 1, 4099), (128, 2, 4099), (128, 8, 4099), (128, 32, 129), (128, 128, 128),
     (128, 128, 100003), (64, 16, 70), (100, 32, 1013), (96, 64, 1013), (33, 1, 64), (7, 2, 9),
     (12, 5, 64), (48, 3, 49), (130, 2, 1000), (200, 64, 777), (256, 1, 513), (37, 37, 37),
+    # Z > d: rows clubbed into one block (R = Z/d = 4, 3, 4 with constant wrapping, 2, 2, 4, 2)
+    (16, 64, 1000), (16, 48, 1000), (8, 32, 33), (64, 128, 5000), (128, 256, 100003), (1, 4, 7),
+    (160, 320, 999),
 ]
 
 
@@ -153,6 +156,7 @@ BWD_SHAPES = [
     (16, 4, 4096), (16, 16, 17), (16, 4, 17), (1, 1, 1), (2, 2, 3), (128, 1, 4099), (128, 8, 4099),
     (128, 32, 129), (128, 128, 128), (64, 16, 70), (100, 32, 1013), (12, 5, 64), (48, 3, 49),
     (130, 2, 1000), (200, 64, 777), (37, 37, 37), (16, 8, 5000),
+    (16, 64, 1000), (16, 48, 1000), (8, 32, 33), (64, 128, 5000), (1, 4, 7), (160, 320, 999),
 ]
 
 
