@@ -313,35 +313,56 @@ def run_ours(args, w):
     nnz_per_step = float(np.mean([len(batches[(args.warmup + i) % NB][0]) for i in range(args.steps)]))
 
     # ---- end to end: host buffers in, result out, every step ------------------------------
+    # Three streams, two sets of buffers: while step i computes, the inputs of step i+1 come in
+    # from pinned host memory and the output of step i-1 goes back - what a caller that feeds the
+    # library from the host would do.  Every byte of every step still crosses the bus inside
+    # the timed region.
     h_ids = [torch.from_numpy(b[0]).pin_memory() for b in batches]
     h_offs = [None if b[1] is None else torch.from_numpy(b[1]).pin_memory() for b in batches]
     h_grad = grad_out.cpu().pin_memory()
-    h_out = torch.empty(B, T, d, dtype=torch.float32).pin_memory()
-    e_ids = torch.empty(max(len(b[0]) for b in batches), dtype=torch.int64, device=dev)
-    e_offs = torch.empty(nbags + 1, dtype=torch.int64, device=dev) if bags else None
-    e_grad = torch.empty_like(grad_out)
+    h_out = [torch.empty(B, T, d, dtype=torch.float32).pin_memory() for _ in range(2)]
+    max_nnz = max(len(b[0]) for b in batches)
+    e_ids = [torch.empty(max_nnz, dtype=torch.int64, device=dev) for _ in range(2)]
+    e_offs = [torch.empty(nbags + 1, dtype=torch.int64, device=dev) if bags else None for _ in range(2)]
+    e_grad = [torch.empty_like(grad_out) for _ in range(2)]
+    e_out = [torch.empty_like(out) for _ in range(2)]
+    s_in, s_comp, s_out = torch.cuda.Stream(dev), torch.cuda.Stream(dev), torch.cuda.Stream(dev)
+    ev_in = [torch.cuda.Event() for _ in range(2)]
+    ev_comp = [torch.cuda.Event() for _ in range(2)]
+    ev_out = [torch.cuda.Event() for _ in range(2)]
 
     def e2e_step(i):
-        k = i % NB
+        b, k = i % 2, i % NB
         n = h_ids[k].numel()
-        ids_d = e_ids[:n]
-        ids_d.copy_(h_ids[k], non_blocking=True)
-        if bags:
-            e_offs.copy_(h_offs[k], non_blocking=True)
-        e_grad.copy_(h_grad, non_blocking=True)
-        robe.robe_forward(h, ids_d, e_offs, B, out)
-        robe.robe_backward(h, e_grad, ids_d, e_offs, B, dense, lr, ws)
-        h_out.copy_(out, non_blocking=True)
+        ids_d = e_ids[b][:n]
+        with torch.cuda.stream(s_in):
+            s_in.wait_event(ev_comp[b])  # the step that last read this set of inputs is done
+            ids_d.copy_(h_ids[k], non_blocking=True)
+            if bags:
+                e_offs[b].copy_(h_offs[k], non_blocking=True)
+            e_grad[b].copy_(h_grad, non_blocking=True)
+            ev_in[b].record(s_in)
+        s_comp.wait_event(ev_in[b])
+        s_comp.wait_event(ev_out[b])     # the output buffer has been copied out
+        robe.robe_forward(h, ids_d, e_offs[b], B, e_out[b], stream=s_comp)
+        robe.robe_backward(h, e_grad[b], ids_d, e_offs[b], B, dense, lr, ws, stream=s_comp)
+        ev_comp[b].record(s_comp)
+        with torch.cuda.stream(s_out):
+            s_out.wait_event(ev_comp[b])
+            h_out[b].copy_(e_out[b], non_blocking=True)
+            ev_out[b].record(s_out)
 
-    e2e_steps = max(3, min(args.steps, 10))
-    for i in range(2):
+    e2e_steps = max(4, min(args.steps, 20))
+    for i in range(4):
         e2e_step(i)
     barrier()
     s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    s0.record()
+    s0.record(s_in)
     for i in range(e2e_steps):
         e2e_step(i)
-    s1.record()
+    s_out.wait_stream(s_comp)
+    s_out.wait_stream(s_in)
+    s1.record(s_out)
     barrier()
     e2e_ms = s0.elapsed_time(s1)
     e2e_nnz = float(np.mean([len(batches[i % NB][0]) for i in range(e2e_steps)]))
