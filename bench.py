@@ -52,16 +52,16 @@ def measured_peaks():
     return 6650.0, "fallback"
 
 
-def algorithmic_bytes(w, nbags, nnz, bags):
+def algorithmic_bytes(w, nbags, nnz, bags, id_bytes=8):
     """Bytes the method itself must move per launch (useful-bytes model):
-    forward  = 8 per id (index) + d*s_a per id (array elements read) + 8 per bag (offset, pooled
+    forward  = 8 (4 with int32 ids) per id (index) + d*s_a per id (array elements read) + 8 per bag (offset, pooled
                only) + 4d per bag (output row written);
     backward = 8 per id + 2*4d per id (read-modify-write of the slots) + 8 per bag (pooled only)
                + 4d per bag (gradient row read once)."""
     s_a = 4 if w.array_dtype == "f32" else 2
     off = 8 * (nbags + 1) if bags else 0
-    fwd = 8 * nnz + w.d * s_a * nnz + off + 4 * w.d * nbags
-    bwd = 8 * nnz + 2 * 4 * w.d * nnz + off + 4 * w.d * nbags
+    fwd = id_bytes * nnz + w.d * s_a * nnz + off + 4 * w.d * nbags
+    bwd = id_bytes * nnz + 2 * 4 * w.d * nnz + off + 4 * w.d * nbags
     return fwd, bwd
 
 
@@ -257,7 +257,9 @@ def run_ours(args, w):
     gen.manual_seed(w.data_seed + 17 * rank)
     grad_out = torch.randn(B, T, d, device=dev, dtype=torch.float32, generator=gen)
     out = torch.empty(B, T, d, device=dev, dtype=torch.float32)
-    d_ids = [torch.from_numpy(b[0]).to(dev) for b in batches]
+    id_dtype = torch.int32 if args.ids == "int32" else torch.int64
+    id_bytes = 4 if args.ids == "int32" else 8
+    d_ids = [torch.from_numpy(b[0]).to(dev).to(id_dtype) for b in batches]
     d_offs = [None if b[1] is None else torch.from_numpy(b[1]).to(dev) for b in batches]
 
     h = robe.robe_create(w.M, w.Z, w.d, T, w.hash_seed)
@@ -317,12 +319,12 @@ def run_ours(args, w):
     # from pinned host memory and the output of step i-1 goes back - what a caller that feeds the
     # library from the host would do.  Every byte of every step still crosses the bus inside
     # the timed region.
-    h_ids = [torch.from_numpy(b[0]).pin_memory() for b in batches]
+    h_ids = [torch.from_numpy(b[0]).to(id_dtype).pin_memory() for b in batches]
     h_offs = [None if b[1] is None else torch.from_numpy(b[1]).pin_memory() for b in batches]
     h_grad = grad_out.cpu().pin_memory()
     h_out = [torch.empty(B, T, d, dtype=torch.float32).pin_memory() for _ in range(2)]
     max_nnz = max(len(b[0]) for b in batches)
-    e_ids = [torch.empty(max_nnz, dtype=torch.int64, device=dev) for _ in range(2)]
+    e_ids = [torch.empty(max_nnz, dtype=id_dtype, device=dev) for _ in range(2)]
     e_offs = [torch.empty(nbags + 1, dtype=torch.int64, device=dev) if bags else None for _ in range(2)]
     e_grad = [torch.empty_like(grad_out) for _ in range(2)]
     e_out = [torch.empty_like(out) for _ in range(2)]
@@ -366,7 +368,7 @@ def run_ours(args, w):
     barrier()
     e2e_ms = s0.elapsed_time(s1)
     e2e_nnz = float(np.mean([len(batches[i % NB][0]) for i in range(e2e_steps)]))
-    h2d = int(8 * e2e_nnz + (8 * (nbags + 1) if bags else 0) + 4 * nbags * d)
+    h2d = int(id_bytes * e2e_nnz + (8 * (nbags + 1) if bags else 0) + 4 * nbags * d)
     d2h = int(4 * nbags * d)
 
     # ---- max over ranks --------------------------------------------------------------------
@@ -381,10 +383,10 @@ def run_ours(args, w):
         return 0
 
     peak, peak_kind = measured_peaks()
-    fwd_bytes, bwd_bytes = algorithmic_bytes(w, nbags, nnz_per_step, bags)
+    fwd_bytes, bwd_bytes = algorithmic_bytes(w, nbags, nnz_per_step, bags, id_bytes)
     dominant = "backward" if bwd_ms >= fwd_ms else "forward"
     dom_bytes, dom_ms = (bwd_bytes, bwd_ms) if dominant == "backward" else (fwd_bytes, fwd_ms)
-    traffic = NCU_TRAFFIC_BYTES.get((w.name, args.backward), {})
+    traffic = NCU_TRAFFIC_BYTES.get((w.name, args.backward), {}) if args.ids == "int64" else {}
 
     def roof(nbytes, ms, which):
         ach = nbytes / (ms * 1e-3) / 1e9
@@ -405,7 +407,7 @@ def run_ours(args, w):
         "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": w.name, "num_tables": T, "d": d, "Z": w.Z, "M": w.M, "batch_per_gpu": B,
-                   "ids_per_step_per_gpu": nnz_per_step, "bags": bags, "backward": ("atomic" if args.backward == "atomic" else "deterministic") +
+                   "ids_per_step_per_gpu": nnz_per_step, "ids": args.ids, "bags": bags, "backward": ("atomic" if args.backward == "atomic" else "deterministic") +
                    (", SGD fused" if dense is None else ", dense fp32 gradient"),
                    "l2": l2_note,
                    "parallelism": f"dp{world} replicas, no collective"},
@@ -441,6 +443,7 @@ def main():
     ap.add_argument("--workload", default="cfg4", help=WORKLOAD_HELP)
     ap.add_argument("--backward", default="atomic", choices=["atomic", "det"],
                     help="backward variant of the step (default: atomic red.global adds)")
+    ap.add_argument("--ids", default="int64", choices=["int64", "int32"], help="element type of the id arrays")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=0,
                     help="samples per GPU instead of the workload's own batch (small profiler captures)")

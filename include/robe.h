@@ -61,6 +61,13 @@ typedef enum {
                                  kernel variant, for benchmarking only                    */
 #define ROBE_OPT_BWD_KERNEL 5 /* same for the atomic backward                             */
 
+#define ROBE_OPT_INDEX_TYPE 6 /* ROBE_I64 (default) | ROBE_I32: element type of `indices` in the
+                                 calls that follow (offsets stay int64)                   */
+
+/* index element types */
+#define ROBE_I64 0
+#define ROBE_I32 1
+
 #define ROBE_BWD_ATOMIC 0
 #define ROBE_BWD_DETERMINISTIC 1
 
@@ -119,14 +126,15 @@ int robe_get_hash_constants(robe_handle_t h, uint64_t out[9]);
  * robe_forward - embedding lookup with optional sum pooling (Section 3.2 forward).
  *   out[n,e,i] = sum over ids x_p of bag (n,e), in bag order, sequentially in fp32
  *                (first term initialises), of g(e,x_p,i) * M[(h(e,x_p,i/Z) + i%Z) mod M]
- *   indices  device pointer, int64 [nnz], ids >= 0.
+ *   indices  device pointer, int64 [nnz] (int32 [nnz] after ROBE_OPT_INDEX_TYPE = ROBE_I32),
+ *            ids >= 0.
  *   offsets  device pointer, int64 [batch*T + 1], offsets[0] = 0, non-decreasing,
  *            offsets[batch*T] = nnz; or NULL for one-hot (then nnz == batch*T).
  *   batch    number of samples B >= 0;  nnz >= 0 total ids.
  *   out      device pointer, fp32 [batch, T, d], fully overwritten; an empty bag gives +0.
  * Errors: ROBE_ERR_INVALID_ARG, ROBE_ERR_NO_ARRAY, ROBE_ERR_CUDA.
  */
-int robe_forward(robe_handle_t h, const int64_t* indices, const int64_t* offsets, int64_t batch,
+int robe_forward(robe_handle_t h, const void* indices, const int64_t* offsets, int64_t batch,
                  int64_t nnz, float* out, void* stream);
 
 /*
@@ -155,7 +163,7 @@ size_t robe_backward_workspace_bytes(robe_handle_t h, int64_t batch, int64_t nnz
  * Errors: ROBE_ERR_INVALID_ARG (also: fused SGD on a bf16 array), ROBE_ERR_NO_ARRAY,
  * ROBE_ERR_WORKSPACE, ROBE_ERR_CUDA.
  */
-int robe_backward(robe_handle_t h, const float* grad_out, const int64_t* indices,
+int robe_backward(robe_handle_t h, const float* grad_out, const void* indices,
                   const int64_t* offsets, int64_t batch, int64_t nnz, float* grad_array, float lr,
                   void* workspace, size_t workspace_bytes, void* stream);
 
@@ -199,7 +207,7 @@ int robe_backward(robe_handle_t h, const float* grad_out, const int64_t* indices
  */
 #define ROBE_STATIC_SCRATCH_BYTES (32u << 20) /* 32 MiB per device */
 int robe_backward_deterministic_static(robe_handle_t h, const float* grad_out,
-                                       const int64_t* indices, const int64_t* offsets,
+                                       const void* indices, const int64_t* offsets,
                                        int64_t batch, int64_t nnz, float* grad_array, float lr,
                                        void* stream);
 

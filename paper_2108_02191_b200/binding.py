@@ -30,6 +30,10 @@ ROBE_OPT_BWD_MODE = 2
 ROBE_OPT_VALIDATE = 3
 ROBE_OPT_FWD_KERNEL = 4
 ROBE_OPT_BWD_KERNEL = 5
+ROBE_OPT_INDEX_TYPE = 6
+
+ROBE_I64 = 0
+ROBE_I32 = 1
 
 ROBE_BWD_ATOMIC = 0
 ROBE_BWD_DETERMINISTIC = 1
@@ -99,6 +103,21 @@ def _stream_ptr(stream):
     return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
 
 
+def _ids_ptr(t):
+    """Device pointer of an id tensor: int64, or int32 for a handle set to ROBE_I32 (the handle's
+    option says which the library reads; nothing is converted here)."""
+    if t.dtype not in (torch.int64, torch.int32):
+        raise TypeError(f"indices must be int64 or int32, got {t.dtype}")
+    return _dev_ptr(t)
+
+
+def _state_index_type(h, indices) -> None:
+    """Tells the handle which element type the id tensor of the coming call has (the C ABI
+    states it through ROBE_OPT_INDEX_TYPE, a tensor carries it in its dtype)."""
+    _check(_lib.robe_set_option(h, ROBE_OPT_INDEX_TYPE,
+                                ROBE_I32 if indices.dtype == torch.int32 else ROBE_I64), "robe_set_option")
+
+
 def robe_status_string(status: int) -> str:
     return _lib.robe_status_string(status).decode()
 
@@ -136,7 +155,8 @@ def robe_get_hash_constants(h):
 
 
 def robe_forward(h, indices, offsets, batch: int, out, stream=None) -> None:
-    _check(_lib.robe_forward(h, _dev_ptr(indices, torch.int64), _dev_ptr(offsets, torch.int64),
+    _state_index_type(h, indices)
+    _check(_lib.robe_forward(h, _ids_ptr(indices), _dev_ptr(offsets, torch.int64),
                              batch, indices.numel(), _dev_ptr(out, torch.float32),
                              _stream_ptr(stream)), "robe_forward")
 
@@ -147,8 +167,9 @@ def robe_backward_workspace_bytes(h, batch: int, nnz: int) -> int:
 
 def robe_backward(h, grad_out, indices, offsets, batch: int, grad_array=None, lr: float = 0.0,
                   workspace=None, stream=None) -> None:
+    _state_index_type(h, indices)
     ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
-    _check(_lib.robe_backward(h, _dev_ptr(grad_out, torch.float32), _dev_ptr(indices, torch.int64),
+    _check(_lib.robe_backward(h, _dev_ptr(grad_out, torch.float32), _ids_ptr(indices),
                               _dev_ptr(offsets, torch.int64), batch, indices.numel(),
                               _dev_ptr(grad_array, torch.float32), lr, _dev_ptr(workspace),
                               ws_bytes, _stream_ptr(stream)), "robe_backward")
@@ -159,8 +180,9 @@ def robe_backward_deterministic_static(h, grad_out, indices, offsets, batch: int
     """Deterministic backward on the library's built-in scratch array, for callers that cannot
     allocate a workspace (include/robe.h has the limit and the sharing rules).  No tensor is
     created here: the arguments are passed through as they are."""
+    _state_index_type(h, indices)
     _check(_lib.robe_backward_deterministic_static(
-        h, _dev_ptr(grad_out, torch.float32), _dev_ptr(indices, torch.int64),
+        h, _dev_ptr(grad_out, torch.float32), _ids_ptr(indices),
         _dev_ptr(offsets, torch.int64), batch, indices.numel(), _dev_ptr(grad_array, torch.float32),
         lr, _stream_ptr(stream)), "robe_backward_deterministic_static")
 

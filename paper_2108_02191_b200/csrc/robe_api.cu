@@ -26,6 +26,7 @@ struct robe_ctx {
     int fwd_variant;
     int bwd_variant;
     int32_t* status_word;
+    int index_type;
 };
 
 namespace {
@@ -53,10 +54,10 @@ void draw_constants(uint64_t seed, uint64_t out[9]) {
     }
 }
 
-__global__ void validate_kernel(const int64_t* indices, const int64_t* offsets, int64_t nbags,
+__global__ void validate_kernel(IdList indices, const int64_t* offsets, int64_t nbags,
                                 int64_t nnz, int32_t* status) {
     const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (t < nnz && indices[t] < 0) atomicCAS(status, ROBE_DEV_OK, ROBE_DEV_BAD_INDEX);
+    if (t < nnz && indices.load(t) < 0) atomicCAS(status, ROBE_DEV_OK, ROBE_DEV_BAD_INDEX);
     if (offsets != nullptr && t <= nbags) {
         const int64_t o = offsets[t];
         bool bad = o < 0 || o > nnz;
@@ -67,7 +68,7 @@ __global__ void validate_kernel(const int64_t* indices, const int64_t* offsets, 
     }
 }
 
-bool check_sizes(robe_ctx* h, const int64_t* indices, const int64_t* offsets, int64_t batch,
+bool check_sizes(robe_ctx* h, const void* indices, const int64_t* offsets, int64_t batch,
                  int64_t nnz) {
     if (h == nullptr || batch < 0 || nnz < 0) return false;
     if (nnz > 0 && indices == nullptr) return false;
@@ -77,14 +78,14 @@ bool check_sizes(robe_ctx* h, const int64_t* indices, const int64_t* offsets, in
     return true;
 }
 
-Problem make_problem(robe_ctx* h, const int64_t* indices, const int64_t* offsets, int64_t batch,
+Problem make_problem(robe_ctx* h, const void* indices, const int64_t* offsets, int64_t batch,
                      int64_t nnz) {
     Problem pb;
     pb.mp = h->mp;
     pb.array = h->array;
     pb.dtype = h->dtype;
     pb.sign = h->sign;
-    pb.indices = indices;
+    pb.indices = IdList{indices, h->index_type == ROBE_I32 ? 1 : 0};
     pb.offsets = offsets;
     pb.nbags = batch * (int64_t)h->T;
     pb.nnz = nnz;
@@ -149,6 +150,7 @@ int robe_create(robe_handle_t* out, uint64_t M, uint32_t Z, uint32_t d, uint32_t
     h->fwd_variant = 0;
     h->bwd_variant = 0;
     h->status_word = nullptr;
+    h->index_type = ROBE_I64;
     *out = h;
     return ROBE_OK;
 }
@@ -178,6 +180,10 @@ int robe_set_option(robe_handle_t h, int key, int64_t value) {
         case ROBE_OPT_FWD_KERNEL:
             if (value < 0 || value > 2) return ROBE_ERR_INVALID_ARG;
             h->fwd_variant = (int)value;
+            return ROBE_OK;
+        case ROBE_OPT_INDEX_TYPE:
+            if (value != ROBE_I64 && value != ROBE_I32) return ROBE_ERR_INVALID_ARG;
+            h->index_type = (int)value;
             return ROBE_OK;
         case ROBE_OPT_BWD_KERNEL:
             if (value < 0 || value > 2) return ROBE_ERR_INVALID_ARG;
@@ -219,7 +225,7 @@ int robe_last_device_status(robe_handle_t h, void* stream) {
     return (int)v;
 }
 
-int robe_forward(robe_handle_t h, const int64_t* indices, const int64_t* offsets, int64_t batch,
+int robe_forward(robe_handle_t h, const void* indices, const int64_t* offsets, int64_t batch,
                  int64_t nnz, float* out, void* stream) {
     if (!check_sizes(h, indices, offsets, batch, nnz)) return ROBE_ERR_INVALID_ARG;
     if (batch > 0 && out == nullptr) return ROBE_ERR_INVALID_ARG;
@@ -239,7 +245,7 @@ size_t robe_backward_workspace_bytes(robe_handle_t h, int64_t batch, int64_t nnz
     return det_workspace_bytes(h->mp, batch * (int64_t)h->T, nnz, true);
 }
 
-int robe_backward(robe_handle_t h, const float* grad_out, const int64_t* indices,
+int robe_backward(robe_handle_t h, const float* grad_out, const void* indices,
                   const int64_t* offsets, int64_t batch, int64_t nnz, float* grad_array, float lr,
                   void* workspace, size_t workspace_bytes, void* stream) {
     if (!check_sizes(h, indices, offsets, batch, nnz)) return ROBE_ERR_INVALID_ARG;
@@ -297,7 +303,7 @@ static int static_scratch_address(void** out) {
 }
 
 int robe_backward_deterministic_static(robe_handle_t h, const float* grad_out,
-                                       const int64_t* indices, const int64_t* offsets,
+                                       const void* indices, const int64_t* offsets,
                                        int64_t batch, int64_t nnz, float* grad_array, float lr,
                                        void* stream) {
     if (!check_sizes(h, indices, offsets, batch, nnz)) return ROBE_ERR_INVALID_ARG;

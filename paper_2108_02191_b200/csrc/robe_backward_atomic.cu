@@ -15,7 +15,7 @@ namespace robe {
 struct BwdArgs {
     MapParams mp;
     const float* grad_out;
-    const int64_t* indices;
+    IdList indices;
     const int64_t* offsets;
     float* target;
     float scale;
@@ -39,7 +39,7 @@ __global__ void __launch_bounds__(256) bwd_atomic_direct_kernel(BwdArgs a) {
         chunk_of(mp, i, c, o);
         const float gv = __ldcs(a.grad_out + k * mp.d + i) * a.scale;
         for (int64_t p = lo; p < hi; ++p) {
-            const uint64_t x = (uint64_t)__ldg(a.indices + p);
+            const uint64_t x = (uint64_t)a.indices.load(p);
             uint32_t j = id_block_start(mp, e, x, c) + o;
             if (j >= mp.m) j -= mp.m;
             float t = gv;

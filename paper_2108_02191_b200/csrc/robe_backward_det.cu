@@ -56,7 +56,7 @@ __device__ __forceinline__ void cta_tiles(uint64_t tiles, uint32_t grid, uint32_
 
 struct KeyArgs {
     MapParams mp;
-    const int64_t* indices;
+    IdList indices;
     const int64_t* offsets;
     int64_t nbags;
     int64_t nnz;
@@ -86,7 +86,7 @@ det_keys_kernel(KeyArgs a, const uint32_t* bag_of, uint32_t* keys, uint32_t* val
     const uint32_t c = (uint32_t)q - p * mp.C;
     const uint64_t bag = bag_of ? (uint64_t)bag_of[p] : (uint64_t)p;
     const uint32_t e = table_of_bag(bag, mp);
-    const uint64_t x = (uint64_t)__ldg(a.indices + p);
+    const uint64_t x = (uint64_t)a.indices.load(p);
     keys[q] = id_block_start(mp, e, x, c);
     vals[q] = SIGN ? (uint32_t)q : (uint32_t)(bag * mp.d + c * mp.Z);
 }
@@ -262,7 +262,7 @@ struct LongWalk {
 struct ApplyArgs {
     MapParams mp;
     const float* grad_out;
-    const int64_t* indices;  // only read when the sign hash is on
+    IdList indices;  // only read when the sign hash is on
     float* target;
     float lr;
     uint64_t nb;
@@ -293,7 +293,7 @@ __device__ __forceinline__ bool block_term(const ApplyArgs& a, const uint32_t* b
     if (i >= mp.d) return false;
     const uint64_t bag = bag_of ? (uint64_t)__ldg(bag_of + p) : (uint64_t)p;
     const uint32_t e = table_of_bag(bag, mp);
-    const uint64_t x = (uint64_t)__ldg(a.indices + p);
+    const uint64_t x = (uint64_t)a.indices.load(p);
     term = sign_of(mp, hash_base(mp.g, e, x), i) * __ldg(a.grad_out + bag * mp.d + i);
     return true;
 }

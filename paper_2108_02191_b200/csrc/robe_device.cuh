@@ -20,6 +20,15 @@ struct HashConsts {  // all < P
     uint64_t A, B, C, D;
 };
 
+// The ids of a call: int64 (default) or int32 elements, read through the read-only path.
+struct IdList {
+    const void* p;
+    int i32;  // 0: int64_t elements, 1: int32_t elements
+    __device__ __forceinline__ int64_t load(int64_t pos) const {
+        return i32 ? (int64_t)__ldg((const int32_t*)p + pos) : __ldg((const int64_t*)p + pos);
+    }
+};
+
 // Everything a kernel needs to map (e, x, c) to a block start.
 struct MapParams {
     HashConsts h;      // location hash

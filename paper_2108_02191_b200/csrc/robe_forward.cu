@@ -16,7 +16,7 @@ namespace robe {
 struct FwdArgs {
     MapParams mp;
     const void* array;
-    const int64_t* indices;
+    IdList indices;
     const int64_t* offsets;
     float* out;
     int64_t nbags;
@@ -39,7 +39,7 @@ __global__ void __launch_bounds__(256) fwd_direct_kernel(FwdArgs a) {
         chunk_of(mp, i, c, o);
         float acc = 0.0f;
         for (int64_t p = lo; p < hi; ++p) {
-            const uint64_t x = (uint64_t)__ldg(a.indices + p);
+            const uint64_t x = (uint64_t)a.indices.load(p);
             uint32_t j = id_block_start(mp, e, x, c) + o;  // < m + d <= 2^32
             if (j >= mp.m) j -= mp.m;
             float v = load_elem<DT>(a.array, j);

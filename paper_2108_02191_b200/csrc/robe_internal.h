@@ -13,7 +13,7 @@ struct Problem {
     const void* array;       // device, M elements
     int dtype;               // 0 fp32, 1 bf16
     int sign;                // 0 / 1
-    const int64_t* indices;  // device [nnz]
+    IdList indices;          // device [nnz], int64 or int32
     const int64_t* offsets;  // device [nbags+1] or nullptr (one-hot)
     int64_t nbags;           // batch * T
     int64_t nnz;

@@ -67,14 +67,14 @@ __device__ __forceinline__ void stage_init(StageSmem& sm, const MapParams& mp) {
 // the end of the array, i.e. whether the gather has to wrap slot numbers at all.
 template <bool SIGN, bool BAGS>
 __device__ __forceinline__ bool stage_batch(StageSmem& sm, const MapParams& mp,
-                                            const int64_t* indices, int64_t p0, uint32_t cnt,
+                                            const IdList& indices, int64_t p0, uint32_t cnt,
                                             uint32_t stride, uint64_t tterm, uint64_t gterm,
                                             uint32_t cmagic, uint32_t w, uint32_t lane) {
     uint64_t* base_s = sm.base[w];
     uint64_t* gbase_s = base_s + kStageIds / 2;
     uint32_t* start_s = sm.start[w];
     for (uint32_t t = lane; t < cnt; t += 32) {
-        const uint64_t x = (uint64_t)__ldg(indices + p0 + t);
+        const uint64_t x = (uint64_t)indices.load(p0 + t);
         uint64_t xh = x;  // what the location hash sees in place of the id
         if (mp.R > 1) {   // R rows share a block: hashed by floor(x/R), row x starts (x mod R) d in
             xh = x / mp.R;

@@ -71,6 +71,26 @@ def test_forward_bf16_array():
             assert_bits_equal(c.forward(kernel).cpu().numpy(), want, "bf16")
 
 
+@pytest.mark.parametrize("bags", [None, (3, 0, 9)])
+def test_int32_indices(bags):
+    # the same ids as int32: identical bits out of every kernel
+    for w in (synth.workload(1).with_(bag_rule=bags), small(d=128, Z=32, M=4099, bag_rule=bags, batch=97),
+              small(d=16, Z=64, M=1000, bag_rule=bags, batch=97)):
+        for sign in (False, True):
+            with Case(w, sign=sign) as c:
+                want = c.oracle_forward()
+                g_h, g_d = _grad(c, 7)
+                delta64, l1 = c.oracle.backward_f64(g_h, c.indices_h, c.offsets_h, c.B)
+                can, _ = c.oracle.backward_canonical(g_h, c.indices_h, c.offsets_h, c.B)
+                c.indices = c.indices.to(torch.int32)
+                for kernel in FWD_KERNELS:
+                    assert_bits_equal(c.forward(kernel).cpu().numpy(), want, "int32 ids forward")
+                for kernel in (1, 2):
+                    assert_within_l1(c.backward(g_d, "atomic", kernel=kernel).cpu().numpy(), delta64, l1,
+                                     what="int32 ids atomic")
+                assert_bits_equal(c.backward(g_d, "det").cpu().numpy(), can, "int32 ids deterministic")
+
+
 def test_forward_empty_and_degenerate_inputs():
     w = small(bag_rule=(2, 0, 5))
     with Case(w, batch=4) as c:
