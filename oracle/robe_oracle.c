@@ -337,3 +337,32 @@ void robe_oracle_accumulate(float *grad_array, const float *delta, const uint8_t
     for (uint64_t j = 0; j < n; ++j)
         if (touched[j]) grad_array[j] = grad_array[j] + delta[j];
 }
+
+/* Adam step (Kingma & Ba, Algorithm 1; Section 5 trains five of the six models with Adam) on
+   the slots that received at least one term, in fp32, one operation at a time:
+     m1 <- beta1 m1 + (1-beta1) g;  m2 <- beta2 m2 + (1-beta2) g^2
+     M  <- M - lr (m1 / bias1) / (sqrt(m2 / bias2) + eps),  bias_k = 1 - beta_k^t (passed in)
+   Slots without a term keep M, m1 and m2 (lazy update). */
+void robe_oracle_adam_apply(float *array, float *m1, float *m2, const float *delta,
+                            const uint8_t *touched, uint64_t n, float lr, float beta1, float beta2,
+                            float eps, float bias1, float bias2) {
+    for (uint64_t j = 0; j < n; ++j) {
+        if (!touched[j]) continue;
+        float g = delta[j];
+        float a = beta1 * m1[j];
+        float b = (1.0f - beta1) * g;
+        float m = a + b;
+        float c = beta2 * m2[j];
+        float gg = g * g;
+        float dd = (1.0f - beta2) * gg;
+        float v = c + dd;
+        m1[j] = m;
+        m2[j] = v;
+        float mhat = m / bias1;
+        float vhat = v / bias2;
+        float den = sqrtf(vhat) + eps;
+        float upd = mhat / den;
+        float step = lr * upd;
+        array[j] = array[j] - step;
+    }
+}

@@ -57,6 +57,7 @@ def lib() -> C.CDLL:
         _lib.robe_oracle_backward_canonical.restype = C.c_int
         _lib.robe_oracle_sgd_apply.argtypes = [p, p, p, u64, C.c_float]
         _lib.robe_oracle_accumulate.argtypes = [p, p, p, u64]
+        _lib.robe_oracle_adam_apply.argtypes = [p, p, p, p, p, u64] + [C.c_float] * 6
     return _lib
 
 
@@ -170,3 +171,17 @@ def accumulate(grad_array, delta, touched) -> None:
     """In place: grad_array[j] = grad_array[j] + delta[j] on touched slots."""
     assert grad_array.dtype == np.float32 and delta.dtype == np.float32
     lib().robe_oracle_accumulate(_ptr(grad_array), _ptr(delta), _ptr(touched), len(delta))
+
+
+def adam_bias(beta: float, step: int) -> np.float32:
+    """1 - beta^t, from the fp32 value of beta, evaluated in double and rounded to fp32."""
+    return np.float32(1.0 - float(np.float32(beta)) ** step)
+
+
+def adam_apply(array, m1, m2, delta, touched, lr, beta1, beta2, eps, step) -> None:
+    """In place: one lazy Adam step (update number `step`) on the touched slots."""
+    for a in (array, m1, m2, delta):
+        assert a.dtype == np.float32
+    lib().robe_oracle_adam_apply(_ptr(array), _ptr(m1), _ptr(m2), _ptr(delta), _ptr(touched), len(delta),
+                                 C.c_float(lr), C.c_float(beta1), C.c_float(beta2), C.c_float(eps),
+                                 C.c_float(adam_bias(beta1, step)), C.c_float(adam_bias(beta2, step)))

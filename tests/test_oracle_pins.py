@@ -527,6 +527,39 @@ def test_sgd_apply_and_accumulate():
 # 7. Theorem 1: the sketch's inner-product estimator is unbiased with the printed variance
 # ---------------------------------------------------------------------------------------
 
+def test_adam_apply_matches_torch_adam_and_closed_form():
+    # all slots touched: the lazy step is the textbook one, so torch.optim.Adam (a library routine,
+    # fp32) must agree to rounding over several steps; and step 1 has the closed form
+    # M - lr g / (|g| + eps) whatever the betas are
+    import torch
+    rng = np.random.default_rng(11)
+    n, lr, b1, b2, eps = 1000, 0.01, 0.9, 0.999, 1e-8
+    arr = rng.standard_normal(n).astype(np.float32)
+    m1, m2 = np.zeros(n, np.float32), np.zeros(n, np.float32)
+    p = torch.nn.Parameter(torch.from_numpy(arr.copy()))
+    opt = torch.optim.Adam([p], lr=lr, betas=(b1, b2), eps=eps)
+    ones = np.ones(n, np.uint8)
+    first = None
+    for t in range(1, 6):
+        g = rng.standard_normal(n).astype(np.float32)
+        if t == 1:
+            first = arr.astype(np.float64) - lr * g / (np.abs(g.astype(np.float64)) + eps)
+        orc.adam_apply(arr, m1, m2, g, ones, lr, b1, b2, eps, t)
+        if t == 1:
+            np.testing.assert_allclose(arr, first, rtol=0, atol=2e-7)
+        p.grad = torch.from_numpy(g.copy())
+        opt.step()
+        np.testing.assert_allclose(arr, p.detach().numpy(), rtol=0, atol=5e-7)
+    # lazy: an untouched slot keeps array and moments bit for bit
+    before = (arr.copy(), m1.copy(), m2.copy())
+    touched = np.zeros(n, np.uint8)
+    touched[::3] = 1
+    orc.adam_apply(arr, m1, m2, rng.standard_normal(n).astype(np.float32), touched, lr, b1, b2, eps, 6)
+    for now, was in zip((arr, m1, m2), before):
+        np.testing.assert_array_equal(now[touched == 0], was[touched == 0])
+        assert np.all(now[touched == 1] != was[touched == 1])
+
+
 def test_theorem_1_mean_and_variance_monte_carlo():
     # parameter vector of n = V*d entries (one table), sketched into m slots with the sign hash on.
     # Theorem 1: E = <x,y>,  V = (1/m) * sum over i,j in different blocks of (x_i^2 y_j^2 + x_i y_i x_j y_j)
