@@ -168,6 +168,30 @@ int robe_backward(robe_handle_t h, const float* grad_out, const void* indices,
                   void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * robe_backward_adam - deterministic backward with the Adam step fused in (the paper trains
+ * five of its six Criteo-Kaggle models with Adam, Section 5; the update is Algorithm 1 of
+ * Kingma & Ba, "Adam: a method for stochastic optimization").  For every array slot j that
+ * receives at least one gradient term, with delta[j] summed in the deterministic order of
+ * robe_backward:
+ *     m1[j] = beta1 m1[j] + (1 - beta1) delta[j]
+ *     m2[j] = beta2 m2[j] + (1 - beta2) delta[j]^2
+ *     M[j]  = M[j] - lr * (m1[j] / (1 - beta1^step)) / (sqrt(m2[j] / (1 - beta2^step)) + eps)
+ * each operation a separate round-to-nearest fp32 one; slots without a term keep M, m1 and m2
+ * as they are (the "lazy" form that sparse embedding updates use).  Bit-reproducible.
+ *   m1, m2   device pointers, fp32 [M], caller-owned, zeroed by the caller before step 1.
+ *   step     t >= 1, the number of this update (used for the bias corrections only).
+ *   workspace / workspace_bytes  as for robe_backward in deterministic mode; size it with
+ *            robe_backward_workspace_bytes after ROBE_OPT_BWD_MODE = ROBE_BWD_DETERMINISTIC.
+ * The handle's ROBE_OPT_BWD_MODE is not consulted.  The attached array must be fp32.
+ * Errors: as robe_backward; ROBE_ERR_INVALID_ARG also for null moments, step < 1, beta outside
+ * [0, 1) or eps < 0.
+ */
+int robe_backward_adam(robe_handle_t h, const float* grad_out, const void* indices,
+                       const int64_t* offsets, int64_t batch, int64_t nnz, float* m1, float* m2,
+                       float lr, float beta1, float beta2, float eps, int64_t step, void* workspace,
+                       size_t workspace_bytes, void* stream);
+
+/*
  * robe_backward_deterministic_static - the deterministic robe_backward for callers that
  * cannot supply scratch memory.  (The paper has no counterpart: this is a convenience of
  * this library, not part of the method.)

@@ -44,7 +44,7 @@ EXPORTS = [
     "robe_create", "robe_destroy", "robe_set_option", "robe_attach_array",
     "robe_get_hash_constants", "robe_forward", "robe_backward_workspace_bytes", "robe_backward",
     "robe_set_status_word", "robe_last_device_status", "robe_status_string",
-    "robe_backward_deterministic_static",
+    "robe_backward_deterministic_static", "robe_backward_adam",
 ]
 
 if not os.path.exists(LIB_PATH):
@@ -65,6 +65,8 @@ _lib.robe_backward_workspace_bytes.argtypes = [_vp, _i64, _i64]
 _lib.robe_backward_workspace_bytes.restype = C.c_size_t
 _lib.robe_backward.argtypes = [_vp, _vp, _vp, _vp, _i64, _i64, _vp, C.c_float, _vp, C.c_size_t, _vp]
 _lib.robe_backward_deterministic_static.argtypes = [_vp, _vp, _vp, _vp, _i64, _i64, _vp, C.c_float, _vp]
+_lib.robe_backward_adam.argtypes = [_vp, _vp, _vp, _vp, _i64, _i64, _vp, _vp, C.c_float, C.c_float,
+                                    C.c_float, C.c_float, _i64, _vp, C.c_size_t, _vp]
 _lib.robe_set_status_word.argtypes = [_vp, _vp]
 _lib.robe_last_device_status.argtypes = [_vp, _vp]
 _lib.robe_status_string.argtypes = [C.c_int]
@@ -185,6 +187,16 @@ def robe_backward_deterministic_static(h, grad_out, indices, offsets, batch: int
         h, _dev_ptr(grad_out, torch.float32), _ids_ptr(indices),
         _dev_ptr(offsets, torch.int64), batch, indices.numel(), _dev_ptr(grad_array, torch.float32),
         lr, _stream_ptr(stream)), "robe_backward_deterministic_static")
+
+
+def robe_backward_adam(h, grad_out, indices, offsets, batch: int, m1, m2, lr: float, beta1: float,
+                       beta2: float, eps: float, step: int, workspace, stream=None) -> None:
+    _state_index_type(h, indices)
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(_lib.robe_backward_adam(
+        h, _dev_ptr(grad_out, torch.float32), _ids_ptr(indices), _dev_ptr(offsets, torch.int64), batch,
+        indices.numel(), _dev_ptr(m1, torch.float32), _dev_ptr(m2, torch.float32), lr, beta1, beta2, eps,
+        step, _dev_ptr(workspace), ws_bytes, _stream_ptr(stream)), "robe_backward_adam")
 
 
 def robe_set_status_word(h, word) -> None:

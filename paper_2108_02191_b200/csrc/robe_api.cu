@@ -1,5 +1,6 @@
 // C ABI of librobe.so: handle, options, argument checks, hash-constant draw, dispatch.
 // The entry points are documented in include/robe.h.
+#include <cmath>
 #include <mutex>
 #include <new>
 
@@ -277,7 +278,7 @@ int robe_backward(robe_handle_t h, const float* grad_out, const void* indices,
     if (nnz > 0 && (workspace == nullptr || workspace_bytes < need)) return ROBE_ERR_WORKSPACE;
     if (((uintptr_t)workspace & 255u) != 0) return ROBE_ERR_WORKSPACE;
     if (launch_validate(pb, st) != cudaSuccess) return ROBE_ERR_CUDA;
-    if (launch_backward_det(pb, grad_out, target, sgd ? 1 : 0, lr, workspace, workspace_bytes,
+    if (launch_backward_det(pb, grad_out, target, sgd ? 1 : 0, lr, nullptr, workspace, workspace_bytes,
                             st) != cudaSuccess)
         return ROBE_ERR_CUDA;
     return ROBE_OK;
@@ -334,8 +335,46 @@ int robe_backward_deterministic_static(robe_handle_t h, const float* grad_out,
     // Stale contents are harmless: keys, values and digit counters are fully rewritten before
     // they are read, and the one buffer that must start from zero (the bag number of each id,
     // pooled input only) is cleared by the launch itself on the same stream.
-    if (launch_backward_det(pb, grad_out, target, sgd ? 1 : 0, lr, scratch,
+    if (launch_backward_det(pb, grad_out, target, sgd ? 1 : 0, lr, nullptr, scratch,
                             (size_t)ROBE_STATIC_SCRATCH_BYTES, st) != cudaSuccess)
+        return ROBE_ERR_CUDA;
+    return ROBE_OK;
+}
+
+int robe_backward_adam(robe_handle_t h, const float* grad_out, const void* indices,
+                       const int64_t* offsets, int64_t batch, int64_t nnz, float* m1, float* m2,
+                       float lr, float beta1, float beta2, float eps, int64_t step, void* workspace,
+                       size_t workspace_bytes, void* stream) {
+    if (!check_sizes(h, indices, offsets, batch, nnz)) return ROBE_ERR_INVALID_ARG;
+    if (batch > 0 && grad_out == nullptr) return ROBE_ERR_INVALID_ARG;
+    if (m1 == nullptr || m2 == nullptr || step < 1) return ROBE_ERR_INVALID_ARG;
+    if (!(beta1 >= 0.0f && beta1 < 1.0f && beta2 >= 0.0f && beta2 < 1.0f && eps >= 0.0f))
+        return ROBE_ERR_INVALID_ARG;
+    if (h->validate && h->status_word == nullptr) return ROBE_ERR_INVALID_ARG;
+    if (h->array == nullptr) return ROBE_ERR_NO_ARRAY;
+    if (h->dtype != ROBE_F32) return ROBE_ERR_INVALID_ARG;
+    const Problem pb = make_problem(h, indices, offsets, batch, nnz);
+    const uint64_t nb = (uint64_t)nnz * h->mp.C;
+    uint32_t zp = 1;
+    while (zp < h->mp.Z) zp <<= 1;
+    if (nb >= (1ull << 32) || (uint64_t)pb.nbags >= (1ull << 32)) return ROBE_ERR_UNSUPPORTED;
+    if (nb * zp / 256 >= (1ull << 31)) return ROBE_ERR_UNSUPPORTED;
+    if ((uint64_t)pb.nbags * h->mp.d > (1ull << 32)) return ROBE_ERR_UNSUPPORTED;
+    const size_t need = det_workspace_bytes(h->mp, pb.nbags, nnz, offsets != nullptr);
+    if (nnz > 0 && (workspace == nullptr || workspace_bytes < need)) return ROBE_ERR_WORKSPACE;
+    if (((uintptr_t)workspace & 255u) != 0) return ROBE_ERR_WORKSPACE;
+    AdamState ad;
+    ad.m1 = m1;
+    ad.m2 = m2;
+    ad.beta1 = beta1;
+    ad.beta2 = beta2;
+    ad.eps = eps;
+    ad.bias1 = (float)(1.0 - pow((double)beta1, (double)step));
+    ad.bias2 = (float)(1.0 - pow((double)beta2, (double)step));
+    cudaStream_t st = (cudaStream_t)stream;
+    if (launch_validate(pb, st) != cudaSuccess) return ROBE_ERR_CUDA;
+    if (launch_backward_det(pb, grad_out, (float*)h->array, 2, lr, &ad, workspace, workspace_bytes,
+                            st) != cudaSuccess)
         return ROBE_ERR_CUDA;
     return ROBE_OK;
 }

@@ -267,6 +267,7 @@ struct ApplyArgs {
     float lr;
     uint64_t nb;
     const int32_t* status;
+    AdamState adam;          // update mode 2 only
     uint32_t* long_count;    // number of handed-over rounds (may run past long_cap)
     LongWalk* long_walks;
     uint32_t long_cap;
@@ -298,10 +299,26 @@ __device__ __forceinline__ bool block_term(const ApplyArgs& a, const uint32_t* b
     return true;
 }
 
-template <bool SGD>
-__device__ __forceinline__ void commit_slot(float* target, uint32_t j, float acc, float lr) {
-    if (SGD) target[j] = __fmaf_rn(-lr, acc, target[j]);
-    else target[j] = __fadd_rn(target[j], acc);
+// What a served slot does with its sum delta (MODE): 0 - add it to a dense gradient; 1 - the
+// SGD step M[j] = fma(-lr, delta, M[j]); 2 - the Adam step (Kingma & Ba, Algorithm 1; the paper
+// trains five of its six models with Adam, Section 5) on the slot and its two moment slots, every
+// operation a separate correctly rounded fp32 one.  `old` is target[j].
+template <int MODE>
+__device__ __forceinline__ void commit_slot(const ApplyArgs& a, uint32_t j, float delta, float old) {
+    if (MODE == 0) {
+        a.target[j] = __fadd_rn(old, delta);
+    } else if (MODE == 1) {
+        a.target[j] = __fmaf_rn(-a.lr, delta, old);
+    } else {
+        const AdamState& ad = a.adam;
+        const float m = __fadd_rn(__fmul_rn(ad.beta1, ad.m1[j]), __fmul_rn(__fsub_rn(1.0f, ad.beta1), delta));
+        const float v = __fadd_rn(__fmul_rn(ad.beta2, ad.m2[j]),
+                                  __fmul_rn(__fsub_rn(1.0f, ad.beta2), __fmul_rn(delta, delta)));
+        ad.m1[j] = m;
+        ad.m2[j] = v;
+        const float den = __fadd_rn(__fsqrt_rn(__fdiv_rn(v, ad.bias2)), ad.eps);
+        a.target[j] = __fsub_rn(old, __fmul_rn(a.lr, __fdiv_rn(__fdiv_rn(m, ad.bias1), den)));
+    }
 }
 
 // Slots j in [Z-1, m).  The sorted blocks that reach slot j are those with key in [j-Z+1, j];
@@ -458,7 +475,7 @@ __device__ __forceinline__ bool walk_deep(const ApplyArgs& a, ApplyTile& tl, App
     }
 }
 
-template <bool SIGN, bool SGD, bool SHORT>
+template <bool SIGN, int MODE, bool SHORT>
 __global__ void __launch_bounds__(256)
 det_apply_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint32_t* __restrict__ V,
                  const uint32_t* __restrict__ bag_of) {
@@ -572,7 +589,7 @@ det_apply_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint32_t* __
                 walk_steps<SIGN, SHORT, UN>(a, bag_of, tl, wk, j, e, 32u, lane, 0);
             }
         }
-        if (wk.touched) a.target[j] = SGD ? __fmaf_rn(-a.lr, wk.acc, old) : __fadd_rn(old, wk.acc);
+        if (wk.touched) commit_slot<MODE>(a, j, wk.acc, old);
     }
 }
 
@@ -585,7 +602,7 @@ det_apply_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint32_t* __
 constexpr int kLongStep = 64;
 constexpr uint32_t kLongRing = 256;
 
-template <bool SGD>
+template <int MODE>
 __global__ void __launch_bounds__(64)
 det_apply_long_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint32_t* __restrict__ V) {
     __shared__ float terms_s[2][2][kLongStep][32];
@@ -665,8 +682,7 @@ det_apply_long_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint32_
         }
         asm volatile("cp.async.wait_group 0;" ::: "memory");
         if (mine && touched) {
-            const float old = a.target[j];
-            a.target[j] = SGD ? __fmaf_rn(-a.lr, acc, old) : __fadd_rn(old, acc);
+            commit_slot<MODE>(a, j, acc, a.target[j]);
         }
         __syncwarp();  // the buffers and the ring are reused by the warp's next round
     }
@@ -674,7 +690,7 @@ det_apply_long_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint32_
 
 // Slots j in [0, Z-1): plain blocks with key <= j first, then the wrapped tails of blocks
 // whose key lies in [m + j - (Z-1), m-1] (o = j + m - key).
-template <bool SIGN, bool SGD, bool SHORT>
+template <bool SIGN, int MODE, bool SHORT>
 __global__ void __launch_bounds__(128)
 det_apply_low_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint32_t* __restrict__ V,
                      const uint32_t* __restrict__ bag_of) {
@@ -699,7 +715,7 @@ det_apply_low_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint32_t
                 acc = __fadd_rn(acc, term);
                 touched = true;
             }
-        if (touched) commit_slot<SGD>(a.target, j, acc, a.lr);
+        if (touched) commit_slot<MODE>(a, j, acc, a.target[j]);
     }
 }
 
@@ -735,22 +751,22 @@ Layout make_layout(uint64_t nb, int64_t nnz, bool bags) {
     return L;
 }
 
-template <bool SIGN, bool SGD>
+template <bool SIGN, int MODE>
 void launch_apply(const ApplyArgs& aa, const uint32_t* K, const uint32_t* V, const uint32_t* bag_of,
                   cudaStream_t st) {
     const MapParams& mp = aa.mp;
     const unsigned blocks = (unsigned)((aa.nb + 255) / 256);  // one warp per 32 sorted positions
     if (mp.d % mp.Z != 0) {
-        det_apply_kernel<SIGN, SGD, true><<<blocks, 256, 0, st>>>(aa, K, V, bag_of);
-        if (mp.Z > 1) det_apply_low_kernel<SIGN, SGD, true><<<1, 128, 0, st>>>(aa, K, V, bag_of);
+        det_apply_kernel<SIGN, MODE, true><<<blocks, 256, 0, st>>>(aa, K, V, bag_of);
+        if (mp.Z > 1) det_apply_low_kernel<SIGN, MODE, true><<<1, 128, 0, st>>>(aa, K, V, bag_of);
     } else {
-        det_apply_kernel<SIGN, SGD, false><<<blocks, 256, 0, st>>>(aa, K, V, bag_of);
+        det_apply_kernel<SIGN, MODE, false><<<blocks, 256, 0, st>>>(aa, K, V, bag_of);
         if (!SIGN) {
             // the rounds the apply kernel handed over; a grid-stride loop over the list
             const unsigned lblocks = aa.long_cap / 2 < 148u * 8u ? (aa.long_cap + 1) / 2 : 148u * 8u;
-            det_apply_long_kernel<SGD><<<lblocks, 64, 0, st>>>(aa, K, V);
+            det_apply_long_kernel<MODE><<<lblocks, 64, 0, st>>>(aa, K, V);
         }
-        if (mp.Z > 1) det_apply_low_kernel<SIGN, SGD, false><<<1, 128, 0, st>>>(aa, K, V, bag_of);
+        if (mp.Z > 1) det_apply_low_kernel<SIGN, MODE, false><<<1, 128, 0, st>>>(aa, K, V, bag_of);
     }
 }
 
@@ -762,9 +778,9 @@ size_t det_workspace_bytes(const MapParams& mp, int64_t nbags, int64_t nnz, bool
     return make_layout(nb, nnz, bags).total;
 }
 
-cudaError_t launch_backward_det(const Problem& pb, const float* grad_out, float* target, int sgd,
-                                float lr, void* workspace, size_t workspace_bytes,
-                                cudaStream_t st) {
+cudaError_t launch_backward_det(const Problem& pb, const float* grad_out, float* target, int mode,
+                                float lr, const AdamState* adam, void* workspace,
+                                size_t workspace_bytes, cudaStream_t st) {
     if (pb.nnz == 0 || pb.nbags == 0) return cudaSuccess;
     const MapParams& mp = pb.mp;
     const bool bags = pb.offsets != nullptr;
@@ -811,14 +827,16 @@ cudaError_t launch_backward_det(const Problem& pb, const float* grad_out, float*
 
     uint32_t* long_count = (uint32_t*)(ws + L.long_count);
     cudaMemsetAsync(long_count, 0, sizeof(uint32_t), st);
-    ApplyArgs aa{mp, grad_out, pb.indices, target, lr, nb, pb.status,
+    ApplyArgs aa{mp, grad_out, pb.indices, target, lr, nb, pb.status, adam ? *adam : AdamState{},
                  long_count, (LongWalk*)(ws + L.long_walks), L.long_cap};
     if (pb.sign) {
-        if (sgd) launch_apply<true, true>(aa, kA, vA, bag_of, st);
-        else launch_apply<true, false>(aa, kA, vA, bag_of, st);
+        if (mode == 2) launch_apply<true, 2>(aa, kA, vA, bag_of, st);
+        else if (mode == 1) launch_apply<true, 1>(aa, kA, vA, bag_of, st);
+        else launch_apply<true, 0>(aa, kA, vA, bag_of, st);
     } else {
-        if (sgd) launch_apply<false, true>(aa, kA, vA, bag_of, st);
-        else launch_apply<false, false>(aa, kA, vA, bag_of, st);
+        if (mode == 2) launch_apply<false, 2>(aa, kA, vA, bag_of, st);
+        else if (mode == 1) launch_apply<false, 1>(aa, kA, vA, bag_of, st);
+        else launch_apply<false, 0>(aa, kA, vA, bag_of, st);
     }
     return cudaGetLastError();
 }

@@ -29,9 +29,20 @@ cudaError_t launch_backward_atomic(const Problem& pb, const float* grad_out, flo
 
 // deterministic backward
 size_t det_workspace_bytes(const MapParams& mp, int64_t nbags, int64_t nnz, bool bags);
-// sgd != 0: target = attached array, target[j] = fma(-lr, delta, target[j]); else target[j] += delta
-cudaError_t launch_backward_det(const Problem& pb, const float* grad_out, float* target, int sgd,
-                                float lr, void* workspace, size_t workspace_bytes, cudaStream_t st);
+// Adam moments and constants of the deterministic backward's update mode 2
+struct AdamState {
+    float* m1;     // device [M], first moment
+    float* m2;     // device [M], second moment
+    float beta1, beta2, eps;
+    float bias1;   // 1 - beta1^t
+    float bias2;   // 1 - beta2^t
+};
+
+// mode 0: target[j] += delta; 1: target = attached array, target[j] = fma(-lr, delta, target[j]);
+// 2: Adam step on the attached array with the moments in *adam
+cudaError_t launch_backward_det(const Problem& pb, const float* grad_out, float* target, int mode,
+                                float lr, const AdamState* adam, void* workspace,
+                                size_t workspace_bytes, cudaStream_t st);
 
 // id / offset range check into the status word
 cudaError_t launch_validate(const Problem& pb, cudaStream_t st);

@@ -239,6 +239,35 @@ def test_cfg1_backward_dense_and_sgd(mode):
                 assert_bits_equal(after[l1 == 0], before[l1 == 0], "untouched slots")
 
 
+@pytest.mark.parametrize("bags", [None, (3, 0, 9)])
+def test_backward_adam_matches_oracle_over_steps(bags):
+    # three Adam steps in a row (array and moments carried over), bit for bit
+    lr, b1, b2, eps = 0.05, 0.9, 0.999, 1e-8
+    for w in (synth.workload(1).with_(bag_rule=bags), small(d=64, Z=16, M=70, bag_rule=bags, batch=200),
+              small(d=16, Z=64, M=1000, bag_rule=bags, batch=97, vocab_arg=(3, 7, 1000))):
+        with Case(w) as c:
+            robe.robe_set_option(c.h, robe.ROBE_OPT_BWD_MODE, robe.ROBE_BWD_DETERMINISTIC)
+            ws = torch.empty(robe.robe_backward_workspace_bytes(c.h, c.B, c.indices.numel()),
+                             dtype=torch.uint8, device=c.dev)
+            m1_d = torch.zeros(w.M, device=c.dev)
+            m2_d = torch.zeros(w.M, device=c.dev)
+            arr, m1, m2 = c.array_h.copy(), np.zeros(w.M, np.float32), np.zeros(w.M, np.float32)
+            for step in (1, 2, 3):
+                g_h, g_d = _grad(c, 10 + step)
+                can, touched = c.oracle.backward_canonical(g_h, c.indices_h, c.offsets_h, c.B)
+                orc.adam_apply(arr, m1, m2, can, touched, lr, b1, b2, eps, step)
+                robe.robe_backward_adam(c.h, g_d, c.indices, c.offsets, c.B, m1_d, m2_d, lr, b1, b2, eps,
+                                        step, ws)
+                torch.cuda.synchronize()
+                assert_bits_equal(c.array.cpu().numpy(), arr, f"adam array, step {step}")
+                assert_bits_equal(m1_d.cpu().numpy(), m1, f"adam first moment, step {step}")
+                assert_bits_equal(m2_d.cpu().numpy(), m2, f"adam second moment, step {step}")
+            with pytest.raises(robe.RobeError):
+                robe.robe_backward_adam(c.h, g_d, c.indices, c.offsets, c.B, m1_d, m2_d, lr, 1.0, b2, eps, 1, ws)
+            with pytest.raises(robe.RobeError):
+                robe.robe_backward_adam(c.h, g_d, c.indices, c.offsets, c.B, m1_d, m2_d, lr, b1, b2, eps, 0, ws)
+
+
 def test_deterministic_is_bit_reproducible_and_order_sensitive_case():
     # a hot id: thousands of terms on the same slots; five runs must give identical bits
     w = small(d=32, Z=8, M=300, batch=2000, vocab_arg=(2, 3, 1000))
