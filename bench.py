@@ -274,9 +274,12 @@ def run_ours(args, w):
         robe.robe_set_option(h, robe.ROBE_OPT_BWD_MODE, robe.ROBE_BWD_DETERMINISTIC)
         ws = torch.empty(robe.robe_backward_workspace_bytes(h, B, max(len(b[0]) for b in batches)),
                          dtype=torch.uint8, device=dev)
-        # keys (+ bag numbers), three kernels per 8-bit sort pass, apply (+ the low-slot kernel)
+        # keys (+ bag numbers), three kernels per 8-bit sort pass, apply, long walks (when no
+        # block is short), low slots (when blocks are longer than one element)
         npass = -(-max(1, (w.M - 1).bit_length()) // 8)
-        bwd_launches = (1 if bags else 0) + 1 + 3 * npass + 1 + (1 if w.Z > 1 else 0)
+        zb = min(w.Z, w.d)
+        bwd_launches = ((1 if bags else 0) + 1 + 3 * npass + 1 + (1 if w.d % zb == 0 else 0)
+                        + (1 if zb > 1 else 0))
 
     def step(i, events=None):
         k = i % NB
