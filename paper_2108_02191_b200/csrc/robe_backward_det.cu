@@ -593,98 +593,114 @@ det_apply_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint32_t* __
     }
 }
 
-// Long walks (plain blocks only).  One warp per handed-over round, in steps of kLongStep
-// positions.  The keys come from a warp-private ring of 256 positions; every lane copies the
-// gradient terms of its slot with cp.async into its own column of a shared-memory buffer, so a
-// whole step is in flight at once without a register per term.  Two buffers: the copies of step
-// n+1 are issued before the terms of step n are added (in sorted order), and the keys two
-// steps ahead are fetched meanwhile.
+// Long walks (plain blocks only).  One CTA of four warps per handed-over round, in steps of
+// kLongStep positions.  Lane l of EVERY warp stands for slot l of the round.  The keys come from
+// a ring of 256 positions in shared memory.  Copying a step's gradient terms into shared memory
+// is split over the four warps (each takes a quarter of the positions; a lane copies the term
+// of its slot with cp.async into its own column, so a whole step is in flight without a
+// register per term); warp 0 then adds the terms of each slot in sorted order.  Two buffers:
+// the copies of step n+1 are issued before the adds of step n.  Sorted keys make "this
+// position still reaches slot j" a prefix property, so the copiers need no state and the adder
+// finds the length of the prefix by bisection.
 constexpr int kLongStep = 64;
+constexpr int kLongWarps = 4;
 constexpr uint32_t kLongRing = 256;
 
 template <int MODE>
-__global__ void __launch_bounds__(64)
+__global__ void __launch_bounds__(32 * kLongWarps)
 det_apply_long_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint32_t* __restrict__ V) {
-    __shared__ float terms_s[2][2][kLongStep][32];
-    __shared__ uint2 ring_s[2][kLongRing];
+    __shared__ float terms_s[2][kLongStep][32];
+    __shared__ uint2 ring[kLongRing];
+    __shared__ uint32_t go_on;
     if (a.status != nullptr && *a.status != 0) return;
-    const uint32_t lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const uint32_t tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
     const uint32_t n_rec = *a.long_count < a.long_cap ? *a.long_count : a.long_cap;
-    uint2* ring = ring_s[w];
-    const uint32_t dst0 = (uint32_t)__cvta_generic_to_shared(&terms_s[w][0][0][lane]);
+    const uint32_t dst0 = (uint32_t)__cvta_generic_to_shared(&terms_s[0][0][lane]);
     constexpr uint32_t kBufBytes = kLongStep * 32 * sizeof(float);
-    for (uint32_t rec = blockIdx.x * 2 + w; rec < n_rec; rec += gridDim.x * 2) {
+    constexpr int kPerWarp = kLongStep / kLongWarps;
+    for (uint32_t rec = blockIdx.x; rec < n_rec; rec += gridDim.x) {
         const LongWalk* lw = a.long_walks + rec;
         const uint64_t i0 = lw->i0;
         const uint32_t j = lw->j[lane];
-        float acc = lw->acc[lane];
         const uint32_t st = lw->state[lane];
         const uint32_t e = st & 0xFFu;
         const bool mine = (st >> 8) & 1u;  // this lane's walk was handed over
-        bool going = mine, touched = (st >> 9) & 1u;
+        float acc = lw->acc[lane];         // used by warp 0 only
+        bool touched = (st >> 9) & 1u;
         auto fetch = [&](uint32_t r) -> uint2 {
             const uint64_t idx = i0 + r;
             if (idx >= a.nb) return make_uint2(kNoKey, 0u);
             return make_uint2(__ldg(K + idx), __ldg(V + idx));
         };
-        // Issues the copies of the step that starts at tile-relative position `base` into buffer
-        // `buf`; returns how many positions of the step reach slot j (sorted keys: a prefix).
-        auto issue = [&](uint32_t base, uint32_t buf) -> uint32_t {
-            uint32_t n = 0;
+        // This warp's quarter of the copies of the step that starts at tile-relative position `base`.
+        auto issue = [&](uint32_t base, uint32_t buf) {
             const uint32_t dst = dst0 + buf * kBufBytes;
-#pragma unroll 8
-            for (int t = 0; t < kLongStep; ++t) {
+#pragma unroll
+            for (int q = 0; q < kPerWarp; ++q) {
+                const uint32_t t = w * kPerWarp + q;
                 const uint2 kv = ring[(base + e + t) & (kLongRing - 1)];
-                if (going && kv.x <= j) {
+                if (mine && kv.x <= j) {
                     const float* src = a.grad_out + (kv.y + (j - kv.x));
-                    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst + (uint32_t)t * 128u),
-                                 "l"(src));
-                    ++n;
+                    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst + t * 128u), "l"(src));
                 }
             }
             asm volatile("cp.async.commit_group;");
-            going = going && n == (uint32_t)kLongStep;
-            return n;
+        };
+        // How many positions of that step reach slot j: first t with key > j, by bisection.
+        auto reach = [&](uint32_t base) -> uint32_t {
+            if (!mine) return 0u;
+            uint32_t lo = 0, hi = kLongStep;
+            while (lo < hi) {
+                const uint32_t mid = (lo + hi) >> 1;
+                if (ring[(base + e + mid) & (kLongRing - 1)].x <= j) lo = mid + 1; else hi = mid;
+            }
+            return lo;
         };
         // a step reads positions base + e + t, e < 32, t < kLongStep: [base, base + 96)
         uint32_t base = lw->fbase;
         uint32_t ring_end = base + 160;
-        __syncwarp();
-#pragma unroll
-        for (int q = 0; q < 5; ++q) ring[(base + 32 * q + lane) & (kLongRing - 1)] = fetch(base + 32 * q + lane);
-        __syncwarp();
-        uint32_t n_cur = issue(base, 0);
+        __syncthreads();  // the previous round's readers are done with the ring and the buffers
+        ring[(base + tid) & (kLongRing - 1)] = fetch(base + tid);
+        if (tid < 32) ring[(base + 128 + tid) & (kLongRing - 1)] = fetch(base + 128 + tid);
+        __syncthreads();
+        uint32_t n_cur = w == 0 ? reach(base) : 0u;
+        issue(base, 0);
         for (uint32_t step = 0;; ++step) {
             // step+1: its keys [base + 64, base + 160) are in the ring (ring_end = base + 160)
-            const uint32_t n_nxt = issue(base + kLongStep, (step + 1) & 1u);
-            const uint2 f0 = fetch(ring_end + lane), f1 = fetch(ring_end + 32 + lane);
-            asm volatile("cp.async.wait_group 1;" ::: "memory");  // the copies of `step` are in
-            const float(*buf)[32] = terms_s[w][step & 1u];
-            const uint32_t n_max = __reduce_max_sync(0xFFFFFFFFu, n_cur);
-            for (uint32_t t0 = 0; t0 < n_max; t0 += 8) {
-                float x[8];
-#pragma unroll
-                for (int q = 0; q < 8; ++q) x[q] = buf[t0 + q][lane];
-#pragma unroll
-                for (int q = 0; q < 8; ++q)
-                    if (t0 + q < n_cur) acc = __fadd_rn(acc, x[q]);
+            issue(base + kLongStep, (step + 1) & 1u);
+            uint2 fresh = make_uint2(kNoKey, 0u);
+            if (tid < 64) fresh = fetch(ring_end + tid);
+            uint32_t n_nxt = 0;
+            if (w == 0) {
+                n_nxt = reach(base + kLongStep);
+                const bool any_next = __ballot_sync(0xFFFFFFFFu, n_nxt != 0) != 0;
+                if (lane == 0) go_on = any_next ? 1u : 0u;
             }
-            if (n_cur != 0) touched = true;
-            const bool any_next = __ballot_sync(0xFFFFFFFFu, n_nxt != 0) != 0;
-            if (!any_next) break;
-            __syncwarp();  // every lane is past its ring reads of step+1: the keys of step+2 may enter
-            ring[(ring_end + lane) & (kLongRing - 1)] = f0;
-            ring[(ring_end + 32 + lane) & (kLongRing - 1)] = f1;
+            asm volatile("cp.async.wait_group 1;" ::: "memory");  // this thread's copies of `step`
+            __syncthreads();  // everybody's copies of `step` are in; all ring reads of step+1 are done
+            if (w == 0) {
+                const float(*buf)[32] = terms_s[step & 1u];
+                const uint32_t n_max = __reduce_max_sync(0xFFFFFFFFu, n_cur);
+                for (uint32_t t0 = 0; t0 < n_max; t0 += 8) {
+                    float x[8];
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) x[q] = buf[t0 + q][lane];
+#pragma unroll
+                    for (int q = 0; q < 8; ++q)
+                        if (t0 + q < n_cur) acc = __fadd_rn(acc, x[q]);
+                }
+                if (n_cur != 0) touched = true;
+            }
+            if (tid < 64) ring[(ring_end + tid) & (kLongRing - 1)] = fresh;  // keys of step+2
+            const bool more = go_on != 0;
+            __syncthreads();  // adds of `step` done before its buffer is refilled; ring updated
+            if (!more) break;
             ring_end += 64;
-            __syncwarp();
             n_cur = n_nxt;
             base += kLongStep;
         }
         asm volatile("cp.async.wait_group 0;" ::: "memory");
-        if (mine && touched) {
-            commit_slot<MODE>(a, j, acc, a.target[j]);
-        }
-        __syncwarp();  // the buffers and the ring are reused by the warp's next round
+        if (w == 0 && mine && touched) commit_slot<MODE>(a, j, acc, a.target[j]);
     }
 }
 
@@ -763,8 +779,8 @@ void launch_apply(const ApplyArgs& aa, const uint32_t* K, const uint32_t* V, con
         det_apply_kernel<SIGN, MODE, false><<<blocks, 256, 0, st>>>(aa, K, V, bag_of);
         if (!SIGN) {
             // the rounds the apply kernel handed over; a grid-stride loop over the list
-            const unsigned lblocks = aa.long_cap / 2 < 148u * 8u ? (aa.long_cap + 1) / 2 : 148u * 8u;
-            det_apply_long_kernel<MODE><<<lblocks, 64, 0, st>>>(aa, K, V);
+            const unsigned lblocks = aa.long_cap < 148u * 8u ? aa.long_cap : 148u * 8u;
+            det_apply_long_kernel<MODE><<<lblocks, 32 * kLongWarps, 0, st>>>(aa, K, V);
         }
         if (mp.Z > 1) det_apply_low_kernel<SIGN, MODE, false><<<1, 128, 0, st>>>(aa, K, V, bag_of);
     }
