@@ -594,17 +594,17 @@ det_apply_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint32_t* __
 }
 
 // Long walks (plain blocks only).  One CTA of four warps per handed-over round, in steps of
-// kLongStep positions.  Lane l of EVERY warp stands for slot l of the round.  The keys come from
-// a ring of 256 positions in shared memory.  Copying a step's gradient terms into shared memory
+// kLongStep = 128 positions.  Lane l of EVERY warp stands for slot l of the round.  The keys come from
+// a ring of 512 positions in shared memory.  Copying a step's gradient terms into shared memory
 // is split over the four warps (each takes a quarter of the positions; a lane copies the term
 // of its slot with cp.async into its own column, so a whole step is in flight without a
 // register per term); warp 0 then adds the terms of each slot in sorted order.  Two buffers:
 // the copies of step n+1 are issued before the adds of step n.  Sorted keys make "this
 // position still reaches slot j" a prefix property, so the copiers need no state and the adder
 // finds the length of the prefix by bisection.
-constexpr int kLongStep = 64;
+constexpr int kLongStep = 128;
 constexpr int kLongWarps = 4;
-constexpr uint32_t kLongRing = 256;
+constexpr uint32_t kLongRing = 512;  // >= 2 steps + 32 positions of lane spread, power of two
 
 template <int MODE>
 __global__ void __launch_bounds__(32 * kLongWarps)
@@ -656,20 +656,22 @@ det_apply_long_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint32_
             }
             return lo;
         };
-        // a step reads positions base + e + t, e < 32, t < kLongStep: [base, base + 96)
+        // a step reads positions base + e + t, e < 32, t < kLongStep: [base, base + kLongStep + 32);
+        // the ring is kept filled one step further than that
+        constexpr uint32_t kAhead = 2 * kLongStep + 32;
         uint32_t base = lw->fbase;
-        uint32_t ring_end = base + 160;
+        uint32_t ring_end = base + kAhead;
         __syncthreads();  // the previous round's readers are done with the ring and the buffers
-        ring[(base + tid) & (kLongRing - 1)] = fetch(base + tid);
-        if (tid < 32) ring[(base + 128 + tid) & (kLongRing - 1)] = fetch(base + 128 + tid);
+        for (uint32_t r = tid; r < kAhead; r += 32 * kLongWarps)
+            ring[(base + r) & (kLongRing - 1)] = fetch(base + r);
         __syncthreads();
         uint32_t n_cur = w == 0 ? reach(base) : 0u;
         issue(base, 0);
         for (uint32_t step = 0;; ++step) {
-            // step+1: its keys [base + 64, base + 160) are in the ring (ring_end = base + 160)
+            // step+1: its keys are in the ring already (ring_end = base + 2 steps + 32)
             issue(base + kLongStep, (step + 1) & 1u);
             uint2 fresh = make_uint2(kNoKey, 0u);
-            if (tid < 64) fresh = fetch(ring_end + tid);
+            if (tid < (uint32_t)kLongStep) fresh = fetch(ring_end + tid);
             uint32_t n_nxt = 0;
             if (w == 0) {
                 n_nxt = reach(base + kLongStep);
@@ -691,11 +693,11 @@ det_apply_long_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint32_
                 }
                 if (n_cur != 0) touched = true;
             }
-            if (tid < 64) ring[(ring_end + tid) & (kLongRing - 1)] = fresh;  // keys of step+2
+            if (tid < (uint32_t)kLongStep) ring[(ring_end + tid) & (kLongRing - 1)] = fresh;  // keys of step+2
             const bool more = go_on != 0;
             __syncthreads();  // adds of `step` done before its buffer is refilled; ring updated
             if (!more) break;
-            ring_end += 64;
+            ring_end += kLongStep;
             n_cur = n_nxt;
             base += kLongStep;
         }
