@@ -39,8 +39,8 @@ UNIT = "ids/s"
 # full-size default workload that profiles/dram_traffic_cfg4_multihot.md summarises; None = not
 # captured for that workload or backward variant.
 NCU_TRAFFIC_BYTES = {
-    ("cfg4_multihot", "atomic"): {"forward": 4_155_085_568, "backward": 7_510_767_360},
-    ("cfg4_multihot", "det"): {"forward": 4_155_085_568, "backward": None},
+    ("cfg4_multihot", "atomic"): {"forward": 4_197_885_696, "backward": 7_509_030_400},
+    ("cfg4_multihot", "det"): {"forward": 4_197_885_696, "backward": None},
 }
 
 
