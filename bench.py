@@ -65,6 +65,23 @@ def algorithmic_bytes(w, nbags, nnz, bags, id_bytes=8):
     return fwd, bwd
 
 
+def forward_byte_models(w, nbags, nnz, bags, id_bytes=8):
+    """The forward's bytes per launch under the three models the results are read against:
+    useful       what the method itself must move (algorithmic_bytes);
+    sector       the same with the array counted in 32-byte sectors: a Z-element block at an
+                 arbitrary element offset covers 1 + (Z-1)/E sectors on average (E elements per
+                 sector) - the paper's Table 1 restated for sectors;
+    l2_resident  ids, offsets and output only: the floor when the array is served from L2."""
+    s_a = 4 if w.array_dtype == "f32" else 2
+    zb = min(w.Z, w.d)
+    e_per_sector = 32 // s_a
+    blocks = -(-w.d // zb)
+    rest = id_bytes * nnz + (8 * (nbags + 1) if bags else 0) + 4 * w.d * nbags
+    return {"useful": rest + w.d * s_a * nnz,
+            "sector": rest + blocks * (1 + (zb - 1) / e_per_sector) * 32 * nnz,
+            "l2_resident": rest}
+
+
 class ClockSampler:
     """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
 
@@ -422,6 +439,9 @@ def run_ours(args, w):
         "roofline": roof(dom_bytes, dom_ms, dominant),
         "roofline_forward": roof(fwd_bytes, fwd_ms, "forward"),
         "roofline_backward": roof(bwd_bytes, bwd_ms, "backward"),
+        "forward_models": {k: {"bytes": int(v), "GB/s": v / (fwd_ms * 1e-3) / 1e9,
+                               "frac": v / (fwd_ms * 1e-3) / 1e9 / peak}
+                           for k, v in forward_byte_models(w, nbags, nnz_per_step, bags, id_bytes).items()},
         "forward_only": {"value": world * nnz_per_step / (fwd_ms * 1e-3), "unit": UNIT,
                          "bags_per_s": world * nbags / (fwd_ms * 1e-3), "ms": fwd_ms},
     }
