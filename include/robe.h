@@ -53,7 +53,7 @@ typedef enum {
 
 /* option keys for robe_set_option */
 #define ROBE_OPT_SIGN 1     /* 0 (default) | 1: multiply by the sign hash g(e,x,i)        */
-#define ROBE_OPT_BWD_MODE 2 /* ROBE_BWD_ATOMIC (default) | ROBE_BWD_DETERMINISTIC         */
+#define ROBE_OPT_BWD_MODE 2 /* ROBE_BWD_ATOMIC (default) | ROBE_BWD_DETERMINISTIC | ROBE_BWD_BINNED */
 #define ROBE_OPT_VALIDATE 3 /* 0 (default) | 1: range-check ids/offsets on the device and
                                record the first violation in a status word instead of
                                using the bad value                                        */
@@ -70,6 +70,7 @@ typedef enum {
 
 #define ROBE_BWD_ATOMIC 0
 #define ROBE_BWD_DETERMINISTIC 1
+#define ROBE_BWD_BINNED 2
 
 /* values of the device status word (robe_last_device_status) */
 #define ROBE_DEV_OK 0
@@ -140,7 +141,8 @@ int robe_forward(robe_handle_t h, const void* indices, const int64_t* offsets, i
 /*
  * robe_backward_workspace_bytes - bytes of caller-provided device scratch that
  * robe_backward needs in the handle's current backward mode for a call of this
- * size (0 in atomic mode).  Returns 0 for a bad handle.
+ * size (0 in atomic mode; binned and deterministic mode need the same).  Returns 0 for a
+ * bad handle.
  */
 size_t robe_backward_workspace_bytes(robe_handle_t h, int64_t batch, int64_t nnz);
 
@@ -156,7 +158,11 @@ size_t robe_backward_workspace_bytes(robe_handle_t h, int64_t batch, int64_t nnz
  *   lr          learning rate, used only when grad_array == NULL.
  *   workspace   device pointer to workspace_bytes bytes, 256-byte aligned; may be NULL
  *               in atomic mode.
- * Atomic mode adds with red.global (fp32, order not fixed).  Deterministic mode sorts
+ * Atomic mode adds with red.global (fp32, order not fixed).  Binned mode does the same adds
+ * after grouping the blocks by array region (one radix pass on the top bits of the block
+ * start), so that the read-modify-write of an array much larger than the L2 happens in L2; it
+ * needs the workspace of the deterministic mode and gives atomic-mode accuracy, not
+ * reproducible bits.  Deterministic mode sorts
  * the blocks by start offset (stable) and lets each array slot sum its terms in that
  * order in fp32 from +0, then applies ONE add (dense) or ONE fma (SGD) per touched
  * slot: results are bit-reproducible.

@@ -37,6 +37,7 @@ ROBE_I32 = 1
 
 ROBE_BWD_ATOMIC = 0
 ROBE_BWD_DETERMINISTIC = 1
+ROBE_BWD_BINNED = 2
 
 ROBE_STATIC_SCRATCH_BYTES = 32 << 20
 

@@ -170,7 +170,7 @@ int robe_set_option(robe_handle_t h, int key, int64_t value) {
             h->sign = (int)value;
             return ROBE_OK;
         case ROBE_OPT_BWD_MODE:
-            if (value != ROBE_BWD_ATOMIC && value != ROBE_BWD_DETERMINISTIC)
+            if (value != ROBE_BWD_ATOMIC && value != ROBE_BWD_DETERMINISTIC && value != ROBE_BWD_BINNED)
                 return ROBE_ERR_INVALID_ARG;
             h->bwd_mode = (int)value;
             return ROBE_OK;
@@ -241,7 +241,7 @@ int robe_forward(robe_handle_t h, const void* indices, const int64_t* offsets, i
 
 size_t robe_backward_workspace_bytes(robe_handle_t h, int64_t batch, int64_t nnz) {
     if (h == nullptr || batch < 0 || nnz < 0) return 0;
-    if (h->bwd_mode != ROBE_BWD_DETERMINISTIC) return 0;
+    if (h->bwd_mode == ROBE_BWD_ATOMIC) return 0;
     // the pooled layout is the larger of the two; a caller may size once for both
     return det_workspace_bytes(h->mp, batch * (int64_t)h->T, nnz, true);
 }
@@ -278,7 +278,9 @@ int robe_backward(robe_handle_t h, const float* grad_out, const void* indices,
     if (nnz > 0 && (workspace == nullptr || workspace_bytes < need)) return ROBE_ERR_WORKSPACE;
     if (((uintptr_t)workspace & 255u) != 0) return ROBE_ERR_WORKSPACE;
     if (launch_validate(pb, st) != cudaSuccess) return ROBE_ERR_CUDA;
-    if (launch_backward_det(pb, grad_out, target, sgd ? 1 : 0, lr, nullptr, workspace, workspace_bytes,
+    const bool binned = h->bwd_mode == ROBE_BWD_BINNED;
+    if (launch_backward_det(pb, grad_out, target, binned ? 3 : (sgd ? 1 : 0),
+                            binned ? (sgd ? -lr : 1.0f) : lr, nullptr, workspace, workspace_bytes,
                             st) != cudaSuccess)
         return ROBE_ERR_CUDA;
     return ROBE_OK;

@@ -737,6 +737,46 @@ det_apply_low_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint32_t
     }
 }
 
+// Binned (not deterministic) backward: after ONE scatter pass on the top key bits the blocks are
+// grouped by array region (a bin covers 2^shift consecutive slots, a few MB), and this kernel
+// adds them in that order with red.global: thread (i, u) adds term u of sorted block i.  The
+// blocks in flight at any moment fall into one or two bins, so the read-modify-write of the array
+// happens in L2 and every array sector crosses the DRAM bus about once per call instead of once
+// per block that touches it.  a.lr carries the scale (1 for a dense gradient, -lr for SGD).
+constexpr int kBinnedPer = 8;  // sorted blocks per thread group, all their loads in flight together
+
+template <bool SIGN, bool SHORT>
+__global__ void __launch_bounds__(256)
+binned_apply_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint32_t* __restrict__ V,
+                    const uint32_t* __restrict__ bag_of, uint32_t log2Zp) {
+    if (a.status != nullptr && *a.status != 0) return;
+    const MapParams& mp = a.mp;
+    const uint64_t tid = (uint64_t)blockIdx.x * 256 + threadIdx.x;
+    const uint64_t i0 = (tid >> log2Zp) * kBinnedPer;
+    const uint32_t u = (uint32_t)(tid & ((1u << log2Zp) - 1u));
+    if (i0 >= a.nb || u >= mp.Z) return;
+    uint32_t k[kBinnedPer], v[kBinnedPer];
+#pragma unroll
+    for (int t = 0; t < kBinnedPer; ++t) {
+        const uint64_t i = i0 + t < a.nb ? i0 + t : a.nb - 1;
+        k[t] = __ldg(K + i);
+        v[t] = __ldg(V + i);
+    }
+    float term[kBinnedPer];
+    bool ok[kBinnedPer];
+#pragma unroll
+    for (int t = 0; t < kBinnedPer; ++t)
+        ok[t] = i0 + t < a.nb && block_term<SIGN, SHORT>(a, bag_of, v[t], u, term[t]);
+#pragma unroll
+    for (int t = 0; t < kBinnedPer; ++t) {
+        if (ok[t]) {
+            uint64_t j = (uint64_t)k[t] + u;
+            if (j >= mp.m) j -= mp.m;
+            atomicAdd(a.target + j, a.lr * term[t]);
+        }
+    }
+}
+
 uint32_t bits_for(uint32_t m) {  // bits needed for keys in [0, m)
     uint32_t b = 1;
     while (b < 32 && (1ull << b) < (uint64_t)m) ++b;
@@ -829,6 +869,29 @@ cudaError_t launch_backward_det(const Problem& pb, const float* grad_out, float*
 
     const SortPlan sp = make_plan(nb);
     const uint32_t bits = bits_for(mp.m);
+    if (mode == 3) {
+        // binned: one pass on the top 8 key bits, then atomic adds in bin order
+        const uint32_t shift = bits > 8 ? bits - 8 : 0;
+        const uint32_t mask = (1u << (bits - shift)) - 1u;
+        sort_count_kernel<<<sp.grid, kSortThreads, 0, st>>>(kA, counts, nb, sp.tiles, shift, mask);
+        sort_scan_kernel<<<kRadix, kSortThreads, 0, st>>>(counts, totals, sp.grid);
+        sort_scatter_kernel<<<sp.grid, kSortThreads, 0, st>>>(kA, vA, kB, vB, counts, totals, nb,
+                                                             sp.tiles, shift, mask);
+        ApplyArgs ab{mp, grad_out, pb.indices, target, lr, nb, pb.status, AdamState{}, nullptr, nullptr, 0};
+        uint32_t log2Zp = 0;
+        while ((1u << log2Zp) < mp.Z) ++log2Zp;
+        const uint64_t groups = (nb + kBinnedPer - 1) / kBinnedPer;
+        const unsigned blocks = (unsigned)(((groups << log2Zp) + 255) / 256);
+        const bool shortb = mp.d % mp.Z != 0;
+        if (pb.sign) {
+            if (shortb) binned_apply_kernel<true, true><<<blocks, 256, 0, st>>>(ab, kB, vB, bag_of, log2Zp);
+            else binned_apply_kernel<true, false><<<blocks, 256, 0, st>>>(ab, kB, vB, bag_of, log2Zp);
+        } else {
+            if (shortb) binned_apply_kernel<false, true><<<blocks, 256, 0, st>>>(ab, kB, vB, bag_of, log2Zp);
+            else binned_apply_kernel<false, false><<<blocks, 256, 0, st>>>(ab, kB, vB, bag_of, log2Zp);
+        }
+        return cudaGetLastError();
+    }
     const uint32_t npass = (bits + 7) / 8;
     const uint32_t bpp = (bits + npass - 1) / npass;
     for (uint32_t pass = 0; pass < npass; ++pass) {

@@ -39,7 +39,8 @@ struct AdamState {
 };
 
 // mode 0: target[j] += delta; 1: target = attached array, target[j] = fma(-lr, delta, target[j]);
-// 2: Adam step on the attached array with the moments in *adam
+// 2: Adam step on the attached array with the moments in *adam; 3: binned atomic adds of
+// lr * delta terms into target (one sort pass on the top key bits, then red.global in bin order)
 cudaError_t launch_backward_det(const Problem& pb, const float* grad_out, float* target, int mode,
                                 float lr, const AdamState* adam, void* workspace,
                                 size_t workspace_bytes, cudaStream_t st);

@@ -60,7 +60,8 @@ class Case:
                  grad_array=None):
         """Returns the dense gradient array (sgd=False) or None (sgd=True: array updated in place)."""
         robe.robe_set_option(self.h, robe.ROBE_OPT_BWD_MODE,
-                             robe.ROBE_BWD_ATOMIC if mode == "atomic" else robe.ROBE_BWD_DETERMINISTIC)
+                             {"atomic": robe.ROBE_BWD_ATOMIC, "det": robe.ROBE_BWD_DETERMINISTIC,
+                              "binned": robe.ROBE_BWD_BINNED}[mode])
         robe.robe_set_option(self.h, robe.ROBE_OPT_BWD_KERNEL, kernel)
         ws = None
         nbytes = robe.robe_backward_workspace_bytes(self.h, self.B, self.indices.numel())

@@ -193,6 +193,8 @@ def test_backward_shapes(d, Z, M, bags):
             for kernel in ([0, 1, 2] if warp_ok else [0, 1]):
                 ga = c.backward(g_d, "atomic", kernel=kernel).cpu().numpy()
                 assert_within_l1(ga, delta64, l1, what=f"atomic d={d} Z={Z} M={M} k={kernel}")
+            gb = c.backward(g_d, "binned").cpu().numpy()
+            assert_within_l1(gb, delta64, l1, what=f"binned d={d} Z={Z} M={M}")
             det = c.backward(g_d, "det").cpu().numpy()
             assert_bits_equal(det, can, f"deterministic d={d} Z={Z} M={M} sign={sign}")
             # integer gradients: every order gives the same bits, so atomic == canonical == fp64
@@ -364,6 +366,13 @@ def test_cfg4_forward_backward_full_size():
         delta64, l1 = c.oracle.backward_f64(g_h, c.indices_h, c.offsets_h, c.B)
         ga = c.backward(g_d, "atomic").cpu().numpy()
         assert_within_l1(ga, delta64, l1, what="cfg4 atomic")
+        gb = c.backward(g_d, "binned").cpu().numpy()
+        assert_within_l1(gb, delta64, l1, what="cfg4 binned")
+        before = c.array_h.copy()
+        c.backward(g_d, "binned", sgd=True, lr=0.5)
+        assert_within_l1(c.array.cpu().numpy(), before.astype(np.float64) - 0.5 * delta64,
+                         0.5 * l1 + np.abs(before), what="cfg4 binned sgd")
+        c.array.copy_(torch.from_numpy(before))
         # gradient mass is conserved (holds at any size)
         lengths = np.diff(c.offsets_h)
         mass = float((lengths * g_h.astype(np.float64).reshape(c.nbags, -1).sum(axis=1)).sum())
