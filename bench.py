@@ -284,6 +284,17 @@ def run_ours(args, w):
     lr = 1.0  # the paper trains its DLRM with plain SGD at learning rate 1.0 (Section 5)
     ws = None
     bwd_launches = 1
+    if args.backward == "auto":
+        # Binned pays when the array lives in HBM and a launch touches each array sector several
+        # times (ids per step x d >= array length); else the plain atomic variant is the faster one.
+        hbm_resident = w.M * (4 if w.array_dtype == "f32" else 2) > 2 * 126e6
+        coverage = float(np.mean([len(b[0]) for b in batches])) * w.d / w.M
+        args.backward = "binned" if (hbm_resident and coverage >= 1.0 and w.array_dtype == "f32") else "atomic"
+    if args.backward == "binned":
+        robe.robe_set_option(h, robe.ROBE_OPT_BWD_MODE, robe.ROBE_BWD_BINNED)
+        ws = torch.empty(robe.robe_backward_workspace_bytes(h, B, max(len(b[0]) for b in batches)),
+                         dtype=torch.uint8, device=dev)
+        bwd_launches = (1 if bags else 0) + 5  # (bag numbers,) keys, count, scan, scatter, apply
     # a bf16 array is read-only for the library: its gradient goes to a dense fp32 array instead
     # of the fused SGD step (the array stays as it is)
     dense = torch.zeros(w.M, dtype=torch.float32, device=dev) if w.array_dtype != "f32" else None
@@ -427,7 +438,7 @@ def run_ours(args, w):
         "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": w.name, "num_tables": T, "d": d, "Z": w.Z, "M": w.M, "batch_per_gpu": B,
-                   "ids_per_step_per_gpu": nnz_per_step, "ids": args.ids, "bags": bags, "backward": ("atomic" if args.backward == "atomic" else "deterministic") +
+                   "ids_per_step_per_gpu": nnz_per_step, "ids": args.ids, "bags": bags, "backward": {"atomic": "atomic", "det": "deterministic", "binned": "binned atomic"}[args.backward] +
                    (", SGD fused" if dense is None else ", dense fp32 gradient"),
                    "l2": l2_note,
                    "parallelism": f"dp{world} replicas, no collective"},
@@ -464,8 +475,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg4", help=WORKLOAD_HELP)
-    ap.add_argument("--backward", default="atomic", choices=["atomic", "det"],
-                    help="backward variant of the step (default: atomic red.global adds)")
+    ap.add_argument("--backward", default="auto", choices=["auto", "atomic", "binned", "det"],
+                    help="backward variant of the step; auto = binned atomic adds when the array lives in "
+                         "HBM and is touched several times per step, else plain atomic adds")
     ap.add_argument("--ids", default="int64", choices=["int64", "int32"], help="element type of the id arrays")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=0,

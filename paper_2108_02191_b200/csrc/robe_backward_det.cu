@@ -76,9 +76,36 @@ __global__ void __launch_bounds__(256) det_bag_of_kernel(KeyArgs a, uint32_t* ba
 
 // key[q] = h(e, x_p, c) for q = p*C + c.  val[q] = q when the sign hash is on (the apply kernel
 // then needs the id again), else the position bag*d + c*Z of the block's first gradient element.
+// One thread per id: the part of the hash that all chunks of the id share is evaluated once.
 template <bool SIGN>
 __global__ void __launch_bounds__(256)
 det_keys_kernel(KeyArgs a, const uint32_t* bag_of, uint32_t* keys, uint32_t* vals, uint64_t nb) {
+    const uint64_t p = (uint64_t)blockIdx.x * 256 + threadIdx.x;
+    if (p >= (uint64_t)a.nnz) return;
+    const MapParams& mp = a.mp;
+    const uint64_t bag = bag_of ? (uint64_t)bag_of[p] : p;
+    const uint32_t e = table_of_bag(bag, mp);
+    const uint64_t x = (uint64_t)a.indices.load((int64_t)p);
+    const uint64_t q0 = p * mp.C;
+    if (mp.R > 1) {  // rows clubbed into one block: a single key
+        keys[q0] = id_block_start(mp, e, x, 0);
+        vals[q0] = SIGN ? (uint32_t)q0 : (uint32_t)(bag * mp.d);
+        return;
+    }
+    const uint64_t base = hash_base(mp.h, e, x);
+    for (uint32_t c = 0; c < mp.C; ++c) {
+        keys[q0 + c] = block_start(mp, base, c);
+        vals[q0 + c] = SIGN ? (uint32_t)(q0 + c) : (uint32_t)(bag * mp.d + c * mp.Z);
+    }
+    (void)nb;
+}
+
+// The same, one thread per block: for many blocks per id (small Z) the writes of one thread per
+// id would be far apart, and re-evaluating the shared part of the hash per block costs less.
+template <bool SIGN>
+__global__ void __launch_bounds__(256)
+det_keys_by_block_kernel(KeyArgs a, const uint32_t* bag_of, uint32_t* keys, uint32_t* vals,
+                         uint64_t nb) {
     const uint64_t q = (uint64_t)blockIdx.x * 256 + threadIdx.x;
     if (q >= nb) return;
     const MapParams& mp = a.mp;
@@ -862,10 +889,15 @@ cudaError_t launch_backward_det(const Problem& pb, const float* grad_out, float*
         cudaMemsetAsync(bag_of, 0, (size_t)pb.nnz * sizeof(uint32_t), st);
         det_bag_of_kernel<<<(unsigned)((pb.nbags + 7) / 8), 256, 0, st>>>(ka, bag_of);
     }
-    if (pb.sign)
-        det_keys_kernel<true><<<(unsigned)((nb + 255) / 256), 256, 0, st>>>(ka, bag_of, kA, vA, nb);
-    else
-        det_keys_kernel<false><<<(unsigned)((nb + 255) / 256), 256, 0, st>>>(ka, bag_of, kA, vA, nb);
+    if (mp.C <= 8) {
+        const unsigned kb = (unsigned)((pb.nnz + 255) / 256);
+        if (pb.sign) det_keys_kernel<true><<<kb, 256, 0, st>>>(ka, bag_of, kA, vA, nb);
+        else det_keys_kernel<false><<<kb, 256, 0, st>>>(ka, bag_of, kA, vA, nb);
+    } else {
+        const unsigned kb = (unsigned)((nb + 255) / 256);
+        if (pb.sign) det_keys_by_block_kernel<true><<<kb, 256, 0, st>>>(ka, bag_of, kA, vA, nb);
+        else det_keys_by_block_kernel<false><<<kb, 256, 0, st>>>(ka, bag_of, kA, vA, nb);
+    }
 
     const SortPlan sp = make_plan(nb);
     const uint32_t bits = bits_for(mp.m);
