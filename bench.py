@@ -41,6 +41,8 @@ UNIT = "ids/s"
 NCU_TRAFFIC_BYTES = {
     ("cfg4_multihot", "atomic"): {"forward": 4_197_885_696, "backward": 7_509_030_400},
     ("cfg4_multihot", "det"): {"forward": 4_197_885_696, "backward": None},
+    # binned: the six kernels of the backward together (profiles/launches_cfg4_multihot.md)
+    ("cfg4_multihot", "binned"): {"forward": 4_197_885_696, "backward": 5204871680},
 }
 
 
@@ -416,6 +418,9 @@ def run_ours(args, w):
     peak, peak_kind = measured_peaks()
     fwd_bytes, bwd_bytes = algorithmic_bytes(w, nbags, nnz_per_step, bags, id_bytes)
     dominant = "backward" if bwd_ms >= fwd_ms else "forward"
+    bwd_label = {"atomic": "backward (bwd_atomic_staged_kernel)",
+                 "binned": "backward (keys, count, scan, scatter, binned_apply kernels together)",
+                 "det": "backward (keys, sort passes, apply kernels together)"}[args.backward]
     dom_bytes, dom_ms = (bwd_bytes, bwd_ms) if dominant == "backward" else (fwd_bytes, fwd_ms)
     traffic = NCU_TRAFFIC_BYTES.get((w.name, args.backward), {}) if args.ids == "int64" else {}
 
@@ -450,6 +455,7 @@ def run_ours(args, w):
         "roofline": roof(dom_bytes, dom_ms, dominant),
         "roofline_forward": roof(fwd_bytes, fwd_ms, "forward"),
         "roofline_backward": roof(bwd_bytes, bwd_ms, "backward"),
+        "kernels": {"forward": "fwd_staged_kernel", "backward": bwd_label},
         "forward_models": {k: {"bytes": int(v), "GB/s": v / (fwd_ms * 1e-3) / 1e9,
                                "frac": v / (fwd_ms * 1e-3) / 1e9 / peak}
                            for k, v in forward_byte_models(w, nbags, nnz_per_step, bags, id_bytes).items()},
