@@ -179,10 +179,12 @@ sort_scan_kernel(uint32_t* counts, uint32_t* totals, uint32_t grid) {
     if (threadIdx.x == 0) totals[blockIdx.x] = carry;
 }
 
-// ---- kernel 3: stable ranked scatter.  Per tile of 4096 pairs: every warp ranks its 512 pairs
+// ---- kernel 3: ranked scatter (STABLE: keeps the input order inside a digit - the LSD sort needs
+// that; the binned backward does not and takes ranks from shared-memory counters).  Per tile of 4096 pairs: every warp ranks its 512 pairs
 // by digit (16 rounds of ballots, earlier rounds and lower lanes first), the ranks are
 // extended over the warps, the pairs are laid out in shared memory in (digit, original order),
 // and then written out so that each digit's pairs go to consecutive addresses.
+template <bool STABLE>
 __global__ void __launch_bounds__(kSortThreads, 3)
 sort_scatter_kernel(const uint32_t* __restrict__ kin, const uint32_t* __restrict__ vin,
                     uint32_t* __restrict__ kout, uint32_t* __restrict__ vout,
@@ -215,8 +217,16 @@ sort_scatter_kernel(const uint32_t* __restrict__ kin, const uint32_t* __restrict
             const uint64_t idx = wbegin + r * 32 + lane;
             key[r] = idx < nb ? kin[idx] : 0u;
         }
+        if (!STABLE) {
+            // any order inside a digit will do: the rank is what a shared-memory counter hands out
 #pragma unroll
-        for (int r = 0; r < kSortItems; ++r) {
+            for (int r = 0; r < kSortItems; ++r) {
+                rank[r] = 0;
+                if (wbegin + r * 32 + lane < nb) rank[r] = atomicAdd(&wcnt[w][(key[r] >> shift) & mask], 1u);
+            }
+        }
+#pragma unroll
+        for (int r = 0; STABLE && r < kSortItems; ++r) {
             const bool valid = wbegin + r * 32 + lane < nb;
             const uint32_t dg = valid ? ((key[r] >> shift) & mask) : 0u;
             // lanes holding the same digit: one ballot per digit bit (a fixed cost, where
@@ -907,8 +917,8 @@ cudaError_t launch_backward_det(const Problem& pb, const float* grad_out, float*
         const uint32_t mask = (1u << (bits - shift)) - 1u;
         sort_count_kernel<<<sp.grid, kSortThreads, 0, st>>>(kA, counts, nb, sp.tiles, shift, mask);
         sort_scan_kernel<<<kRadix, kSortThreads, 0, st>>>(counts, totals, sp.grid);
-        sort_scatter_kernel<<<sp.grid, kSortThreads, 0, st>>>(kA, vA, kB, vB, counts, totals, nb,
-                                                             sp.tiles, shift, mask);
+        sort_scatter_kernel<false><<<sp.grid, kSortThreads, 0, st>>>(kA, vA, kB, vB, counts, totals, nb,
+                                                                    sp.tiles, shift, mask);
         ApplyArgs ab{mp, grad_out, pb.indices, target, lr, nb, pb.status, AdamState{}, nullptr, nullptr, 0};
         uint32_t log2Zp = 0;
         while ((1u << log2Zp) < mp.Z) ++log2Zp;
@@ -932,7 +942,7 @@ cudaError_t launch_backward_det(const Problem& pb, const float* grad_out, float*
         const uint32_t mask = (1u << width) - 1u;
         sort_count_kernel<<<sp.grid, kSortThreads, 0, st>>>(kA, counts, nb, sp.tiles, shift, mask);
         sort_scan_kernel<<<kRadix, kSortThreads, 0, st>>>(counts, totals, sp.grid);
-        sort_scatter_kernel<<<sp.grid, kSortThreads, 0, st>>>(kA, vA, kB, vB, counts, totals, nb,
+        sort_scatter_kernel<true><<<sp.grid, kSortThreads, 0, st>>>(kA, vA, kB, vB, counts, totals, nb,
                                                              sp.tiles, shift, mask);
         uint32_t* t = kA; kA = kB; kB = t;
         t = vA; vA = vB; vB = t;
