@@ -185,7 +185,7 @@ sort_scan_kernel(uint32_t* counts, uint32_t* totals, uint32_t grid) {
 // extended over the warps, the pairs are laid out in shared memory in (digit, original order),
 // and then written out so that each digit's pairs go to consecutive addresses.
 template <bool STABLE>
-__global__ void __launch_bounds__(kSortThreads, 3)
+__global__ void __launch_bounds__(kSortThreads, 4)
 sort_scatter_kernel(const uint32_t* __restrict__ kin, const uint32_t* __restrict__ vin,
                     uint32_t* __restrict__ kout, uint32_t* __restrict__ vout,
                     const uint32_t* __restrict__ cta_offsets, const uint32_t* __restrict__ totals,
