@@ -296,8 +296,7 @@ def run_ours(args, w):
         robe.robe_set_option(h, robe.ROBE_OPT_BWD_MODE, robe.ROBE_BWD_BINNED)
         ws = torch.empty(robe.robe_backward_workspace_bytes(h, B, max(len(b[0]) for b in batches)),
                          dtype=torch.uint8, device=dev)
-        # (bag numbers: only with more than 8 blocks per id,) keys, count, scan, scatter, apply
-        bwd_launches = (1 if bags and -(-w.d // min(w.Z, w.d)) > 8 else 0) + 5
+        bwd_launches = (1 if bags else 0) + 5  # (bag numbers,) keys, count, scan, scatter, apply
     # a bf16 array is read-only for the library: its gradient goes to a dense fp32 array instead
     # of the fused SGD step (the array stays as it is)
     dense = torch.zeros(w.M, dtype=torch.float32, device=dev) if w.array_dtype != "f32" else None
@@ -309,7 +308,7 @@ def run_ours(args, w):
         # block is short), low slots (when blocks are longer than one element)
         npass = -(-max(1, (w.M - 1).bit_length()) // 8)
         zb = min(w.Z, w.d)
-        bwd_launches = ((1 if bags and -(-w.d // zb) > 8 else 0) + 1 + 3 * npass + 1 + (1 if w.d % zb == 0 else 0)
+        bwd_launches = ((1 if bags else 0) + 1 + 3 * npass + 1 + (1 if w.d % zb == 0 else 0)
                         + (1 if zb > 1 else 0))
 
     def step(i, events=None):

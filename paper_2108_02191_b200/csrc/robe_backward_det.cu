@@ -100,39 +100,6 @@ det_keys_kernel(KeyArgs a, const uint32_t* bag_of, uint32_t* keys, uint32_t* val
     (void)nb;
 }
 
-// The same for pooled input with the sign hash off, one warp per bag and one lane per id: the bag
-// number is known without the bag_of table.  Ids that malformed offsets leave outside every bag
-// (only possible before the first and after the last bag once the offsets are clamped to be
-// monotone) are given to the first / last bag, so that every key is written.
-__global__ void __launch_bounds__(256)
-det_keys_by_bag_kernel(KeyArgs a, uint32_t* keys, uint32_t* vals) {
-    const int64_t k = ((int64_t)blockIdx.x * 256 + threadIdx.x) >> 5;
-    const uint32_t lane = threadIdx.x & 31;
-    if (k >= a.nbags) return;
-    const MapParams& mp = a.mp;
-    int64_t lo = __ldg(a.offsets + k), hi = __ldg(a.offsets + k + 1);
-    lo = lo < 0 ? 0 : (lo > a.nnz ? a.nnz : lo);
-    hi = hi < lo ? lo : (hi > a.nnz ? a.nnz : hi);
-    if (k == 0) lo = 0;
-    if (k == a.nbags - 1) hi = a.nnz;
-    const uint32_t e = table_of_bag((uint64_t)k, mp);
-    const uint64_t tterm = table_term(mp.h, e);
-    for (int64_t p = lo + lane; p < hi; p += 32) {
-        const uint64_t x = (uint64_t)a.indices.load(p);
-        const uint64_t q0 = (uint64_t)p * mp.C;
-        if (mp.R > 1) {
-            keys[q0] = id_block_start(mp, e, x, 0);
-            vals[q0] = (uint32_t)((uint64_t)k * mp.d);
-            continue;
-        }
-        const uint64_t base = addmod_p61(tterm, mulmod_p61_any(mp.h.B, x));
-        for (uint32_t c = 0; c < mp.C; ++c) {
-            keys[q0 + c] = block_start(mp, base, c);
-            vals[q0 + c] = (uint32_t)((uint64_t)k * mp.d + c * mp.Z);
-        }
-    }
-}
-
 // The same, one thread per block: for many blocks per id (small Z) the writes of one thread per
 // id would be far apart, and re-evaluating the shared part of the hash per block costs less.
 template <bool SIGN>
@@ -927,18 +894,12 @@ cudaError_t launch_backward_det(const Problem& pb, const float* grad_out, float*
     uint32_t* totals = (uint32_t*)(ws + L.totals);
 
     KeyArgs ka{mp, pb.indices, pb.offsets, pb.nbags, pb.nnz, pb.status};
-    const bool keys_by_bag = bags && !pb.sign && mp.C <= 8;
-    if (keys_by_bag) {
-        bag_of = nullptr;  // nothing downstream needs it when the sign hash is off
-        det_keys_by_bag_kernel<<<(unsigned)((pb.nbags + 7) / 8), 256, 0, st>>>(ka, kA, vA);
-    } else if (bags) {
+    if (bags) {
         // positions that malformed offsets leave uncovered fall back to bag 0 (memory-safe)
         cudaMemsetAsync(bag_of, 0, (size_t)pb.nnz * sizeof(uint32_t), st);
         det_bag_of_kernel<<<(unsigned)((pb.nbags + 7) / 8), 256, 0, st>>>(ka, bag_of);
     }
-    if (keys_by_bag) {
-        // done above
-    } else if (mp.C <= 8) {
+    if (mp.C <= 8) {
         const unsigned kb = (unsigned)((pb.nnz + 255) / 256);
         if (pb.sign) det_keys_kernel<true><<<kb, 256, 0, st>>>(ka, bag_of, kA, vA, nb);
         else det_keys_kernel<false><<<kb, 256, 0, st>>>(ka, bag_of, kA, vA, nb);
