@@ -775,7 +775,7 @@ det_apply_low_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint32_t
 }
 
 // Binned (not deterministic) backward: after ONE scatter pass on the top key bits the blocks are
-// grouped by array region (a bin covers 2^shift consecutive slots, a few MB), and this kernel
+// grouped by array region (a bin covers 2^shift consecutive slots, 16 MB or so), and this kernel
 // adds them in that order with red.global: thread (i, u) adds term u of sorted block i.  The
 // blocks in flight at any moment fall into one or two bins, so the read-modify-write of the array
 // happens in L2 and every array sector crosses the DRAM bus about once per call instead of once
@@ -912,8 +912,11 @@ cudaError_t launch_backward_det(const Problem& pb, const float* grad_out, float*
     const SortPlan sp = make_plan(nb);
     const uint32_t bits = bits_for(mp.m);
     if (mode == 3) {
-        // binned: one pass on the top 8 key bits, then atomic adds in bin order
-        const uint32_t shift = bits > 8 ? bits - 8 : 0;
+        // binned: one pass on the top key bits, then atomic adds in bin order.  A bin spans 2^22
+        // slots (16 MB of fp32: the span that measured fastest on a 1 GB array - small enough to
+        // be updated in L2, large enough that the scatter writes long runs) unless that would
+        // need more than 256 bins or the array is smaller than one such span.
+        const uint32_t shift = bits > 30 ? bits - 8 : (bits > 22 ? 22 : (bits > 8 ? bits - 8 : 0));
         const uint32_t mask = (1u << (bits - shift)) - 1u;
         sort_count_kernel<<<sp.grid, kSortThreads, 0, st>>>(kA, counts, nb, sp.tiles, shift, mask);
         sort_scan_kernel<<<kRadix, kSortThreads, 0, st>>>(counts, totals, sp.grid);
