@@ -42,7 +42,7 @@ NCU_TRAFFIC_BYTES = {
     ("cfg4_multihot", "atomic"): {"forward": 4_197_885_696, "backward": 7_509_030_400},
     ("cfg4_multihot", "det"): {"forward": 4_197_885_696, "backward": None},
     # binned: the six kernels of the backward together (profiles/launches_cfg4_multihot.md)
-    ("cfg4_multihot", "binned"): {"forward": 4197141266, "backward": 5260333275},
+    ("cfg4_multihot", "binned"): {"forward": 4196867254, "backward": 5141565238},
 }
 
 
