@@ -79,7 +79,7 @@ __global__ void __launch_bounds__(256) det_bag_of_kernel(KeyArgs a, uint32_t* ba
 // One thread per id: the part of the hash that all chunks of the id share is evaluated once.
 template <bool SIGN>
 __global__ void __launch_bounds__(256)
-det_keys_kernel(KeyArgs a, const uint32_t* bag_of, uint32_t* keys, uint32_t* vals, uint64_t nb) {
+det_keys_kernel(KeyArgs a, const uint32_t* bag_of, uint32_t* keys, uint32_t* vals) {
     const uint64_t p = (uint64_t)blockIdx.x * 256 + threadIdx.x;
     if (p >= (uint64_t)a.nnz) return;
     const MapParams& mp = a.mp;
@@ -97,7 +97,6 @@ det_keys_kernel(KeyArgs a, const uint32_t* bag_of, uint32_t* keys, uint32_t* val
         keys[q0 + c] = block_start(mp, base, c);
         vals[q0 + c] = SIGN ? (uint32_t)(q0 + c) : (uint32_t)(bag * mp.d + c * mp.Z);
     }
-    (void)nb;
 }
 
 // The same, one thread per block: for many blocks per id (small Z) the writes of one thread per
@@ -374,9 +373,6 @@ __device__ __forceinline__ void commit_slot(const ApplyArgs& a, uint32_t j, floa
 // after those asked into L2 ahead of time; one that is still going after 256 positions is
 // handed, with its sums so far, to the long-walk kernel below (or finished here if the list of
 // handed-over rounds is full).
-#ifndef ROBE_DEEP_UN
-#define ROBE_DEEP_UN 16
-#endif
 constexpr uint32_t kRing = 128;
 constexpr uint32_t kNoKey = 0xFFFFFFFFu;  // above every slot number (m + d <= 2^32)
 
@@ -469,7 +465,7 @@ __device__ __forceinline__ bool walk_steps(const ApplyArgs& a, const uint32_t* b
 __device__ __forceinline__ bool walk_deep(const ApplyArgs& a, ApplyTile& tl, ApplyWalk& wk, uint32_t j,
                                           uint32_t sub, uint32_t EPW, uint32_t lane,
                                           uint32_t chunk_off, uint32_t limit) {
-    constexpr int UN = ROBE_DEEP_UN;
+    constexpr int UN = 16;
     const float* pf = a.grad_out + chunk_off;
     // the ring has to reach the end of the first step before the one-step-ahead fetches take over
     if (wk.pending) walk_commit(tl, wk, lane, pf);
@@ -901,8 +897,8 @@ cudaError_t launch_backward_det(const Problem& pb, const float* grad_out, float*
     }
     if (mp.C <= 8) {
         const unsigned kb = (unsigned)((pb.nnz + 255) / 256);
-        if (pb.sign) det_keys_kernel<true><<<kb, 256, 0, st>>>(ka, bag_of, kA, vA, nb);
-        else det_keys_kernel<false><<<kb, 256, 0, st>>>(ka, bag_of, kA, vA, nb);
+        if (pb.sign) det_keys_kernel<true><<<kb, 256, 0, st>>>(ka, bag_of, kA, vA);
+        else det_keys_kernel<false><<<kb, 256, 0, st>>>(ka, bag_of, kA, vA);
     } else {
         const unsigned kb = (unsigned)((nb + 255) / 256);
         if (pb.sign) det_keys_by_block_kernel<true><<<kb, 256, 0, st>>>(ka, bag_of, kA, vA, nb);
