@@ -455,6 +455,24 @@ def test_validate_mode_reports_bad_inputs_without_faulting():
         assert robe.robe_last_device_status(c.h) == 1
 
 
+@pytest.mark.parametrize("mode", ["atomic", "binned", "det"])
+def test_validate_mode_stops_every_backward_variant(mode):
+    # a bad id under ROBE_OPT_VALIDATE: the status word says so and no kernel touches the target
+    w = small(bag_rule=(2, 0, 5))
+    with Case(w, batch=8) as c:
+        word = torch.zeros(1, dtype=torch.int32, device=c.dev)
+        robe.robe_set_status_word(c.h, word)
+        robe.robe_set_option(c.h, robe.ROBE_OPT_VALIDATE, 1)
+        _, g_d = _grad(c, 3)
+        good = c.backward(g_d, mode).cpu().numpy()
+        assert robe.robe_last_device_status(c.h) == 0 and np.any(good != 0)
+        c.indices = c.indices.clone()
+        c.indices[1] = -7
+        ga = c.backward(g_d, mode).cpu().numpy()
+        assert robe.robe_last_device_status(c.h) == 1
+        assert not np.any(ga)
+
+
 def test_argument_errors_on_device():
     with Case(small()) as c:
         out = torch.empty(c.B, c.T, c.w.d, device=c.dev)
