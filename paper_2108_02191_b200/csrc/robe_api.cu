@@ -94,6 +94,18 @@ Problem make_problem(robe_ctx* h, const void* indices, const int64_t* offsets, i
     return pb;
 }
 
+// Size limits of the sort-based backward variants (binned, deterministic, Adam): block numbers,
+// bag numbers and positions in grad_out are 32-bit, and the binned adds run one thread per
+// (block, offset) on a one-dimensional grid.
+bool sorted_path_fits(const robe_ctx* h, const Problem& pb) {
+    const uint64_t nb = (uint64_t)pb.nnz * h->mp.C;
+    uint32_t zp = 1;
+    while (zp < h->mp.Z) zp <<= 1;
+    if (nb >= (1ull << 32) || (uint64_t)pb.nbags >= (1ull << 32)) return false;
+    if (nb * zp / 256 >= (1ull << 31)) return false;
+    return (uint64_t)pb.nbags * h->mp.d <= (1ull << 32);
+}
+
 }  // namespace
 
 namespace robe {
@@ -267,13 +279,8 @@ int robe_backward(robe_handle_t h, const float* grad_out, const void* indices,
             return ROBE_ERR_CUDA;
         return ROBE_OK;
     }
-    // deterministic: 32-bit block numbers and a grid of one thread per (block, offset)
-    const uint64_t nb = (uint64_t)nnz * h->mp.C;
-    uint32_t zp = 1;
-    while (zp < h->mp.Z) zp <<= 1;
-    if (nb >= (1ull << 32) || (uint64_t)pb.nbags >= (1ull << 32)) return ROBE_ERR_UNSUPPORTED;
-    if (nb * zp / 256 >= (1ull << 31)) return ROBE_ERR_UNSUPPORTED;
-    if ((uint64_t)pb.nbags * h->mp.d > (1ull << 32)) return ROBE_ERR_UNSUPPORTED;
+    // the sort-based variants (binned, deterministic)
+    if (!sorted_path_fits(h, pb)) return ROBE_ERR_UNSUPPORTED;
     const size_t need = det_workspace_bytes(h->mp, pb.nbags, nnz, offsets != nullptr);
     if (nnz > 0 && (workspace == nullptr || workspace_bytes < need)) return ROBE_ERR_WORKSPACE;
     if (((uintptr_t)workspace & 255u) != 0) return ROBE_ERR_WORKSPACE;
@@ -319,12 +326,7 @@ int robe_backward_deterministic_static(robe_handle_t h, const float* grad_out,
     }
     float* target = sgd ? (float*)h->array : grad_array;
     const Problem pb = make_problem(h, indices, offsets, batch, nnz);
-    const uint64_t nb = (uint64_t)nnz * h->mp.C;
-    uint32_t zp = 1;
-    while (zp < h->mp.Z) zp <<= 1;
-    if (nb >= (1ull << 32) || (uint64_t)pb.nbags >= (1ull << 32)) return ROBE_ERR_UNSUPPORTED;
-    if (nb * zp / 256 >= (1ull << 31)) return ROBE_ERR_UNSUPPORTED;
-    if ((uint64_t)pb.nbags * h->mp.d > (1ull << 32)) return ROBE_ERR_UNSUPPORTED;
+    if (!sorted_path_fits(h, pb)) return ROBE_ERR_UNSUPPORTED;
     // the fixed array is the whole workspace: a call that needs more is refused up front (by
     // the same figure robe_backward_workspace_bytes reports, which covers pooled input too)
     const size_t need = det_workspace_bytes(h->mp, pb.nbags, nnz, true);
@@ -356,12 +358,7 @@ int robe_backward_adam(robe_handle_t h, const float* grad_out, const void* indic
     if (h->array == nullptr) return ROBE_ERR_NO_ARRAY;
     if (h->dtype != ROBE_F32) return ROBE_ERR_INVALID_ARG;
     const Problem pb = make_problem(h, indices, offsets, batch, nnz);
-    const uint64_t nb = (uint64_t)nnz * h->mp.C;
-    uint32_t zp = 1;
-    while (zp < h->mp.Z) zp <<= 1;
-    if (nb >= (1ull << 32) || (uint64_t)pb.nbags >= (1ull << 32)) return ROBE_ERR_UNSUPPORTED;
-    if (nb * zp / 256 >= (1ull << 31)) return ROBE_ERR_UNSUPPORTED;
-    if ((uint64_t)pb.nbags * h->mp.d > (1ull << 32)) return ROBE_ERR_UNSUPPORTED;
+    if (!sorted_path_fits(h, pb)) return ROBE_ERR_UNSUPPORTED;
     const size_t need = det_workspace_bytes(h->mp, pb.nbags, nnz, offsets != nullptr);
     if (nnz > 0 && (workspace == nullptr || workspace_bytes < need)) return ROBE_ERR_WORKSPACE;
     if (((uintptr_t)workspace & 255u) != 0) return ROBE_ERR_WORKSPACE;
