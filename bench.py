@@ -36,12 +36,12 @@ METRIC = "robe_lookups_per_s_fwd_bwd"
 UNIT = "ids/s"
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu capture of the
-# full-size default workload that profiles/dram_traffic_cfg4_multihot.md summarises; None = not
+# full-size default workload (summaries of those captures are kept under profiles/); None = not
 # captured for that workload or backward variant.
 NCU_TRAFFIC_BYTES = {
     ("cfg4_multihot", "atomic"): {"forward": 4_197_885_696, "backward": 7_509_030_400},
     ("cfg4_multihot", "det"): {"forward": 4_197_885_696, "backward": None},
-    # binned: the six kernels of the backward together (profiles/launches_cfg4_multihot.md)
+    # binned: the six kernels of the backward together
     ("cfg4_multihot", "binned"): {"forward": 4196867254, "backward": 5141565238},
 }
 
