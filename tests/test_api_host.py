@@ -102,3 +102,26 @@ def test_workspace_grows_with_blocks():
     b = robe.robe_backward_workspace_bytes(h, 2048, 2048 * 26)
     assert b > a >= 16 * 1024 * 26 * 128
     robe.robe_destroy(h)
+
+
+def test_sort_based_variants_refuse_sizes_beyond_their_32_bit_numbering():
+    # block numbers, bag numbers and gradient positions are 32-bit in the binned / deterministic /
+    # Adam paths: larger calls are refused before anything is launched (dummy pointers are never read)
+    lib = robe.binding.raw()
+    dummy = C.c_void_p(0x1000)
+    h = robe.robe_create(1 << 20, 4, 16, 1, 3)        # C = 4 blocks per id
+    assert lib.robe_attach_array(h, dummy, robe.ROBE_F32) == robe.ROBE_OK
+    big = 1 << 30                                     # 2^30 ids -> 2^32 blocks
+    for mode in (robe.ROBE_BWD_DETERMINISTIC, robe.ROBE_BWD_BINNED):
+        robe.robe_set_option(h, robe.ROBE_OPT_BWD_MODE, mode)
+        assert lib.robe_backward(h, dummy, dummy, None, big, big, dummy, 0.0, dummy, 1 << 40, None) \
+            == robe.ROBE_ERR_UNSUPPORTED
+    assert lib.robe_backward_adam(h, dummy, dummy, None, big, big, dummy, dummy, 0.1, 0.9, 0.999, 1e-8, 1,
+                                  dummy, 1 << 40, None) == robe.ROBE_ERR_UNSUPPORTED
+    assert lib.robe_backward_deterministic_static(h, dummy, dummy, None, big, big, dummy, 0.0, None) \
+        == robe.ROBE_ERR_UNSUPPORTED
+    # atomic mode has no such limit on the host side, but still wants consistent sizes
+    robe.robe_set_option(h, robe.ROBE_OPT_BWD_MODE, robe.ROBE_BWD_ATOMIC)
+    assert lib.robe_backward(h, dummy, dummy, None, big, big - 1, dummy, 0.0, None, 0, None) \
+        == robe.ROBE_ERR_INVALID_ARG
+    robe.robe_destroy(h)
