@@ -28,6 +28,10 @@ struct robe_ctx {
     int bwd_variant;
     int32_t* status_word;
     int index_type;
+    // second stream of the deterministic backward, made at the first call that can use it
+    bool side_tried;
+    cudaStream_t side;
+    cudaEvent_t fork_event, join_event;
 };
 
 namespace {
@@ -92,6 +96,34 @@ Problem make_problem(robe_ctx* h, const void* indices, const int64_t* offsets, i
     pb.nnz = nnz;
     pb.status = (h->validate && h->status_word) ? h->status_word : nullptr;
     return pb;
+}
+
+// The deterministic backward runs its two apply kernels side by side: the one that walks often
+// repeated ids (few CTAs, long) in a stream of higher priority, forked from and joined to the
+// caller's stream by events.  Made once per handle; if that fails the kernels run one after the
+// other in the caller's stream.
+void lend_side_stream(robe_ctx* h, Problem& pb) {
+    if (!h->side_tried) {
+        h->side_tried = true;
+        int least = 0, greatest = 0;
+        cudaStream_t s = nullptr;
+        cudaEvent_t e0 = nullptr, e1 = nullptr;
+        if (cudaDeviceGetStreamPriorityRange(&least, &greatest) == cudaSuccess &&
+            cudaStreamCreateWithPriority(&s, cudaStreamNonBlocking, greatest) == cudaSuccess &&
+            cudaEventCreateWithFlags(&e0, cudaEventDisableTiming) == cudaSuccess &&
+            cudaEventCreateWithFlags(&e1, cudaEventDisableTiming) == cudaSuccess) {
+            h->side = s;
+            h->fork_event = e0;
+            h->join_event = e1;
+        } else {
+            if (e0 != nullptr) cudaEventDestroy(e0);
+            if (s != nullptr) cudaStreamDestroy(s);
+            (void)cudaGetLastError();
+        }
+    }
+    pb.side = h->side;
+    pb.fork_event = h->fork_event;
+    pb.join_event = h->join_event;
 }
 
 // Size limits of the sort-based backward variants (binned, deterministic, Adam): block numbers,
@@ -164,12 +196,21 @@ int robe_create(robe_handle_t* out, uint64_t M, uint32_t Z, uint32_t d, uint32_t
     h->bwd_variant = 0;
     h->status_word = nullptr;
     h->index_type = ROBE_I64;
+    h->side_tried = false;
+    h->side = nullptr;
+    h->fork_event = h->join_event = nullptr;
     *out = h;
     return ROBE_OK;
 }
 
 int robe_destroy(robe_handle_t h) {
     if (h == nullptr) return ROBE_ERR_INVALID_ARG;
+    if (h->side != nullptr) {
+        cudaStreamSynchronize(h->side);
+        cudaStreamDestroy(h->side);
+        cudaEventDestroy(h->fork_event);
+        cudaEventDestroy(h->join_event);
+    }
     delete h;
     return ROBE_OK;
 }
@@ -270,7 +311,7 @@ int robe_backward(robe_handle_t h, const float* grad_out, const void* indices,
         if (h->dtype != ROBE_F32) return ROBE_ERR_INVALID_ARG;
     }
     float* target = sgd ? (float*)h->array : grad_array;
-    const Problem pb = make_problem(h, indices, offsets, batch, nnz);
+    Problem pb = make_problem(h, indices, offsets, batch, nnz);
     cudaStream_t st = (cudaStream_t)stream;
     if (h->bwd_mode == ROBE_BWD_ATOMIC) {
         if (launch_validate(pb, st) != cudaSuccess) return ROBE_ERR_CUDA;
@@ -286,6 +327,7 @@ int robe_backward(robe_handle_t h, const float* grad_out, const void* indices,
     if (((uintptr_t)workspace & 255u) != 0) return ROBE_ERR_WORKSPACE;
     if (launch_validate(pb, st) != cudaSuccess) return ROBE_ERR_CUDA;
     const bool binned = h->bwd_mode == ROBE_BWD_BINNED;
+    if (!binned) lend_side_stream(h, pb);
     if (launch_backward_det(pb, grad_out, target, binned ? 3 : (sgd ? 1 : 0),
                             binned ? (sgd ? -lr : 1.0f) : lr, nullptr, workspace, workspace_bytes,
                             st) != cudaSuccess)
@@ -325,7 +367,7 @@ int robe_backward_deterministic_static(robe_handle_t h, const float* grad_out,
         if (h->dtype != ROBE_F32) return ROBE_ERR_INVALID_ARG;
     }
     float* target = sgd ? (float*)h->array : grad_array;
-    const Problem pb = make_problem(h, indices, offsets, batch, nnz);
+    Problem pb = make_problem(h, indices, offsets, batch, nnz);
     if (!sorted_path_fits(h, pb)) return ROBE_ERR_UNSUPPORTED;
     // the fixed array is the whole workspace: a call that needs more is refused up front (by
     // the same figure robe_backward_workspace_bytes reports, which covers pooled input too)
@@ -357,11 +399,12 @@ int robe_backward_adam(robe_handle_t h, const float* grad_out, const void* indic
     if (h->validate && h->status_word == nullptr) return ROBE_ERR_INVALID_ARG;
     if (h->array == nullptr) return ROBE_ERR_NO_ARRAY;
     if (h->dtype != ROBE_F32) return ROBE_ERR_INVALID_ARG;
-    const Problem pb = make_problem(h, indices, offsets, batch, nnz);
+    Problem pb = make_problem(h, indices, offsets, batch, nnz);
     if (!sorted_path_fits(h, pb)) return ROBE_ERR_UNSUPPORTED;
     const size_t need = det_workspace_bytes(h->mp, pb.nbags, nnz, offsets != nullptr);
     if (nnz > 0 && (workspace == nullptr || workspace_bytes < need)) return ROBE_ERR_WORKSPACE;
     if (((uintptr_t)workspace & 255u) != 0) return ROBE_ERR_WORKSPACE;
+    lend_side_stream(h, pb);
     AdamState ad;
     ad.m1 = m1;
     ad.m2 = m2;

@@ -307,6 +307,11 @@ struct ApplyArgs {
     uint32_t* long_count;    // number of handed-over rounds (may run past long_cap)
     LongWalk* long_walks;
     uint32_t long_cap;
+    // window apply (densely touched arrays): per array window of 2^win_log2 slots, did the window kernel
+    // leave it to the position-tile kernel?  nullptr = there is no window kernel in this call
+    const uint8_t* win_left;
+    const uint32_t* any_left;  // number of windows left over (0: the tile kernel has nothing to do)
+    uint32_t win_log2;         // log2 of the window length
 };
 
 // The term that the sorted block with payload v contributes to the slot at in-block offset o
@@ -374,6 +379,11 @@ __device__ __forceinline__ void commit_slot(const ApplyArgs& a, uint32_t j, floa
 // handed, with its sums so far, to the long-walk kernel below (or finished here if the list of
 // handed-over rounds is full).
 constexpr uint32_t kRing = 128;
+// window apply: the array is cut into windows of 2^8 .. 2^11 slots, one CTA each
+constexpr uint32_t kWinLog2Min = 8, kWinLog2Max = 11;
+constexpr uint32_t kWinMaxZ = 128;        // longest block the window kernel takes
+constexpr uint32_t kWinEnt = 1024;        // sorted blocks per chunk, at most
+constexpr uint32_t kWinStage = 6144;      // gradient elements per chunk, at most (>= kWinMaxZ)
 constexpr uint32_t kNoKey = 0xFFFFFFFFu;  // above every slot number (m + d <= 2^32)
 
 struct ApplyTile {
@@ -517,6 +527,7 @@ det_apply_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint32_t* __
     constexpr uint32_t kHandOverAfter = 256;  // ... and after which it goes to the long-walk kernel
     __shared__ uint2 ring_s[8][kRing];
     if (a.status != nullptr && *a.status != 0) return;
+    if (a.any_left != nullptr && *a.any_left == 0) return;  // the window kernel served every slot
     const MapParams& mp = a.mp;
     const uint32_t lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     ApplyTile tl;
@@ -572,7 +583,8 @@ det_apply_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint32_t* __
         const uint32_t u = mp.Z - (incl_e - idx);  // lo_e <= u < Z for a real pair
         const uint64_t j64 = (uint64_t)s + u;
         // j64 >= m: wrapped part, j64 < Z-1: low slots - both belong to the other kernel
-        const bool active = idx < total && u >= lo_e && u < mp.Z && j64 < mp.m && j64 + 1 >= mp.Z;
+        bool active = idx < total && u >= lo_e && u < mp.Z && j64 < mp.m && j64 + 1 >= mp.Z;
+        if (active && a.win_left != nullptr) active = a.win_left[j64 >> a.win_log2] != 0;
         if (__ballot_sync(0xFFFFFFFFu, active) == 0) continue;
         const uint32_t j = (uint32_t)j64;
         float old = 0.0f;
@@ -624,6 +636,173 @@ det_apply_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint32_t* __
         }
         if (wk.touched) commit_slot<MODE>(a, j, wk.acc, old);
     }
+}
+
+// ---- window apply: the slot-major way, for arrays that a call touches densely (plain blocks
+// of full length).  The array is cut into windows of W = 2^win_log2 slots.
+//
+// lo_of[b] = first sorted position whose block reaches slot b*W or a later one (key + Z-1 >= b*W),
+// hi_of[b] = first sorted position whose key is >= b*W; both for b = 0 .. number of windows.
+constexpr int kBoundsPer = 8;  // sorted positions per thread
+
+__global__ void __launch_bounds__(256)
+det_bounds_kernel(const uint32_t* __restrict__ K, uint64_t nb, uint32_t* lo_of, uint32_t* hi_of,
+                  uint32_t nwin, uint32_t win_log2, uint32_t Z) {
+    const uint64_t i0 = ((uint64_t)blockIdx.x * 256 + threadIdx.x) * kBoundsPer;
+    if (i0 > nb) return;
+    uint64_t k[kBoundsPer + 1];  // k[t] = key before position i0 + t
+    k[0] = i0 > 0 ? (uint64_t)__ldg(K + i0 - 1) : 0;
+#pragma unroll
+    for (int t = 0; t < kBoundsPer; ++t) k[t + 1] = i0 + t < nb ? (uint64_t)__ldg(K + i0 + t) : ~0ull;
+#pragma unroll
+    for (int t = 0; t < kBoundsPer; ++t) {
+        const uint64_t i = i0 + t;
+        if (i > nb) break;
+        // windows b with b*W in (k[t], k[t+1]] get hi_of[b] = i (and b = 0 at i = 0)
+        uint64_t from = i > 0 ? (k[t] >> win_log2) + 1 : 0;
+        uint64_t to = i < nb ? (k[t + 1] >> win_log2) : nwin;
+        for (uint64_t b = from; b <= to && b <= nwin; ++b) hi_of[b] = (uint32_t)i;
+        from = i > 0 ? ((k[t] + (Z - 1)) >> win_log2) + 1 : 0;
+        to = i < nb ? ((k[t + 1] + (Z - 1)) >> win_log2) : nwin;
+        for (uint64_t b = from; b <= to && b <= nwin; ++b) lo_of[b] = (uint32_t)i;
+    }
+}
+
+// win_left[b] = 1 for a window reached by more than n_max sorted blocks (an id that occurs very
+// often in the batch falls there): the position-tile kernel and the long-walk kernel serve the
+// slots of such windows, the window kernel all others.  *any_left counts them.
+__global__ void __launch_bounds__(256)
+det_window_classify_kernel(const uint32_t* __restrict__ lo_of, const uint32_t* __restrict__ hi_of,
+                           uint32_t nwin, uint32_t n_max, uint8_t* win_left, uint32_t* any_left) {
+    const uint32_t b = blockIdx.x * 256 + threadIdx.x;
+    const bool left = b < nwin && hi_of[b + 1] - lo_of[b] > n_max;
+    if (b < nwin) win_left[b] = left ? 1 : 0;
+    const uint32_t votes = __ballot_sync(0xFFFFFFFFu, left);
+    if ((threadIdx.x & 31) == 0 && votes != 0) atomicAdd(any_left, (uint32_t)__popc(votes));
+}
+
+// One CTA per window.  The sorted blocks that reach the window are positions [lo_of[b],
+// hi_of[b+1]).  A histogram of their keys (relative to w0 - (Z-1)) and its prefix sums give, for
+// every slot of the window, the range of blocks that reach it - those with key in [j-Z+1, j] -
+// already in sorted order.  The blocks then stream through shared memory in chunks, each chunk
+// with its gradient elements (fetched by coalesced loads); every thread owns the slots
+// tid, tid+256, ... of the window and adds, per chunk, the terms of its slots' ranges from first
+// to last, keeping the running sums in registers.  All slots are committed at the end.
+template <int MODE>
+__global__ void __launch_bounds__(256, 5)
+det_apply_window_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint32_t* __restrict__ V,
+                        const uint32_t* __restrict__ lo_of, const uint32_t* __restrict__ hi_of,
+                        uint32_t chunk, int vec4) {
+    __shared__ uint2 ent[kWinEnt];
+    __shared__ __align__(16) float stage[kWinStage];
+    __shared__ uint32_t pre[(1u << kWinLog2Max) + kWinMaxZ + 8];  // count per key offset, then prefix
+    __shared__ uint32_t warp_sums[8];
+    if (a.status != nullptr && *a.status != 0) return;
+    const MapParams& mp = a.mp;
+    const uint32_t tid = threadIdx.x, lane = tid & 31;
+    const uint32_t b = blockIdx.x;
+    if (a.win_left[b] != 0) return;
+    const uint32_t W = 1u << a.win_log2, Z = mp.Z;
+    const uint64_t w0 = (uint64_t)b << a.win_log2;
+    const uint32_t lo = lo_of[b], hi = hi_of[b + 1];
+    const uint32_t n = hi - lo;
+    if (n == 0) return;
+    const bool one_chunk = n <= chunk;
+    const uint32_t span = W + Z - 1;  // key offsets 0 .. span-1, relative to w0 - (Z-1)
+    for (uint32_t t = tid; t <= span; t += 256) pre[t] = 0;
+    __syncthreads();
+    for (uint32_t e0 = 0; e0 < n; e0 += 256) {
+        const uint32_t e = e0 + tid;
+        uint32_t off = 0xFFFFFFFFu;
+        if (e < n) {
+            const uint32_t k = __ldg(K + lo + e);
+            if (one_chunk) ent[e] = make_uint2(k, __ldg(V + lo + e));
+            off = (uint32_t)((uint64_t)k + (Z - 1) - w0);
+        }
+        const uint32_t off0 = __shfl_sync(0xFFFFFFFFu, off, 0);
+        if (__all_sync(0xFFFFFFFFu, off == off0)) {  // a run of one key: count it once
+            if (lane == 0 && off != 0xFFFFFFFFu) atomicAdd(&pre[off], 32u);
+        } else if (off != 0xFFFFFFFFu) {
+            atomicAdd(&pre[off], 1u);
+        }
+    }
+    __syncthreads();
+    // exclusive prefix sums over pre[0 .. span], each thread a run of consecutive offsets
+    {
+        const uint32_t per = (span + 1 + 255) / 256;
+        const uint32_t t0 = tid * per < span + 1 ? tid * per : span + 1;
+        const uint32_t t1 = t0 + per < span + 1 ? t0 + per : span + 1;
+        uint32_t mine = 0;
+        for (uint32_t t = t0; t < t1; ++t) mine += pre[t];
+        uint32_t run = cta_exclusive_scan_256(mine, warp_sums);  // syncs inside
+        for (uint32_t t = t0; t < t1; ++t) {
+            const uint32_t c = pre[t];
+            pre[t] = run;
+            run += c;
+        }
+    }
+    __syncthreads();
+    // slot j = w0 + sl is reached by the blocks with key offset in [sl, sl + Z - 1]:
+    // sorted positions lo + [pre[sl], pre[sl + Z])
+    constexpr int kSlots = (1 << kWinLog2Max) / 256;
+    float acc[kSlots];
+#pragma unroll
+    for (int q = 0; q < kSlots; ++q) acc[q] = 0.0f;
+    for (uint32_t c0 = 0; c0 < n; c0 += chunk) {
+        const uint32_t c1 = c0 + chunk < n ? c0 + chunk : n;
+        const uint32_t ne = c1 - c0;
+        if (!one_chunk) {
+            if (c0 != 0) __syncthreads();  // the chunk before has been used
+            for (uint32_t e = tid; e < ne; e += 256)
+                ent[e] = make_uint2(__ldg(K + lo + c0 + e), __ldg(V + lo + c0 + e));
+            __syncthreads();
+        }
+        if (vec4) {
+            const uint32_t zq = Z >> 2, tot = ne * zq;
+            const bool pow2 = mp.log2Z != 0xFFFFFFFFu;
+            for (uint32_t t = tid; t < tot; t += 256) {
+                const uint32_t e = pow2 ? t >> (mp.log2Z - 2) : t / zq, o = t - e * zq;
+                reinterpret_cast<float4*>(stage)[t] =
+                    __ldg(reinterpret_cast<const float4*>(a.grad_out + ent[e].y) + o);
+            }
+        } else {
+            const uint32_t tot = ne * Z;
+            for (uint32_t t = tid; t < tot; t += 256) {
+                const uint32_t e = t / Z, o = t - e * Z;
+                stage[t] = __ldg(a.grad_out + ((uint64_t)ent[e].y + o));
+            }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int q = 0; q < kSlots; ++q) {
+            const uint32_t sl = tid + q * 256;
+            if (sl >= W) break;
+            const uint32_t first = pre[sl], last = pre[sl + Z];
+            const uint32_t f = first > c0 ? first : c0;
+            const uint32_t l = last < c1 ? last : c1;
+            if (f < l) {
+                const uint32_t j = (uint32_t)w0 + sl;  // (a slot past the array is dropped below)
+                float s = acc[q];
+                for (uint32_t e = f - c0; e < l - c0; ++e)
+                    s = __fadd_rn(s, stage[e * Z + (j - ent[e].x)]);
+                acc[q] = s;
+            }
+        }
+    }
+    // commit: the old values of all the thread's slots are asked for together
+    float old[kSlots];
+    bool has[kSlots];
+#pragma unroll
+    for (int q = 0; q < kSlots; ++q) {
+        const uint32_t sl = tid + q * 256;
+        const uint64_t j64 = w0 + sl;
+        // low slots belong to the low-slot kernel; past the array lie the wrapped tails (the same)
+        has[q] = sl < W && j64 < mp.m && j64 + 1 >= Z && pre[sl + Z] != pre[sl];
+        old[q] = has[q] ? a.target[j64] : 0.0f;
+    }
+#pragma unroll
+    for (int q = 0; q < kSlots; ++q)
+        if (has[q]) commit_slot<MODE>(a, (uint32_t)(w0 + tid + q * 256), acc[q], old[q]);
 }
 
 // Long walks (plain blocks only).  One CTA of four warps per handed-over round, in steps of
@@ -740,34 +919,55 @@ det_apply_long_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint32_
 }
 
 // Slots j in [0, Z-1): plain blocks with key <= j first, then the wrapped tails of blocks
-// whose key lies in [m + j - (Z-1), m-1] (o = j + m - key).
+// whose key lies in [m + j - (Z-1), m-1] (o = j + m - key).  One warp per slot: the lanes fetch
+// the terms of 32 consecutive sorted positions, then all lanes add them in order.
+constexpr unsigned kLowWarps = 4;
+
+template <bool SIGN, bool SHORT>
+__device__ __forceinline__ void low_walk(const ApplyArgs& a, const uint32_t* __restrict__ K,
+                                         const uint32_t* __restrict__ V, const uint32_t* bag_of,
+                                         uint64_t from, uint64_t to, uint64_t j_plus, float& acc,
+                                         bool& touched) {
+    const uint32_t lane = threadIdx.x & 31;
+    for (uint64_t i0 = from; i0 < to; i0 += 32) {
+        const uint64_t i = i0 + lane;
+        float term = 0.0f;
+        bool ok = false;
+        if (i < to) ok = block_term<SIGN, SHORT>(a, bag_of, __ldg(V + i), (uint32_t)(j_plus - __ldg(K + i)), term);
+        const uint32_t oks = __ballot_sync(0xFFFFFFFFu, ok);
+        if (oks != 0) touched = true;
+        for (uint32_t rest = oks; rest != 0; rest &= rest - 1) {
+            const int src = __ffs((int)rest) - 1;
+            acc = __fadd_rn(acc, __shfl_sync(0xFFFFFFFFu, term, src));
+        }
+    }
+}
+
+// first sorted position with key >= bound (warp-uniform)
+__device__ __forceinline__ uint64_t first_at_least(const uint32_t* __restrict__ K, uint64_t nb, uint64_t bound) {
+    uint64_t lo = 0, hi = nb;
+    while (lo < hi) {
+        const uint64_t mid = lo + ((hi - lo) >> 1);
+        if ((uint64_t)__ldg(K + mid) >= bound) hi = mid; else lo = mid + 1;
+    }
+    return lo;
+}
+
 template <bool SIGN, int MODE, bool SHORT>
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(32 * kLowWarps)
 det_apply_low_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint32_t* __restrict__ V,
                      const uint32_t* __restrict__ bag_of) {
     if (a.status != nullptr && *a.status != 0) return;
     const MapParams& mp = a.mp;
-    for (uint32_t j = threadIdx.x; j + 1 < mp.Z; j += blockDim.x) {
-        float acc = 0.0f, term;
-        bool touched = false;
-        for (uint64_t ii = 0; ii < a.nb && K[ii] <= j; ++ii)
-            if (block_term<SIGN, SHORT>(a, bag_of, V[ii], j - K[ii], term)) {
-                acc = __fadd_rn(acc, term);
-                touched = true;
-            }
-        const uint32_t lowkey = mp.m - (mp.Z - 1) + j;  // > j because m >= Z
-        uint64_t lo = 0, hi = a.nb;                     // first position with key >= lowkey
-        while (lo < hi) {
-            const uint64_t mid = lo + ((hi - lo) >> 1);
-            if (K[mid] >= lowkey) hi = mid; else lo = mid + 1;
-        }
-        for (uint64_t ii = lo; ii < a.nb; ++ii)
-            if (block_term<SIGN, SHORT>(a, bag_of, V[ii], j + (mp.m - K[ii]), term)) {
-                acc = __fadd_rn(acc, term);
-                touched = true;
-            }
-        if (touched) commit_slot<MODE>(a, j, acc, a.target[j]);
-    }
+    const uint32_t j = blockIdx.x * kLowWarps + (threadIdx.x >> 5);
+    if (j + 1 >= mp.Z) return;
+    float acc = 0.0f;
+    bool touched = false;
+    low_walk<SIGN, SHORT>(a, K, V, bag_of, 0, first_at_least(K, a.nb, (uint64_t)j + 1), j, acc, touched);
+    const uint64_t lowkey = (uint64_t)mp.m - (mp.Z - 1) + j;  // > j because m >= Z
+    low_walk<SIGN, SHORT>(a, K, V, bag_of, first_at_least(K, a.nb, lowkey), a.nb, (uint64_t)j + mp.m, acc,
+                          touched);
+    if (touched && (threadIdx.x & 31) == 0) commit_slot<MODE>(a, j, acc, a.target[j]);
 }
 
 // Binned (not deterministic) backward: after ONE scatter pass on the top key bits the blocks are
@@ -817,11 +1017,20 @@ uint32_t bits_for(uint32_t m) {  // bits needed for keys in [0, m)
 }
 
 struct Layout {
-    size_t keysA, keysB, valsA, valsB, bag_of, counts, totals, long_count, long_walks, total;
-    uint32_t long_cap;
+    size_t keysA, keysB, valsA, valsB, bag_of, counts, totals, long_count, long_walks, bounds, win_left,
+        total;
+    uint32_t long_cap, nwin, win_log2;
 };
 
-Layout make_layout(uint64_t nb, int64_t nnz, bool bags) {
+// Window length of the window apply: 2048 slots, fewer for a small array so that there are
+// still several CTAs per SM.
+uint32_t window_log2(uint32_t m) {
+    uint32_t l = kWinLog2Max;
+    while (l > kWinLog2Min && (m >> l) < 1024u) --l;
+    return l;
+}
+
+Layout make_layout(uint64_t nb, int64_t nnz, bool bags, uint32_t m) {
     Layout L;
     size_t off = 0;
     const size_t kb = align256((nb ? nb : 1) * sizeof(uint32_t));
@@ -838,27 +1047,87 @@ Layout make_layout(uint64_t nb, int64_t nnz, bool bags) {
     L.long_cap = (uint32_t)cap;
     L.long_count = off; off += 256;
     L.long_walks = off; off += align256((size_t)cap * sizeof(LongWalk));
+    // window apply: first sorted position of every array window, a left-over flag per window and,
+    // in the flag array's first aligned word past the flags, the count of left-over windows
+    L.win_log2 = window_log2(m);
+    L.nwin = (uint32_t)((((uint64_t)m - 1) >> L.win_log2) + 1);
+    L.bounds = off; off += 2 * align256(((size_t)L.nwin + 1) * sizeof(uint32_t));
+    L.win_left = off; off += align256((size_t)L.nwin + 256);
     L.total = off;
     return L;
 }
 
+// The window kernel pays when most slots are reached, so that walking every slot is no waste.
+bool use_window_apply(const MapParams& mp, uint64_t nb, bool sign) {
+    if (sign || mp.d % mp.Z != 0 || mp.Z > kWinMaxZ || nb == 0) return false;
+    return nb * mp.Z * 2 >= mp.m;
+}
+
+struct WindowBuffers {
+    uint32_t* lo_of;
+    uint32_t* hi_of;
+    uint8_t* left;
+    uint32_t nwin, win_log2;
+    // second stream for the kernels that serve the left-over windows, or nullptr
+    cudaStream_t side;
+    cudaEvent_t fork_event, join_event;
+};
+
 template <bool SIGN, int MODE>
-void launch_apply(const ApplyArgs& aa, const uint32_t* K, const uint32_t* V, const uint32_t* bag_of,
-                  cudaStream_t st) {
+void launch_apply(ApplyArgs aa, const uint32_t* K, const uint32_t* V, const uint32_t* bag_of,
+                  const WindowBuffers& wb, cudaStream_t st) {
     const MapParams& mp = aa.mp;
+    const bool windows = !SIGN && use_window_apply(mp, aa.nb, SIGN);
+    uint32_t chunk = kWinStage / mp.Z;
+    if (chunk > kWinEnt) chunk = kWinEnt;
+    if (windows) {
+        const size_t flags = ((size_t)wb.nwin + 255) & ~(size_t)255;
+        uint32_t* any_left = (uint32_t*)(wb.left + flags);
+        cudaMemsetAsync(any_left, 0, sizeof(uint32_t), st);
+        const uint64_t per_cta = 256ull * kBoundsPer;
+        det_bounds_kernel<<<(unsigned)(aa.nb / per_cta + 1), 256, 0, st>>>(K, aa.nb, wb.lo_of, wb.hi_of,
+                                                                          wb.nwin, wb.win_log2, mp.Z);
+        // a window reached by many times the average number of blocks holds an often repeated id
+        const uint64_t mean = (((uint64_t)1 << wb.win_log2) + mp.Z) * aa.nb / mp.m + 1;
+        const uint64_t n_max = mean * 4 > 512 ? mean * 4 : 512;
+        det_window_classify_kernel<<<(wb.nwin + 255) / 256, 256, 0, st>>>(
+            wb.lo_of, wb.hi_of, wb.nwin, (uint32_t)(n_max < 0xFFFFFFFFull ? n_max : 0xFFFFFFFFull), wb.left,
+            any_left);
+        aa.win_left = wb.left;
+        aa.any_left = any_left;
+        aa.win_log2 = wb.win_log2;
+    }
+    // With windows, the kernels below serve the left-over windows only: a few long-running CTAs.
+    // They go to the second stream (of higher priority) and the window kernel runs beside them.
+    const bool forked = windows && wb.side != nullptr;
+    cudaStream_t ts = st;
+    if (forked) {
+        cudaEventRecord(wb.fork_event, st);
+        cudaStreamWaitEvent(wb.side, wb.fork_event, 0);
+        ts = wb.side;
+    }
     const unsigned blocks = (unsigned)((aa.nb + 255) / 256);  // one warp per 32 sorted positions
+    const unsigned low_blocks = (mp.Z - 1 + kLowWarps - 1) / kLowWarps;  // one warp per low slot
     if (mp.d % mp.Z != 0) {
-        det_apply_kernel<SIGN, MODE, true><<<blocks, 256, 0, st>>>(aa, K, V, bag_of);
-        if (mp.Z > 1) det_apply_low_kernel<SIGN, MODE, true><<<1, 128, 0, st>>>(aa, K, V, bag_of);
+        det_apply_kernel<SIGN, MODE, true><<<blocks, 256, 0, ts>>>(aa, K, V, bag_of);
+        if (mp.Z > 1)
+            det_apply_low_kernel<SIGN, MODE, true><<<low_blocks, 32 * kLowWarps, 0, ts>>>(aa, K, V, bag_of);
     } else {
-        det_apply_kernel<SIGN, MODE, false><<<blocks, 256, 0, st>>>(aa, K, V, bag_of);
+        det_apply_kernel<SIGN, MODE, false><<<blocks, 256, 0, ts>>>(aa, K, V, bag_of);
         if (!SIGN) {
             // the rounds the apply kernel handed over; a grid-stride loop over the list
             const unsigned lblocks = aa.long_cap < 148u * 8u ? aa.long_cap : 148u * 8u;
-            det_apply_long_kernel<MODE><<<lblocks, 32 * kLongWarps, 0, st>>>(aa, K, V);
+            det_apply_long_kernel<MODE><<<lblocks, 32 * kLongWarps, 0, ts>>>(aa, K, V);
         }
-        if (mp.Z > 1) det_apply_low_kernel<SIGN, MODE, false><<<1, 128, 0, st>>>(aa, K, V, bag_of);
+        if (mp.Z > 1)
+            det_apply_low_kernel<SIGN, MODE, false><<<low_blocks, 32 * kLowWarps, 0, ts>>>(aa, K, V, bag_of);
     }
+    if (forked) cudaEventRecord(wb.join_event, wb.side);
+    if (windows) {
+        const int vec4 = mp.Z % 4 == 0 && mp.d % 4 == 0 && ((uintptr_t)aa.grad_out & 15) == 0;
+        det_apply_window_kernel<MODE><<<wb.nwin, 256, 0, st>>>(aa, K, V, wb.lo_of, wb.hi_of, chunk, vec4);
+    }
+    if (forked) cudaStreamWaitEvent(st, wb.join_event, 0);
 }
 
 }  // namespace
@@ -866,7 +1135,7 @@ void launch_apply(const ApplyArgs& aa, const uint32_t* K, const uint32_t* V, con
 size_t det_workspace_bytes(const MapParams& mp, int64_t nbags, int64_t nnz, bool bags) {
     (void)nbags;
     const uint64_t nb = (uint64_t)nnz * mp.C;
-    return make_layout(nb, nnz, bags).total;
+    return make_layout(nb, nnz, bags, mp.m).total;
 }
 
 cudaError_t launch_backward_det(const Problem& pb, const float* grad_out, float* target, int mode,
@@ -876,7 +1145,7 @@ cudaError_t launch_backward_det(const Problem& pb, const float* grad_out, float*
     const MapParams& mp = pb.mp;
     const bool bags = pb.offsets != nullptr;
     const uint64_t nb = (uint64_t)pb.nnz * mp.C;
-    const Layout L = make_layout(nb, pb.nnz, bags);
+    const Layout L = make_layout(nb, pb.nnz, bags, mp.m);
     if (workspace == nullptr || workspace_bytes < L.total) return cudaErrorInvalidValue;
     // the payload of a block is a 32-bit position in grad_out
     if ((uint64_t)pb.nbags * mp.d > (1ull << 32)) return cudaErrorInvalidValue;
@@ -918,7 +1187,8 @@ cudaError_t launch_backward_det(const Problem& pb, const float* grad_out, float*
         sort_scan_kernel<<<kRadix, kSortThreads, 0, st>>>(counts, totals, sp.grid);
         sort_scatter_kernel<false><<<sp.grid, kSortThreads, 0, st>>>(kA, vA, kB, vB, counts, totals, nb,
                                                                     sp.tiles, shift, mask);
-        ApplyArgs ab{mp, grad_out, pb.indices, target, lr, nb, pb.status, AdamState{}, nullptr, nullptr, 0};
+        ApplyArgs ab{mp, grad_out, pb.indices, target, lr, nb, pb.status, AdamState{}, nullptr, nullptr, 0,
+                     nullptr, nullptr, 0};
         uint32_t log2Zp = 0;
         while ((1u << log2Zp) < mp.Z) ++log2Zp;
         const uint64_t groups = (nb + kBinnedPer - 1) / kBinnedPer;
@@ -950,15 +1220,19 @@ cudaError_t launch_backward_det(const Problem& pb, const float* grad_out, float*
     uint32_t* long_count = (uint32_t*)(ws + L.long_count);
     cudaMemsetAsync(long_count, 0, sizeof(uint32_t), st);
     ApplyArgs aa{mp, grad_out, pb.indices, target, lr, nb, pb.status, adam ? *adam : AdamState{},
-                 long_count, (LongWalk*)(ws + L.long_walks), L.long_cap};
+                 long_count, (LongWalk*)(ws + L.long_walks), L.long_cap, nullptr, nullptr, 0};
+    const WindowBuffers wb{(uint32_t*)(ws + L.bounds),
+                           (uint32_t*)(ws + L.bounds + align256(((size_t)L.nwin + 1) * sizeof(uint32_t))),
+                           (uint8_t*)(ws + L.win_left), L.nwin, L.win_log2,
+                           pb.side, pb.fork_event, pb.join_event};
     if (pb.sign) {
-        if (mode == 2) launch_apply<true, 2>(aa, kA, vA, bag_of, st);
-        else if (mode == 1) launch_apply<true, 1>(aa, kA, vA, bag_of, st);
-        else launch_apply<true, 0>(aa, kA, vA, bag_of, st);
+        if (mode == 2) launch_apply<true, 2>(aa, kA, vA, bag_of, wb, st);
+        else if (mode == 1) launch_apply<true, 1>(aa, kA, vA, bag_of, wb, st);
+        else launch_apply<true, 0>(aa, kA, vA, bag_of, wb, st);
     } else {
-        if (mode == 2) launch_apply<false, 2>(aa, kA, vA, bag_of, st);
-        else if (mode == 1) launch_apply<false, 1>(aa, kA, vA, bag_of, st);
-        else launch_apply<false, 0>(aa, kA, vA, bag_of, st);
+        if (mode == 2) launch_apply<false, 2>(aa, kA, vA, bag_of, wb, st);
+        else if (mode == 1) launch_apply<false, 1>(aa, kA, vA, bag_of, wb, st);
+        else launch_apply<false, 0>(aa, kA, vA, bag_of, wb, st);
     }
     return cudaGetLastError();
 }

@@ -18,6 +18,11 @@ struct Problem {
     int64_t nbags;           // batch * T
     int64_t nnz;
     int32_t* status;         // device status word or nullptr (validation off)
+    // deterministic backward: a second stream of higher priority with the two events that fork
+    // it from and join it to the caller's stream, or all nullptr (everything in the caller's)
+    cudaStream_t side = nullptr;
+    cudaEvent_t fork_event = nullptr;
+    cudaEvent_t join_event = nullptr;
 };
 
 // forward: out [nbags, d]
