@@ -281,6 +281,48 @@ def test_deterministic_is_bit_reproducible_and_order_sensitive_case():
             assert_bits_equal(r, can, "hot id deterministic")
 
 
+# Densely touched arrays take the slot-major kernel (one CTA per window of 256..2048 slots); the
+# cases span its branches: windows of every length, a ragged last window, blocks that wrap, ids
+# repeated so often that their windows go back to the position-tile and long-walk kernels while
+# the rest stay, windows whose blocks need several chunks of shared memory, block lengths that
+# are no power of two or no multiple of four, and a gradient buffer that is not 16-byte aligned.
+WINDOW_CASES = [
+    # d, Z, M, batch, tables/vocab, bags, id_dist
+    dict(d=64, Z=16, M=300_007, batch=1500, vocab_arg=(10**6, 10**6, 50_000), bag_rule=(6, 0, 20)),
+    dict(d=32, Z=32, M=2_100_003, batch=9000, vocab_arg=(10**6, 10**5, 10**6, 3000), num_tables=4),
+    dict(d=32, Z=32, M=2_100_003, batch=9000, vocab_arg=(10**6, 10**5, 10**6, 3000), num_tables=4,
+         id_dist="zipf1.05"),
+    dict(d=128, Z=128, M=700_001, batch=3000, vocab_arg=(10**5, 40, 10**6), id_dist="zipf1.05"),
+    dict(d=16, Z=16, M=4099, batch=6000, vocab_arg=(10**6, 10**6, 10**6)),
+    dict(d=48, Z=12, M=100_003, batch=2500, vocab_arg=(10**6, 10**6, 10**6)),
+    dict(d=48, Z=6, M=100_003, batch=2500, vocab_arg=(10**6, 10**6, 10**6)),
+    dict(d=8, Z=1, M=50_021, batch=4000, vocab_arg=(10**6, 10**6, 10**6), id_dist="zipf1.05"),
+    dict(d=64, Z=256, M=600_011, batch=5000, vocab_arg=(10**6, 10**6, 10**6)),
+]
+
+
+@pytest.mark.parametrize("case", WINDOW_CASES, ids=lambda k: f"d{k['d']}_Z{k['Z']}_M{k['M']}_{k.get('id_dist', 'uniform')}")
+def test_deterministic_window_apply(case):
+    w = small(**case)
+    with Case(w) as c:
+        nb = c.indices.numel() * ((w.d + min(w.Z, w.d) - 1) // min(w.Z, w.d))
+        assert nb * min(w.Z, w.d) * 2 >= w.M, "the case must touch the array densely"
+        g_h, g_d = _grad(c, 11)
+        can, touched = c.oracle.backward_canonical(g_h, c.indices_h, c.offsets_h, c.B)
+        assert_bits_equal(c.backward(g_d, "det").cpu().numpy(), can, "window apply, dense gradient")
+        # the same values from a buffer that starts 4 bytes off a 16-byte boundary
+        shifted = torch.empty(g_d.numel() + 1, dtype=torch.float32, device=c.dev)[1:]
+        shifted.copy_(g_d.reshape(-1))
+        assert shifted.data_ptr() % 16 == 4
+        assert_bits_equal(c.backward(shifted.view_as(g_d), "det").cpu().numpy(), can, "unaligned gradient")
+        # fused SGD: untouched slots keep their bits
+        before = c.array_h.copy()
+        c.backward(g_d, "det", sgd=True, lr=0.125)
+        want = before.copy()
+        orc.sgd_apply(want, can, touched, 0.125)
+        assert_bits_equal(c.array.cpu().numpy(), want, "window apply, SGD")
+
+
 def test_backward_empty_inputs():
     w = small(bag_rule=(2, 0, 5))
     with Case(w, batch=4) as c:
