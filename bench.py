@@ -310,15 +310,31 @@ def run_ours(args, w):
         zb = min(w.Z, w.d)
         bwd_launches = ((1 if bags else 0) + 1 + 3 * npass + 1 + (1 if w.d % zb == 0 else 0)
                         + (1 if zb > 1 else 0))
+        # a densely touched array: window bounds, window classes and the window kernel as well
+        terms = float(np.mean([len(b[0]) for b in batches])) * w.d
+        if w.d % zb == 0 and zb <= 128 and 2 * terms >= w.M:
+            bwd_launches += 3
+    # One training step hashes every id once: the forward leaves the block starts in the workspace
+    # and the sort-based backward takes them from there (rows of up to 128 elements; longer rows
+    # use a forward kernel that keeps nothing, and the key kernels then run inside the forward call).
+    share_keys = args.share_keys and ws is not None
+    if share_keys and w.d <= 128:
+        bwd_launches -= (1 if bags else 0) + 1
 
     def step(i, events=None):
         k = i % NB
         if events is not None:
             events[0].record()
-        robe.robe_forward(h, d_ids[k], d_offs[k], B, out)
+        if share_keys:
+            robe.robe_forward_keep(h, d_ids[k], d_offs[k], B, out, ws)
+        else:
+            robe.robe_forward(h, d_ids[k], d_offs[k], B, out)
         if events is not None:
             events[1].record()
-        robe.robe_backward(h, grad_out, d_ids[k], d_offs[k], B, dense, lr, ws)
+        if share_keys:
+            robe.robe_backward_kept(h, grad_out, d_ids[k], d_offs[k], B, dense, lr, ws)
+        else:
+            robe.robe_backward(h, grad_out, d_ids[k], d_offs[k], B, dense, lr, ws)
         if events is not None:
             events[2].record()
 
@@ -379,8 +395,12 @@ def run_ours(args, w):
             ev_in[b].record(s_in)
         s_comp.wait_event(ev_in[b])
         s_comp.wait_event(ev_out[b])     # the output buffer has been copied out
-        robe.robe_forward(h, ids_d, e_offs[b], B, e_out[b], stream=s_comp)
-        robe.robe_backward(h, e_grad[b], ids_d, e_offs[b], B, dense, lr, ws, stream=s_comp)
+        if share_keys:
+            robe.robe_forward_keep(h, ids_d, e_offs[b], B, e_out[b], ws, stream=s_comp)
+            robe.robe_backward_kept(h, e_grad[b], ids_d, e_offs[b], B, dense, lr, ws, stream=s_comp)
+        else:
+            robe.robe_forward(h, ids_d, e_offs[b], B, e_out[b], stream=s_comp)
+            robe.robe_backward(h, e_grad[b], ids_d, e_offs[b], B, dense, lr, ws, stream=s_comp)
         ev_comp[b].record(s_comp)
         with torch.cuda.stream(s_out):
             s_out.wait_event(ev_comp[b])
@@ -445,6 +465,8 @@ def run_ours(args, w):
         "config": {"workload": w.name, "num_tables": T, "d": d, "Z": w.Z, "M": w.M, "batch_per_gpu": B,
                    "ids_per_step_per_gpu": nnz_per_step, "ids": args.ids, "bags": bags, "backward": {"atomic": "atomic", "det": "deterministic", "binned": "binned atomic"}[args.backward] +
                    (", SGD fused" if dense is None else ", dense fp32 gradient"),
+                   "block_starts": ("hashed once per step: kept by the forward for the backward" if share_keys
+                                    else "hashed by the forward and again by the backward"),
                    "l2": l2_note,
                    "parallelism": f"dp{world} replicas, no collective"},
         "clocks": clocks,
@@ -486,6 +508,9 @@ def main():
                          "HBM and is touched several times per step, else plain atomic adds")
     ap.add_argument("--ids", default="int64", choices=["int64", "int32"], help="element type of the id arrays")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-share-keys", dest="share_keys", action="store_false",
+                    help="hash the ids in the backward again (robe_forward + robe_backward) instead of "
+                         "keeping the forward's block starts (robe_forward_keep + robe_backward_kept)")
     ap.add_argument("--batch", type=int, default=0,
                     help="samples per GPU instead of the workload's own batch (small profiler captures)")
     args = ap.parse_args()

@@ -174,6 +174,32 @@ int robe_backward(robe_handle_t h, const float* grad_out, const void* indices,
                   void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * robe_forward_keep / robe_backward_kept - the forward and backward of one training step on
+ * the same ids, sharing the hash work.  The block starts h(e, x_p, c) that the forward computes
+ * (Section 3.2) are what the binned and the deterministic backward sort by; robe_forward_keep
+ * is robe_forward that also stores them in `workspace`, and robe_backward_kept is
+ * robe_backward that takes them from there instead of hashing every id again.  The paper has
+ * no counterpart: it is a fusion across the two passes, results are those of robe_forward and
+ * robe_backward bit for bit (deterministic mode) or within the same bound (binned mode).
+ *   workspace  device pointer, 256-byte aligned, at least robe_backward_workspace_bytes(h,
+ *              batch, nnz) bytes; owned by the caller, who leaves it untouched between the two
+ *              calls.  The backward consumes what was kept: one robe_backward_kept per
+ *              robe_forward_keep.
+ *   The two calls get the same indices, offsets, batch and nnz, with the handle's sign,
+ *   index-type and backward-mode options unchanged in between; anything else is undefined
+ *   (but reads no memory outside the buffers named here).
+ * In atomic mode nothing is sorted: the two calls are then robe_forward and robe_backward, and
+ * workspace may be NULL.
+ * Errors: those of robe_forward and robe_backward; ROBE_ERR_UNSUPPORTED and
+ * ROBE_ERR_WORKSPACE already from robe_forward_keep.
+ */
+int robe_forward_keep(robe_handle_t h, const void* indices, const int64_t* offsets, int64_t batch,
+                      int64_t nnz, float* out, void* workspace, size_t workspace_bytes, void* stream);
+int robe_backward_kept(robe_handle_t h, const float* grad_out, const void* indices,
+                       const int64_t* offsets, int64_t batch, int64_t nnz, float* grad_array, float lr,
+                       void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * robe_backward_adam - deterministic backward with the Adam step fused in (the paper trains
  * five of its six Criteo-Kaggle models with Adam, Section 5; the update is Algorithm 1 of
  * Kingma & Ba, "Adam: a method for stochastic optimization").  For every array slot j that

@@ -46,6 +46,7 @@ EXPORTS = [
     "robe_get_hash_constants", "robe_forward", "robe_backward_workspace_bytes", "robe_backward",
     "robe_set_status_word", "robe_last_device_status", "robe_status_string",
     "robe_backward_deterministic_static", "robe_backward_adam",
+    "robe_forward_keep", "robe_backward_kept",
 ]
 
 if not os.path.exists(LIB_PATH):
@@ -62,9 +63,11 @@ _lib.robe_set_option.argtypes = [_vp, C.c_int, _i64]
 _lib.robe_attach_array.argtypes = [_vp, _vp, C.c_int]
 _lib.robe_get_hash_constants.argtypes = [_vp, C.POINTER(_u64)]
 _lib.robe_forward.argtypes = [_vp, _vp, _vp, _i64, _i64, _vp, _vp]
+_lib.robe_forward_keep.argtypes = [_vp, _vp, _vp, _i64, _i64, _vp, _vp, C.c_size_t, _vp]
 _lib.robe_backward_workspace_bytes.argtypes = [_vp, _i64, _i64]
 _lib.robe_backward_workspace_bytes.restype = C.c_size_t
 _lib.robe_backward.argtypes = [_vp, _vp, _vp, _vp, _i64, _i64, _vp, C.c_float, _vp, C.c_size_t, _vp]
+_lib.robe_backward_kept.argtypes = list(_lib.robe_backward.argtypes)
 _lib.robe_backward_deterministic_static.argtypes = [_vp, _vp, _vp, _vp, _i64, _i64, _vp, C.c_float, _vp]
 _lib.robe_backward_adam.argtypes = [_vp, _vp, _vp, _vp, _i64, _i64, _vp, _vp, C.c_float, C.c_float,
                                     C.c_float, C.c_float, _i64, _vp, C.c_size_t, _vp]
@@ -164,6 +167,15 @@ def robe_forward(h, indices, offsets, batch: int, out, stream=None) -> None:
                              _stream_ptr(stream)), "robe_forward")
 
 
+def robe_forward_keep(h, indices, offsets, batch: int, out, workspace, stream=None) -> None:
+    """robe_forward that also leaves the block starts in `workspace` for robe_backward_kept."""
+    _state_index_type(h, indices)
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(_lib.robe_forward_keep(h, _ids_ptr(indices), _dev_ptr(offsets, torch.int64),
+                                  batch, indices.numel(), _dev_ptr(out, torch.float32),
+                                  _dev_ptr(workspace), ws_bytes, _stream_ptr(stream)), "robe_forward_keep")
+
+
 def robe_backward_workspace_bytes(h, batch: int, nnz: int) -> int:
     return int(_lib.robe_backward_workspace_bytes(h, batch, nnz))
 
@@ -176,6 +188,17 @@ def robe_backward(h, grad_out, indices, offsets, batch: int, grad_array=None, lr
                               _dev_ptr(offsets, torch.int64), batch, indices.numel(),
                               _dev_ptr(grad_array, torch.float32), lr, _dev_ptr(workspace),
                               ws_bytes, _stream_ptr(stream)), "robe_backward")
+
+
+def robe_backward_kept(h, grad_out, indices, offsets, batch: int, grad_array=None, lr: float = 0.0,
+                       workspace=None, stream=None) -> None:
+    """robe_backward on the block starts that robe_forward_keep left in `workspace`."""
+    _state_index_type(h, indices)
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(_lib.robe_backward_kept(h, _dev_ptr(grad_out, torch.float32), _ids_ptr(indices),
+                                   _dev_ptr(offsets, torch.int64), batch, indices.numel(),
+                                   _dev_ptr(grad_array, torch.float32), lr, _dev_ptr(workspace),
+                                   ws_bytes, _stream_ptr(stream)), "robe_backward_kept")
 
 
 def robe_backward_deterministic_static(h, grad_out, indices, offsets, batch: int, grad_array=None,

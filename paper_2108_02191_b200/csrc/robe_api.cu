@@ -292,6 +292,30 @@ int robe_forward(robe_handle_t h, const void* indices, const int64_t* offsets, i
     return ROBE_OK;
 }
 
+int robe_forward_keep(robe_handle_t h, const void* indices, const int64_t* offsets, int64_t batch,
+                      int64_t nnz, float* out, void* workspace, size_t workspace_bytes, void* stream) {
+    if (h != nullptr && h->bwd_mode == ROBE_BWD_ATOMIC)  // that backward sorts nothing
+        return robe_forward(h, indices, offsets, batch, nnz, out, stream);
+    if (!check_sizes(h, indices, offsets, batch, nnz)) return ROBE_ERR_INVALID_ARG;
+    if (batch > 0 && out == nullptr) return ROBE_ERR_INVALID_ARG;
+    if (h->array == nullptr) return ROBE_ERR_NO_ARRAY;
+    if (h->validate && h->status_word == nullptr) return ROBE_ERR_INVALID_ARG;
+    const Problem pb = make_problem(h, indices, offsets, batch, nnz);
+    if (!sorted_path_fits(h, pb)) return ROBE_ERR_UNSUPPORTED;
+    const size_t need = det_workspace_bytes(h->mp, pb.nbags, nnz, offsets != nullptr);
+    if (nnz > 0 && (workspace == nullptr || workspace_bytes < need)) return ROBE_ERR_WORKSPACE;
+    if (((uintptr_t)workspace & 255u) != 0) return ROBE_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (launch_validate(pb, st) != cudaSuccess) return ROBE_ERR_CUDA;
+    uint32_t *keys = nullptr, *vals = nullptr;
+    if (nnz > 0 && batch > 0) block_key_buffers(pb, workspace, &keys, &vals);
+    bool kept = false;
+    if (launch_forward(pb, out, h->fwd_variant, st, keys, vals, &kept) != cudaSuccess) return ROBE_ERR_CUDA;
+    // a forward kernel that keeps nothing (rows longer than 128): the backward's own key kernels
+    if (!kept && launch_block_keys(pb, workspace, workspace_bytes, st) != cudaSuccess) return ROBE_ERR_CUDA;
+    return ROBE_OK;
+}
+
 size_t robe_backward_workspace_bytes(robe_handle_t h, int64_t batch, int64_t nnz) {
     if (h == nullptr || batch < 0 || nnz < 0) return 0;
     if (h->bwd_mode == ROBE_BWD_ATOMIC) return 0;
@@ -299,9 +323,9 @@ size_t robe_backward_workspace_bytes(robe_handle_t h, int64_t batch, int64_t nnz
     return det_workspace_bytes(h->mp, batch * (int64_t)h->T, nnz, true);
 }
 
-int robe_backward(robe_handle_t h, const float* grad_out, const void* indices,
-                  const int64_t* offsets, int64_t batch, int64_t nnz, float* grad_array, float lr,
-                  void* workspace, size_t workspace_bytes, void* stream) {
+static int backward_any(robe_handle_t h, const float* grad_out, const void* indices,
+                        const int64_t* offsets, int64_t batch, int64_t nnz, float* grad_array, float lr,
+                        void* workspace, size_t workspace_bytes, void* stream, bool keys_kept) {
     if (!check_sizes(h, indices, offsets, batch, nnz)) return ROBE_ERR_INVALID_ARG;
     if (batch > 0 && grad_out == nullptr) return ROBE_ERR_INVALID_ARG;
     if (h->validate && h->status_word == nullptr) return ROBE_ERR_INVALID_ARG;
@@ -330,9 +354,23 @@ int robe_backward(robe_handle_t h, const float* grad_out, const void* indices,
     if (!binned) lend_side_stream(h, pb);
     if (launch_backward_det(pb, grad_out, target, binned ? 3 : (sgd ? 1 : 0),
                             binned ? (sgd ? -lr : 1.0f) : lr, nullptr, workspace, workspace_bytes,
-                            st) != cudaSuccess)
+                            st, keys_kept) != cudaSuccess)
         return ROBE_ERR_CUDA;
     return ROBE_OK;
+}
+
+int robe_backward(robe_handle_t h, const float* grad_out, const void* indices,
+                  const int64_t* offsets, int64_t batch, int64_t nnz, float* grad_array, float lr,
+                  void* workspace, size_t workspace_bytes, void* stream) {
+    return backward_any(h, grad_out, indices, offsets, batch, nnz, grad_array, lr, workspace,
+                        workspace_bytes, stream, false);
+}
+
+int robe_backward_kept(robe_handle_t h, const float* grad_out, const void* indices,
+                       const int64_t* offsets, int64_t batch, int64_t nnz, float* grad_array, float lr,
+                       void* workspace, size_t workspace_bytes, void* stream) {
+    return backward_any(h, grad_out, indices, offsets, batch, nnz, grad_array, lr, workspace,
+                        workspace_bytes, stream, true);
 }
 
 // Device address of robe_static_scratch on the current device, looked up once per device.

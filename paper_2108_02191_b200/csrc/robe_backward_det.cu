@@ -1138,9 +1138,51 @@ size_t det_workspace_bytes(const MapParams& mp, int64_t nbags, int64_t nnz, bool
     return make_layout(nb, nnz, bags, mp.m).total;
 }
 
+void block_key_buffers(const Problem& pb, void* workspace, uint32_t** keys, uint32_t** vals) {
+    const uint64_t nb = (uint64_t)pb.nnz * pb.mp.C;
+    const Layout L = make_layout(nb, pb.nnz, pb.offsets != nullptr, pb.mp.m);
+    *keys = (uint32_t*)((char*)workspace + L.keysA);
+    *vals = (uint32_t*)((char*)workspace + L.valsA);
+}
+
+// bag_of (pooled input) into the workspace
+static void launch_bag_of(const Problem& pb, const Layout& L, char* ws, cudaStream_t st) {
+    uint32_t* bag_of = (uint32_t*)(ws + L.bag_of);
+    KeyArgs ka{pb.mp, pb.indices, pb.offsets, pb.nbags, pb.nnz, pb.status};
+    // positions that malformed offsets leave uncovered fall back to bag 0 (memory-safe)
+    cudaMemsetAsync(bag_of, 0, (size_t)pb.nnz * sizeof(uint32_t), st);
+    det_bag_of_kernel<<<(unsigned)((pb.nbags + 7) / 8), 256, 0, st>>>(ka, bag_of);
+}
+
+cudaError_t launch_block_keys(const Problem& pb, void* workspace, size_t workspace_bytes,
+                              cudaStream_t st) {
+    if (pb.nnz == 0 || pb.nbags == 0) return cudaSuccess;
+    const MapParams& mp = pb.mp;
+    const bool bags = pb.offsets != nullptr;
+    const uint64_t nb = (uint64_t)pb.nnz * mp.C;
+    const Layout L = make_layout(nb, pb.nnz, bags, mp.m);
+    if (workspace == nullptr || workspace_bytes < L.total) return cudaErrorInvalidValue;
+    char* ws = (char*)workspace;
+    uint32_t* kA = (uint32_t*)(ws + L.keysA);
+    uint32_t* vA = (uint32_t*)(ws + L.valsA);
+    uint32_t* bag_of = bags ? (uint32_t*)(ws + L.bag_of) : nullptr;
+    KeyArgs ka{mp, pb.indices, pb.offsets, pb.nbags, pb.nnz, pb.status};
+    if (bags) launch_bag_of(pb, L, ws, st);
+    if (mp.C <= 8) {
+        const unsigned kb = (unsigned)((pb.nnz + 255) / 256);
+        if (pb.sign) det_keys_kernel<true><<<kb, 256, 0, st>>>(ka, bag_of, kA, vA);
+        else det_keys_kernel<false><<<kb, 256, 0, st>>>(ka, bag_of, kA, vA);
+    } else {
+        const unsigned kb = (unsigned)((nb + 255) / 256);
+        if (pb.sign) det_keys_by_block_kernel<true><<<kb, 256, 0, st>>>(ka, bag_of, kA, vA, nb);
+        else det_keys_by_block_kernel<false><<<kb, 256, 0, st>>>(ka, bag_of, kA, vA, nb);
+    }
+    return cudaGetLastError();
+}
+
 cudaError_t launch_backward_det(const Problem& pb, const float* grad_out, float* target, int mode,
                                 float lr, const AdamState* adam, void* workspace,
-                                size_t workspace_bytes, cudaStream_t st) {
+                                size_t workspace_bytes, cudaStream_t st, bool keys_kept) {
     if (pb.nnz == 0 || pb.nbags == 0) return cudaSuccess;
     const MapParams& mp = pb.mp;
     const bool bags = pb.offsets != nullptr;
@@ -1158,20 +1200,11 @@ cudaError_t launch_backward_det(const Problem& pb, const float* grad_out, float*
     uint32_t* counts = (uint32_t*)(ws + L.counts);
     uint32_t* totals = (uint32_t*)(ws + L.totals);
 
-    KeyArgs ka{mp, pb.indices, pb.offsets, pb.nbags, pb.nnz, pb.status};
-    if (bags) {
-        // positions that malformed offsets leave uncovered fall back to bag 0 (memory-safe)
-        cudaMemsetAsync(bag_of, 0, (size_t)pb.nnz * sizeof(uint32_t), st);
-        det_bag_of_kernel<<<(unsigned)((pb.nbags + 7) / 8), 256, 0, st>>>(ka, bag_of);
-    }
-    if (mp.C <= 8) {
-        const unsigned kb = (unsigned)((pb.nnz + 255) / 256);
-        if (pb.sign) det_keys_kernel<true><<<kb, 256, 0, st>>>(ka, bag_of, kA, vA);
-        else det_keys_kernel<false><<<kb, 256, 0, st>>>(ka, bag_of, kA, vA);
-    } else {
-        const unsigned kb = (unsigned)((nb + 255) / 256);
-        if (pb.sign) det_keys_by_block_kernel<true><<<kb, 256, 0, st>>>(ka, bag_of, kA, vA, nb);
-        else det_keys_by_block_kernel<false><<<kb, 256, 0, st>>>(ka, bag_of, kA, vA, nb);
+    if (!keys_kept) {
+        const cudaError_t err = launch_block_keys(pb, workspace, workspace_bytes, st);
+        if (err != cudaSuccess) return err;
+    } else if (bags && pb.sign) {
+        launch_bag_of(pb, L, ws, st);  // the signed terms look the id's bag up again
     }
 
     const SortPlan sp = make_plan(nb);

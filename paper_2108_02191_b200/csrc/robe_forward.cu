@@ -22,6 +22,8 @@ struct FwdArgs {
     int64_t nbags;
     int64_t nnz;
     const int32_t* status;
+    uint32_t* keep_keys;  // block starts and payloads kept for the backward, or nullptr
+    uint32_t* keep_vals;
 };
 
 template <int DT, bool SIGN>
@@ -163,6 +165,16 @@ fwd_staged_kernel(FwdArgs a, uint32_t ids_per_batch, uint32_t cmagic) {
         hi = lo + ids_per_batch < a.nbags ? lo + ids_per_batch : a.nbags;
     }
 
+    if (BAGS && a.keep_keys != nullptr) {
+        // id positions before the first bag or after the last one (offsets that break the
+        // contract) get block start 0 and payload 0, so that the backward reads nothing stale
+        const int64_t C = (int64_t)mp.C;
+        if (warp == 0)
+            for (int64_t q = lane; q < lo * C; q += 32) a.keep_keys[q] = a.keep_vals[q] = 0;
+        if (warp == a.nbags - 1)
+            for (int64_t q = hi * C + lane; q < a.nnz * C; q += 32) a.keep_keys[q] = a.keep_vals[q] = 0;
+    }
+
     // per-lane constants of the gather: element i = lane + 32u, its in-block offset, and the
     // column of the staging area that holds the starts of its chunk
     uint32_t off[EPL];
@@ -189,7 +201,8 @@ fwd_staged_kernel(FwdArgs a, uint32_t ids_per_batch, uint32_t cmagic) {
         const uint32_t cnt = (uint32_t)((hi - p0) < (int64_t)ids_per_batch ? (hi - p0)
                                                                             : (int64_t)ids_per_batch);
         const bool wraps = stage_batch<SIGN, BAGS>(sm, mp, a.indices, p0, cnt, ids_per_batch, tterm,
-                                                   gterm, cmagic, w, lane);
+                                                   gterm, cmagic, w, lane,
+                                                   KeepBlocks{a.keep_keys, a.keep_vals, (uint64_t)warp});
         if (wraps)
             gather_batch<EPL, DT, SIGN, BAGS, U, true>(a, col, off, live, gbase_s, cnt, p0, lane, acc);
         else
@@ -247,14 +260,18 @@ static void launch_staged_epl(const FwdArgs& a, bool bags, bool sign, cudaStream
         launch_staged_flags<4, DT>(a, bags, sign, st);
 }
 
-cudaError_t launch_forward(const Problem& pb, float* out, int variant, cudaStream_t st) {
+cudaError_t launch_forward(const Problem& pb, float* out, int variant, cudaStream_t st,
+                           uint32_t* keep_keys, uint32_t* keep_vals, bool* kept) {
+    if (kept != nullptr) *kept = false;
     if (pb.nbags == 0) return cudaSuccess;
-    FwdArgs a{pb.mp, pb.array, pb.indices, pb.offsets, out, pb.nbags, pb.nnz, pb.status};
+    FwdArgs a{pb.mp, pb.array, pb.indices, pb.offsets, out, pb.nbags, pb.nnz, pb.status, keep_keys,
+              keep_vals};
     const bool bags = pb.offsets != nullptr;
     const bool warp_ok = pb.mp.d <= 128;
     if (variant == 2 && !warp_ok) return cudaErrorInvalidValue;
     const bool use_warp = variant == 2 || (variant == 0 && warp_ok);
     if (use_warp) {
+        if (kept != nullptr) *kept = keep_keys != nullptr;  // (the direct kernel keeps nothing)
         if (pb.dtype == 0) launch_staged_epl<0>(a, bags, pb.sign != 0, st);
         else launch_staged_epl<1>(a, bags, pb.sign != 0, st);
     } else {

@@ -58,6 +58,16 @@ __device__ __forceinline__ void stage_init(StageSmem& sm, const MapParams& mp) {
     __syncthreads();
 }
 
+// Where the hash phase also leaves the block starts for a later sort-based backward of the same
+// ids: keys[q] = h(e, x_p, c) and vals[q] for block q = p*C + c, vals[q] = q when the sign hash is
+// on, else the position bag*d + c*Z of the block's first gradient element.  keys == nullptr: not
+// kept.  `bag` is the warp's bag in pooled mode (one-hot: row p is bag p).
+struct KeepBlocks {
+    uint32_t* keys;
+    uint32_t* vals;
+    uint64_t bag;
+};
+
 // Hash phase of one batch of cnt ids starting at position p0 (warp-collective).
 //   step 1: one id per lane          -> base_s[t] = (A e + B x + D) mod P  (and the sign base)
 //   step 2: one (id, chunk) per lane -> start_s[c*stride + t] = h(e, x, c)
@@ -69,7 +79,8 @@ template <bool SIGN, bool BAGS>
 __device__ __forceinline__ bool stage_batch(StageSmem& sm, const MapParams& mp,
                                             const IdList& indices, int64_t p0, uint32_t cnt,
                                             uint32_t stride, uint64_t tterm, uint64_t gterm,
-                                            uint32_t cmagic, uint32_t w, uint32_t lane) {
+                                            uint32_t cmagic, uint32_t w, uint32_t lane,
+                                            const KeepBlocks keep = KeepBlocks{nullptr, nullptr, 0}) {
     uint64_t* base_s = sm.base[w];
     uint64_t* gbase_s = base_s + kStageIds / 2;
     uint32_t* start_s = sm.start[w];
@@ -103,6 +114,12 @@ __device__ __forceinline__ bool stage_batch(StageSmem& sm, const MapParams& mp,
         }
         start_s[c * stride + idl] = s;
         wraps |= s > last_fit;
+        if (keep.keys != nullptr) {  // consecutive lanes, consecutive words
+            const uint64_t q = (uint64_t)p0 * mp.C + t;
+            const uint64_t bag = BAGS ? keep.bag : (uint64_t)p0 + idl;
+            keep.keys[q] = s;
+            keep.vals[q] = SIGN ? (uint32_t)q : (uint32_t)(bag * mp.d + c * mp.Z);
+        }
     }
     const bool any = __any_sync(0xFFFFFFFFu, wraps);
     __syncwarp();  // the stores above are visible to the whole warp from here on

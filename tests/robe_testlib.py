@@ -77,6 +77,25 @@ class Case:
         torch.cuda.synchronize()
         return grad_array
 
+    def step_sharing_keys(self, grad_out: torch.Tensor, mode, sgd=False, lr=0.0):
+        """robe_forward_keep then robe_backward_kept on the same workspace: (out, dense gradient
+        or None)."""
+        robe.robe_set_option(self.h, robe.ROBE_OPT_BWD_MODE,
+                             {"atomic": robe.ROBE_BWD_ATOMIC, "det": robe.ROBE_BWD_DETERMINISTIC,
+                              "binned": robe.ROBE_BWD_BINNED}[mode])
+        robe.robe_set_option(self.h, robe.ROBE_OPT_FWD_KERNEL, 0)
+        robe.robe_set_option(self.h, robe.ROBE_OPT_BWD_KERNEL, 0)
+        ws = None
+        nbytes = robe.robe_backward_workspace_bytes(self.h, self.B, self.indices.numel())
+        if nbytes:  # stale contents from an earlier call must not matter
+            ws = torch.full((nbytes,), 0xA5, dtype=torch.uint8, device=self.dev)
+        out = torch.full((self.B, self.T, self.w.d), float("nan"), dtype=torch.float32, device=self.dev)
+        robe.robe_forward_keep(self.h, self.indices, self.offsets, self.B, out, ws)
+        grad_array = None if sgd else torch.zeros(self.w.M, dtype=torch.float32, device=self.dev)
+        robe.robe_backward_kept(self.h, grad_out, self.indices, self.offsets, self.B, grad_array, lr, ws)
+        torch.cuda.synchronize()
+        return out, grad_array
+
     # ---- oracle side ----------------------------------------------------------------
     def oracle_forward(self):
         return self.oracle.forward(self.array_h, self.indices_h, self.offsets_h, self.B)

@@ -323,6 +323,59 @@ def test_deterministic_window_apply(case):
         assert_bits_equal(c.array.cpu().numpy(), want, "window apply, SGD")
 
 
+# robe_forward_keep + robe_backward_kept: one hash of every id per training step.  The pair must
+# give what robe_forward and robe_backward give: the forward bit for bit, the deterministic
+# backward bit for bit, the binned and atomic ones within the atomic bound.  Shapes: rows of every
+# kernel class (up to 32, 64, 128 elements and longer, where the forward kernel keeps nothing),
+# ragged last blocks, rows clubbed into one block, one-hot and pooled input with empty bags.
+KEEP_SHAPES = [(16, 4, 4096), (64, 16, 70), (100, 32, 1013), (128, 128, 1280), (12, 5, 64), (48, 3, 49),
+               (130, 2, 1000), (200, 64, 777), (16, 64, 1000), (1, 1, 1), (32, 32, 100_003)]
+
+
+@pytest.mark.parametrize("bags", [None, (3, 0, 9)])
+@pytest.mark.parametrize("d,Z,M", KEEP_SHAPES)
+def test_step_sharing_block_starts(d, Z, M, bags):
+    w = small(d=d, Z=Z, M=M, bag_rule=bags, batch=61)
+    for sign in (False, True):
+        with Case(w, sign=sign) as c:
+            g_h, g_d = _grad(c, 21)
+            want_out = c.oracle_forward()
+            delta64, l1 = c.oracle.backward_f64(g_h, c.indices_h, c.offsets_h, c.B)
+            can, touched = c.oracle.backward_canonical(g_h, c.indices_h, c.offsets_h, c.B)
+            out, det = c.step_sharing_keys(g_d, "det")
+            assert_bits_equal(out.cpu().numpy(), want_out, "forward that keeps")
+            assert_bits_equal(det.cpu().numpy(), can, f"deterministic on kept starts d={d} Z={Z} sign={sign}")
+            out, binned = c.step_sharing_keys(g_d, "binned")
+            assert_bits_equal(out.cpu().numpy(), want_out, "forward that keeps")
+            assert_within_l1(binned.cpu().numpy(), delta64, l1, what=f"binned on kept starts d={d} Z={Z}")
+            out, atomic = c.step_sharing_keys(g_d, "atomic")  # nothing to keep: plain calls
+            assert_within_l1(atomic.cpu().numpy(), delta64, l1, what="atomic through the keep calls")
+            # fused SGD through the pair
+            before = c.array_h.copy()
+            c.step_sharing_keys(g_d, "det", sgd=True, lr=0.25)
+            want = before.copy()
+            orc.sgd_apply(want, can, touched, 0.25)
+            assert_bits_equal(c.array.cpu().numpy(), want, "SGD on kept starts")
+
+
+def test_step_sharing_block_starts_int32_ids_and_workspace_check():
+    w = small(d=64, Z=16, M=50_021, bag_rule=(4, 0, 12), batch=300)
+    with Case(w) as c:
+        g_h, g_d = _grad(c, 22)
+        can, _ = c.oracle.backward_canonical(g_h, c.indices_h, c.offsets_h, c.B)
+        c.indices = c.indices.to(torch.int32)
+        _, det = c.step_sharing_keys(g_d, "det")
+        assert_bits_equal(det.cpu().numpy(), can, "kept starts, int32 ids")
+        out = torch.empty(c.B, c.T, w.d, device=c.dev)
+        small_ws = torch.empty(256, dtype=torch.uint8, device=c.dev)
+        with pytest.raises(robe.RobeError) as ei:
+            robe.robe_forward_keep(c.h, c.indices, c.offsets, c.B, out, small_ws)
+        assert ei.value.status == robe.ROBE_ERR_WORKSPACE
+        with pytest.raises(robe.RobeError) as ei:
+            robe.robe_forward_keep(c.h, c.indices, c.offsets, c.B, out, None)
+        assert ei.value.status == robe.ROBE_ERR_WORKSPACE
+
+
 def test_backward_empty_inputs():
     w = small(bag_rule=(2, 0, 5))
     with Case(w, batch=4) as c:
