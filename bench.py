@@ -39,10 +39,12 @@ UNIT = "ids/s"
 # full-size default workload (summaries of those captures are kept under profiles/); None = not
 # captured for that workload or backward variant.
 NCU_TRAFFIC_BYTES = {
-    ("cfg4_multihot", "atomic"): {"forward": 4_197_885_696, "backward": 7_509_030_400},
-    ("cfg4_multihot", "det"): {"forward": 4_197_885_696, "backward": None},
-    # binned: the six kernels of the backward together
-    ("cfg4_multihot", "binned"): {"forward": 4196867254, "backward": 5141565238},
+    # (workload, backward variant, block starts shared between forward and backward)
+    ("cfg4_multihot", "atomic", False): {"forward": 4_197_885_696, "backward": 7_509_030_400},
+    # the forward also writes the block starts; backward = count, scan, scatter, binned_apply
+    ("cfg4_multihot", "binned", True): {"forward": 4_432_388_498, "backward": 4_824_968_027},
+    # backward = four sort passes, window bounds and classes, the four apply kernels
+    ("cfg4_multihot", "det", True): {"forward": 4_432_471_808, "backward": 7_192_080_237},
 }
 
 
@@ -441,8 +443,10 @@ def run_ours(args, w):
     bwd_label = {"atomic": "backward (bwd_atomic_staged_kernel)",
                  "binned": "backward (keys, count, scan, scatter, binned_apply kernels together)",
                  "det": "backward (keys, sort passes, apply kernels together)"}[args.backward]
+    if share_keys:
+        bwd_label = bwd_label.replace("(keys, ", "(")
     dom_bytes, dom_ms = (bwd_bytes, bwd_ms) if dominant == "backward" else (fwd_bytes, fwd_ms)
-    traffic = NCU_TRAFFIC_BYTES.get((w.name, args.backward), {}) if args.ids == "int64" else {}
+    traffic = NCU_TRAFFIC_BYTES.get((w.name, args.backward, bool(share_keys)), {}) if args.ids == "int64" else {}
 
     def roof(nbytes, ms, which):
         ach = nbytes / (ms * 1e-3) / 1e9
