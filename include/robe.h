@@ -186,8 +186,9 @@ int robe_backward(robe_handle_t h, const float* grad_out, const void* indices,
  *              calls.  The backward consumes what was kept: one robe_backward_kept per
  *              robe_forward_keep.
  *   The two calls get the same indices, offsets, batch and nnz, with the handle's sign,
- *   index-type and backward-mode options unchanged in between; anything else is undefined
- *   (but reads no memory outside the buffers named here).
+ *   index-type and backward-mode options unchanged in between.  The backward trusts what the
+ *   workspace holds: after anything else (other sizes, a workspace written to in between, no
+ *   robe_forward_keep before) its behaviour is undefined, as for a wrong pointer.
  * In atomic mode nothing is sorted: the two calls are then robe_forward and robe_backward, and
  * workspace may be NULL.
  * Errors: those of robe_forward and robe_backward; ROBE_ERR_UNSUPPORTED and

@@ -647,7 +647,9 @@ constexpr int kBoundsPer = 8;  // sorted positions per thread
 
 __global__ void __launch_bounds__(256)
 det_bounds_kernel(const uint32_t* __restrict__ K, uint64_t nb, uint32_t* lo_of, uint32_t* hi_of,
-                  uint32_t nwin, uint32_t win_log2, uint32_t Z) {
+                  uint32_t nwin, uint32_t win_log2, uint32_t Z, const int32_t* status) {
+    // after a failed input check K was not written: the loops below rely on sorted keys
+    if (status != nullptr && *status != 0) return;
     const uint64_t i0 = ((uint64_t)blockIdx.x * 256 + threadIdx.x) * kBoundsPer;
     if (i0 > nb) return;
     uint64_t k[kBoundsPer + 1];  // k[t] = key before position i0 + t
@@ -673,7 +675,9 @@ det_bounds_kernel(const uint32_t* __restrict__ K, uint64_t nb, uint32_t* lo_of, 
 // slots of such windows, the window kernel all others.  *any_left counts them.
 __global__ void __launch_bounds__(256)
 det_window_classify_kernel(const uint32_t* __restrict__ lo_of, const uint32_t* __restrict__ hi_of,
-                           uint32_t nwin, uint32_t n_max, uint8_t* win_left, uint32_t* any_left) {
+                           uint32_t nwin, uint32_t n_max, uint8_t* win_left, uint32_t* any_left,
+                           const int32_t* status) {
+    if (status != nullptr && *status != 0) return;
     const uint32_t b = blockIdx.x * 256 + threadIdx.x;
     const bool left = b < nwin && hi_of[b + 1] - lo_of[b] > n_max;
     if (b < nwin) win_left[b] = left ? 1 : 0;
@@ -1086,13 +1090,13 @@ void launch_apply(ApplyArgs aa, const uint32_t* K, const uint32_t* V, const uint
         cudaMemsetAsync(any_left, 0, sizeof(uint32_t), st);
         const uint64_t per_cta = 256ull * kBoundsPer;
         det_bounds_kernel<<<(unsigned)(aa.nb / per_cta + 1), 256, 0, st>>>(K, aa.nb, wb.lo_of, wb.hi_of,
-                                                                          wb.nwin, wb.win_log2, mp.Z);
+                                                                          wb.nwin, wb.win_log2, mp.Z, aa.status);
         // a window reached by many times the average number of blocks holds an often repeated id
         const uint64_t mean = (((uint64_t)1 << wb.win_log2) + mp.Z) * aa.nb / mp.m + 1;
         const uint64_t n_max = mean * 4 > 512 ? mean * 4 : 512;
         det_window_classify_kernel<<<(wb.nwin + 255) / 256, 256, 0, st>>>(
             wb.lo_of, wb.hi_of, wb.nwin, (uint32_t)(n_max < 0xFFFFFFFFull ? n_max : 0xFFFFFFFFull), wb.left,
-            any_left);
+            any_left, aa.status);
         aa.win_left = wb.left;
         aa.any_left = any_left;
         aa.win_log2 = wb.win_log2;
