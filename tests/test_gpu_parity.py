@@ -468,6 +468,13 @@ def test_cfg4_forward_backward_full_size():
         assert_within_l1(c.array.cpu().numpy(), before.astype(np.float64) - 0.5 * delta64,
                          0.5 * l1 + np.abs(before), what="cfg4 binned sgd")
         c.array.copy_(torch.from_numpy(before))
+        # the step as the benchmark runs it: the forward keeps its block starts for the binned backward
+        out, gk = c.step_sharing_keys(g_d, "binned")
+        bags = _sample_bags(c.nbags, 20000, 2)
+        assert_bits_equal(out.reshape(c.nbags, w.d)[torch.from_numpy(bags).to(c.dev)].cpu().numpy(),
+                          c.oracle_forward_bags(bags), "cfg4 forward that keeps")
+        assert_within_l1(gk.cpu().numpy(), delta64, l1, what="cfg4 binned on kept starts")
+        del out, gk
         # gradient mass is conserved (holds at any size)
         lengths = np.diff(c.offsets_h)
         mass = float((lengths * g_h.astype(np.float64).reshape(c.nbags, -1).sum(axis=1)).sum())
@@ -480,6 +487,8 @@ def test_cfg4_forward_backward_full_size():
         assert_bits_equal(det[:100_000], can0, "cfg4 det low slots")
         canl, _ = c.oracle.backward_canonical(g_h, c.indices_h, c.offsets_h, c.B, j0=w.M - 100_000, jn=100_000)
         assert_bits_equal(det[w.M - 100_000:], canl, "cfg4 det high slots")
+        _, detk = c.step_sharing_keys(g_d, "det")
+        assert_bits_equal(detk.cpu().numpy(), det, "cfg4 det on kept starts")
 
 
 @pytest.mark.parametrize("M,Z,dtype", [
