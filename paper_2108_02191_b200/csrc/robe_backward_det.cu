@@ -382,7 +382,7 @@ constexpr uint32_t kRing = 128;
 // window apply: the array is cut into windows of 2^8 .. 2^11 slots, one CTA each
 constexpr uint32_t kWinLog2Min = 8, kWinLog2Max = 11;
 constexpr uint32_t kWinMaxZ = 128;        // longest block the window kernel takes
-constexpr uint32_t kWinEnt = 1024;        // sorted blocks per chunk, at most
+constexpr uint32_t kWinEnt = 512;         // sorted blocks per chunk, at most
 constexpr uint32_t kWinStage = 6144;      // gradient elements per chunk, at most (>= kWinMaxZ)
 constexpr uint32_t kNoKey = 0xFFFFFFFFu;  // above every slot number (m + d <= 2^32)
 
@@ -685,70 +685,56 @@ det_window_classify_kernel(const uint32_t* __restrict__ lo_of, const uint32_t* _
     if ((threadIdx.x & 31) == 0 && votes != 0) atomicAdd(any_left, (uint32_t)__popc(votes));
 }
 
-// One CTA per window.  The sorted blocks that reach the window are positions [lo_of[b],
-// hi_of[b+1]).  A histogram of their keys (relative to w0 - (Z-1)) and its prefix sums give, for
-// every slot of the window, the range of blocks that reach it - those with key in [j-Z+1, j] -
-// already in sorted order.  The blocks then stream through shared memory in chunks, each chunk
-// with its gradient elements (fetched by coalesced loads); every thread owns the slots
-// tid, tid+256, ... of the window and adds, per chunk, the terms of its slots' ranges from first
-// to last, keeping the running sums in registers.  All slots are committed at the end.
-template <int MODE>
-__global__ void __launch_bounds__(256, 5)
+// One CTA per window of W = 2^LOG2W slots.  The sorted blocks that reach the window are positions
+// [lo_of[b], hi_of[b+1]); with their keys taken relative to w0 - (Z-1) ("offsets", 0 .. W+Z-2)
+// pre[t] = number of those blocks with offset < t, so that slot w0 + s is reached by the blocks
+// lo + [pre[s], pre[s+Z]) - those with key in [j-Z+1, j] - already in sorted order.  pre[] is
+// written straight from the sorted keys: the block at relative position e stores e into
+// pre[offset of block e-1 + 1 .. its own offset].  The blocks then stream through shared memory in
+// chunks, each chunk with its gradient elements (fetched by coalesced loads); every thread owns
+// the slots tid, tid+256, ... of the window and adds, per chunk, the terms of its slots' ranges
+// from first to last, keeping the running sums in registers.  All slots are committed at the end.
+template <int MODE, int LOG2W>
+__global__ void __launch_bounds__(256, 6)
 det_apply_window_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint32_t* __restrict__ V,
                         const uint32_t* __restrict__ lo_of, const uint32_t* __restrict__ hi_of,
                         uint32_t chunk, int vec4) {
-    __shared__ uint2 ent[kWinEnt];
+    constexpr uint32_t W = 1u << LOG2W;
+    constexpr int kSlots = W / 256;
+    __shared__ uint2 ent[kWinEnt];  // .x = (row of the block in stage[]) - key, .y = payload
     __shared__ __align__(16) float stage[kWinStage];
-    __shared__ uint32_t pre[(1u << kWinLog2Max) + kWinMaxZ + 8];  // count per key offset, then prefix
-    __shared__ uint32_t warp_sums[8];
+    __shared__ uint32_t pre[W + kWinMaxZ + 8];
     if (a.status != nullptr && *a.status != 0) return;
     const MapParams& mp = a.mp;
-    const uint32_t tid = threadIdx.x, lane = tid & 31;
+    const uint32_t tid = threadIdx.x;
     const uint32_t b = blockIdx.x;
-    if (a.win_left[b] != 0) return;
-    const uint32_t W = 1u << a.win_log2, Z = mp.Z;
-    const uint64_t w0 = (uint64_t)b << a.win_log2;
     const uint32_t lo = lo_of[b], hi = hi_of[b + 1];
+    if (a.win_left[b] != 0) return;
+    const uint32_t Z = mp.Z;
+    const uint64_t w0 = (uint64_t)b << LOG2W;
     const uint32_t n = hi - lo;
     if (n == 0) return;
+    if (tid < W / 32) {  // ask the window's target lines into L2 for the commit at the end
+        const uint64_t j = w0 + ((uint64_t)tid << 5);
+        if (j < mp.m) asm volatile("prefetch.global.L2 [%0];" ::"l"(a.target + j));
+    }
     const bool one_chunk = n <= chunk;
-    const uint32_t span = W + Z - 1;  // key offsets 0 .. span-1, relative to w0 - (Z-1)
-    for (uint32_t t = tid; t <= span; t += 256) pre[t] = 0;
-    __syncthreads();
-    for (uint32_t e0 = 0; e0 < n; e0 += 256) {
-        const uint32_t e = e0 + tid;
-        uint32_t off = 0xFFFFFFFFu;
+    const uint32_t span = W + Z - 1;           // offsets 0 .. span-1; pre[0 .. span]
+    const uint32_t bias = (uint32_t)w0 - (Z - 1);  // offset = key - bias (mod 2^32; keys reach >= bias)
+    for (uint32_t e = tid; e <= n; e += 256) {
+        const uint32_t from = e > 0 ? __ldg(K + lo + e - 1) - bias + 1 : 0;
+        uint32_t to = span;
         if (e < n) {
             const uint32_t k = __ldg(K + lo + e);
-            if (one_chunk) ent[e] = make_uint2(k, __ldg(V + lo + e));
-            off = (uint32_t)((uint64_t)k + (Z - 1) - w0);
+            to = k - bias;
+            if (one_chunk) ent[e] = make_uint2(e * Z - k, __ldg(V + lo + e));
         }
-        const uint32_t off0 = __shfl_sync(0xFFFFFFFFu, off, 0);
-        if (__all_sync(0xFFFFFFFFu, off == off0)) {  // a run of one key: count it once
-            if (lane == 0 && off != 0xFFFFFFFFu) atomicAdd(&pre[off], 32u);
-        } else if (off != 0xFFFFFFFFu) {
-            atomicAdd(&pre[off], 1u);
-        }
+        for (uint32_t t = from; t <= to; ++t) pre[t] = e;
     }
     __syncthreads();
-    // exclusive prefix sums over pre[0 .. span], each thread a run of consecutive offsets
-    {
-        const uint32_t per = (span + 1 + 255) / 256;
-        const uint32_t t0 = tid * per < span + 1 ? tid * per : span + 1;
-        const uint32_t t1 = t0 + per < span + 1 ? t0 + per : span + 1;
-        uint32_t mine = 0;
-        for (uint32_t t = t0; t < t1; ++t) mine += pre[t];
-        uint32_t run = cta_exclusive_scan_256(mine, warp_sums);  // syncs inside
-        for (uint32_t t = t0; t < t1; ++t) {
-            const uint32_t c = pre[t];
-            pre[t] = run;
-            run += c;
-        }
-    }
-    __syncthreads();
-    // slot j = w0 + sl is reached by the blocks with key offset in [sl, sl + Z - 1]:
-    // sorted positions lo + [pre[sl], pre[sl + Z])
-    constexpr int kSlots = (1 << kWinLog2Max) / 256;
+    // a window in the middle of the array: every slot exists and none is a low slot
+    const bool inner = b != 0 && w0 + W <= (uint64_t)mp.m;
+    const uint32_t j0 = (uint32_t)w0 + tid;  // the thread's first slot
     float acc[kSlots];
 #pragma unroll
     for (int q = 0; q < kSlots; ++q) acc[q] = 0.0f;
@@ -758,7 +744,7 @@ det_apply_window_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint3
         if (!one_chunk) {
             if (c0 != 0) __syncthreads();  // the chunk before has been used
             for (uint32_t e = tid; e < ne; e += 256)
-                ent[e] = make_uint2(__ldg(K + lo + c0 + e), __ldg(V + lo + c0 + e));
+                ent[e] = make_uint2(e * Z - __ldg(K + lo + c0 + e), __ldg(V + lo + c0 + e));
             __syncthreads();
         }
         if (vec4) {
@@ -780,15 +766,13 @@ det_apply_window_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint3
 #pragma unroll
         for (int q = 0; q < kSlots; ++q) {
             const uint32_t sl = tid + q * 256;
-            if (sl >= W) break;
             const uint32_t first = pre[sl], last = pre[sl + Z];
-            const uint32_t f = first > c0 ? first : c0;
-            const uint32_t l = last < c1 ? last : c1;
-            if (f < l) {
-                const uint32_t j = (uint32_t)w0 + sl;  // (a slot past the array is dropped below)
+            const uint32_t f = (first > c0 ? first : c0) - c0;
+            const uint32_t l = (last < c1 ? last : c1) - c0;  // (wraps when last < c0: then f >= l)
+            if (first < c1 && last > c0) {
+                const uint32_t j = j0 + q * 256;  // (a slot past the array is dropped at the commit)
                 float s = acc[q];
-                for (uint32_t e = f - c0; e < l - c0; ++e)
-                    s = __fadd_rn(s, stage[e * Z + (j - ent[e].x)]);
+                for (uint32_t e = f; e < l; ++e) s = __fadd_rn(s, stage[ent[e].x + j]);
                 acc[q] = s;
             }
         }
@@ -799,14 +783,17 @@ det_apply_window_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint3
 #pragma unroll
     for (int q = 0; q < kSlots; ++q) {
         const uint32_t sl = tid + q * 256;
-        const uint64_t j64 = w0 + sl;
-        // low slots belong to the low-slot kernel; past the array lie the wrapped tails (the same)
-        has[q] = sl < W && j64 < mp.m && j64 + 1 >= Z && pre[sl + Z] != pre[sl];
-        old[q] = has[q] ? a.target[j64] : 0.0f;
+        has[q] = pre[sl + Z] != pre[sl];
+        if (!inner) {
+            // low slots belong to the low-slot kernel; past the array lie the wrapped tails (the same)
+            const uint64_t j64 = w0 + sl;
+            has[q] = has[q] && j64 < mp.m && j64 + 1 >= Z;
+        }
+        old[q] = has[q] ? a.target[j0 + q * 256] : 0.0f;
     }
 #pragma unroll
     for (int q = 0; q < kSlots; ++q)
-        if (has[q]) commit_slot<MODE>(a, (uint32_t)(w0 + tid + q * 256), acc[q], old[q]);
+        if (has[q]) commit_slot<MODE>(a, j0 + q * 256, acc[q], old[q]);
 }
 
 // Long walks (plain blocks only).  One CTA of four warps per handed-over round, in steps of
@@ -1129,7 +1116,12 @@ void launch_apply(ApplyArgs aa, const uint32_t* K, const uint32_t* V, const uint
     if (forked) cudaEventRecord(wb.join_event, wb.side);
     if (windows) {
         const int vec4 = mp.Z % 4 == 0 && mp.d % 4 == 0 && ((uintptr_t)aa.grad_out & 15) == 0;
-        det_apply_window_kernel<MODE><<<wb.nwin, 256, 0, st>>>(aa, K, V, wb.lo_of, wb.hi_of, chunk, vec4);
+        switch (wb.win_log2) {
+            case 8: det_apply_window_kernel<MODE, 8><<<wb.nwin, 256, 0, st>>>(aa, K, V, wb.lo_of, wb.hi_of, chunk, vec4); break;
+            case 9: det_apply_window_kernel<MODE, 9><<<wb.nwin, 256, 0, st>>>(aa, K, V, wb.lo_of, wb.hi_of, chunk, vec4); break;
+            case 10: det_apply_window_kernel<MODE, 10><<<wb.nwin, 256, 0, st>>>(aa, K, V, wb.lo_of, wb.hi_of, chunk, vec4); break;
+            default: det_apply_window_kernel<MODE, 11><<<wb.nwin, 256, 0, st>>>(aa, K, V, wb.lo_of, wb.hi_of, chunk, vec4); break;
+        }
     }
     if (forked) cudaStreamWaitEvent(st, wb.join_event, 0);
 }
