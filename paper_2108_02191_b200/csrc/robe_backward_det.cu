@@ -380,7 +380,8 @@ __device__ __forceinline__ void commit_slot(const ApplyArgs& a, uint32_t j, floa
 // handed-over rounds is full).
 constexpr uint32_t kRing = 128;
 // window apply: the array is cut into windows of 2^8 .. 2^11 slots, one CTA each
-constexpr uint32_t kWinLog2Min = 8, kWinLog2Max = 11;
+constexpr uint32_t kWinLog2Min = 9, kWinLog2Max = 11;
+constexpr uint32_t kWinThreads = 512;     // threads of the window kernel (<= the shortest window)
 constexpr uint32_t kWinMaxZ = 128;        // longest block the window kernel takes
 constexpr uint32_t kWinEnt = 512;         // sorted blocks per chunk, at most
 constexpr uint32_t kWinStage = 6144;      // gradient elements per chunk, at most (>= kWinMaxZ)
@@ -692,15 +693,15 @@ det_window_classify_kernel(const uint32_t* __restrict__ lo_of, const uint32_t* _
 // written straight from the sorted keys: the block at relative position e stores e into
 // pre[offset of block e-1 + 1 .. its own offset].  The blocks then stream through shared memory in
 // chunks, each chunk with its gradient elements (fetched by coalesced loads); every thread owns
-// the slots tid, tid+256, ... of the window and adds, per chunk, the terms of its slots' ranges
+// the slots tid, tid+T, ... (T threads) of the window and adds, per chunk, the terms of its slots' ranges
 // from first to last, keeping the running sums in registers.  All slots are committed at the end.
 template <int MODE, int LOG2W>
-__global__ void __launch_bounds__(256, 6)
+__global__ void __launch_bounds__(kWinThreads, 4)
 det_apply_window_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint32_t* __restrict__ V,
                         const uint32_t* __restrict__ lo_of, const uint32_t* __restrict__ hi_of,
                         uint32_t chunk, int vec4) {
     constexpr uint32_t W = 1u << LOG2W;
-    constexpr int kSlots = W / 256;
+    constexpr int kSlots = W / kWinThreads;
     __shared__ uint2 ent[kWinEnt];  // .x = (row of the block in stage[]) - key, .y = payload
     __shared__ __align__(16) float stage[kWinStage];
     __shared__ uint32_t pre[W + kWinMaxZ + 8];
@@ -721,7 +722,7 @@ det_apply_window_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint3
     const bool one_chunk = n <= chunk;
     const uint32_t span = W + Z - 1;           // offsets 0 .. span-1; pre[0 .. span]
     const uint32_t bias = (uint32_t)w0 - (Z - 1);  // offset = key - bias (mod 2^32; keys reach >= bias)
-    for (uint32_t e = tid; e <= n; e += 256) {
+    for (uint32_t e = tid; e <= n; e += kWinThreads) {
         const uint32_t from = e > 0 ? __ldg(K + lo + e - 1) - bias + 1 : 0;
         uint32_t to = span;
         if (e < n) {
@@ -743,21 +744,21 @@ det_apply_window_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint3
         const uint32_t ne = c1 - c0;
         if (!one_chunk) {
             if (c0 != 0) __syncthreads();  // the chunk before has been used
-            for (uint32_t e = tid; e < ne; e += 256)
+            for (uint32_t e = tid; e < ne; e += kWinThreads)
                 ent[e] = make_uint2(e * Z - __ldg(K + lo + c0 + e), __ldg(V + lo + c0 + e));
             __syncthreads();
         }
         if (vec4) {
             const uint32_t zq = Z >> 2, tot = ne * zq;
             const bool pow2 = mp.log2Z != 0xFFFFFFFFu;
-            for (uint32_t t = tid; t < tot; t += 256) {
+            for (uint32_t t = tid; t < tot; t += kWinThreads) {
                 const uint32_t e = pow2 ? t >> (mp.log2Z - 2) : t / zq, o = t - e * zq;
                 reinterpret_cast<float4*>(stage)[t] =
                     __ldg(reinterpret_cast<const float4*>(a.grad_out + ent[e].y) + o);
             }
         } else {
             const uint32_t tot = ne * Z;
-            for (uint32_t t = tid; t < tot; t += 256) {
+            for (uint32_t t = tid; t < tot; t += kWinThreads) {
                 const uint32_t e = t / Z, o = t - e * Z;
                 stage[t] = __ldg(a.grad_out + ((uint64_t)ent[e].y + o));
             }
@@ -765,12 +766,12 @@ det_apply_window_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint3
         __syncthreads();
 #pragma unroll
         for (int q = 0; q < kSlots; ++q) {
-            const uint32_t sl = tid + q * 256;
+            const uint32_t sl = tid + q * kWinThreads;
             const uint32_t first = pre[sl], last = pre[sl + Z];
             const uint32_t f = (first > c0 ? first : c0) - c0;
             const uint32_t l = (last < c1 ? last : c1) - c0;  // (wraps when last < c0: then f >= l)
             if (first < c1 && last > c0) {
-                const uint32_t j = j0 + q * 256;  // (a slot past the array is dropped at the commit)
+                const uint32_t j = j0 + q * kWinThreads;  // (a slot past the array is dropped at the commit)
                 float s = acc[q];
                 for (uint32_t e = f; e < l; ++e) s = __fadd_rn(s, stage[ent[e].x + j]);
                 acc[q] = s;
@@ -782,18 +783,18 @@ det_apply_window_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint3
     bool has[kSlots];
 #pragma unroll
     for (int q = 0; q < kSlots; ++q) {
-        const uint32_t sl = tid + q * 256;
+        const uint32_t sl = tid + q * kWinThreads;
         has[q] = pre[sl + Z] != pre[sl];
         if (!inner) {
             // low slots belong to the low-slot kernel; past the array lie the wrapped tails (the same)
             const uint64_t j64 = w0 + sl;
             has[q] = has[q] && j64 < mp.m && j64 + 1 >= Z;
         }
-        old[q] = has[q] ? a.target[j0 + q * 256] : 0.0f;
+        old[q] = has[q] ? a.target[j0 + q * kWinThreads] : 0.0f;
     }
 #pragma unroll
     for (int q = 0; q < kSlots; ++q)
-        if (has[q]) commit_slot<MODE>(a, j0 + q * 256, acc[q], old[q]);
+        if (has[q]) commit_slot<MODE>(a, j0 + q * kWinThreads, acc[q], old[q]);
 }
 
 // Long walks (plain blocks only).  One CTA of four warps per handed-over round, in steps of
@@ -1117,10 +1118,9 @@ void launch_apply(ApplyArgs aa, const uint32_t* K, const uint32_t* V, const uint
     if (windows) {
         const int vec4 = mp.Z % 4 == 0 && mp.d % 4 == 0 && ((uintptr_t)aa.grad_out & 15) == 0;
         switch (wb.win_log2) {
-            case 8: det_apply_window_kernel<MODE, 8><<<wb.nwin, 256, 0, st>>>(aa, K, V, wb.lo_of, wb.hi_of, chunk, vec4); break;
-            case 9: det_apply_window_kernel<MODE, 9><<<wb.nwin, 256, 0, st>>>(aa, K, V, wb.lo_of, wb.hi_of, chunk, vec4); break;
-            case 10: det_apply_window_kernel<MODE, 10><<<wb.nwin, 256, 0, st>>>(aa, K, V, wb.lo_of, wb.hi_of, chunk, vec4); break;
-            default: det_apply_window_kernel<MODE, 11><<<wb.nwin, 256, 0, st>>>(aa, K, V, wb.lo_of, wb.hi_of, chunk, vec4); break;
+            case 9: det_apply_window_kernel<MODE, 9><<<wb.nwin, kWinThreads, 0, st>>>(aa, K, V, wb.lo_of, wb.hi_of, chunk, vec4); break;
+            case 10: det_apply_window_kernel<MODE, 10><<<wb.nwin, kWinThreads, 0, st>>>(aa, K, V, wb.lo_of, wb.hi_of, chunk, vec4); break;
+            default: det_apply_window_kernel<MODE, 11><<<wb.nwin, kWinThreads, 0, st>>>(aa, K, V, wb.lo_of, wb.hi_of, chunk, vec4); break;
         }
     }
     if (forked) cudaStreamWaitEvent(st, wb.join_event, 0);
