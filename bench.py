@@ -44,7 +44,7 @@ NCU_TRAFFIC_BYTES = {
     # the forward also writes the block starts; backward = count, scan, scatter, binned_apply
     ("cfg4_multihot", "binned", True): {"forward": 4_432_388_498, "backward": 4_824_968_027},
     # backward = four sort passes, window bounds and classes, the four apply kernels
-    ("cfg4_multihot", "det", True): {"forward": 4_432_471_808, "backward": 7_192_080_237},
+    ("cfg4_multihot", "det", True): {"forward": 4_432_199_990, "backward": 7_244_786_340},
 }
 
 
