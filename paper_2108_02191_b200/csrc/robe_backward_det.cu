@@ -797,32 +797,49 @@ det_apply_window_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint3
         if (has[q]) commit_slot<MODE>(a, j0 + q * kWinThreads, acc[q], old[q]);
 }
 
-// Long walks (plain blocks only).  One CTA of four warps per handed-over round, in steps of
-// kLongStep = 128 positions.  Lane l of EVERY warp stands for slot l of the round.  The keys come from
-// a ring of 512 positions in shared memory.  Copying a step's gradient terms into shared memory
-// is split over the four warps (each takes a quarter of the positions; a lane copies the term
-// of its slot with cp.async into its own column, so a whole step is in flight without a
-// register per term); warp 0 then adds the terms of each slot in sorted order.  Two buffers:
-// the copies of step n+1 are issued before the adds of step n.  Sorted keys make "this
-// position still reaches slot j" a prefix property, so the copiers need no state and the adder
-// finds the length of the prefix by bisection.
-constexpr int kLongStep = 128;
-constexpr int kLongWarps = 4;
-constexpr uint32_t kLongRing = 512;  // >= 2 steps + 32 positions of lane spread, power of two
+// Long walks (plain blocks only).  One CTA of eight warps per handed-over round, in steps of
+// kLongStep = 64 positions.  Lane l of EVERY warp stands for slot l of the round.  The keys come
+// from a ring of 512 positions in shared memory.  The chain of dependent adds of one slot is the
+// definition's, so everything else is kept off the warp that adds:
+//   warp 0      adds the terms of each slot in sorted order, one step per iteration;
+//   warps 1..6  copy: each takes every sixth position of the step kLongDepth ahead, and a lane
+//               copies the term of its slot with cp.async into its own column of that step's
+//               buffer (a whole step in flight without a register per term);
+//   warp 7      brings the keys of later steps into the ring (asked for an iteration before they
+//               are stored) and finds, by bisection, how many positions of the NEXT step reach
+//               each slot - sorted keys make "this position still reaches slot j" a prefix property.
+// kLongDepth + 1 buffers; ONE barrier per step.
+constexpr int kLongStep = 64;
+constexpr int kLongWarps = 8;
+constexpr int kLongCopiers = kLongWarps - 2;
+constexpr int kLongDepth = 4;                 // steps ahead of the adder whose copies are issued
+constexpr int kLongBufs = kLongDepth + 1;
+constexpr uint32_t kLongRing = 512;           // >= (kLongDepth + 2) steps + 32 positions of lane spread, power of two
+static_assert((kLongDepth + 2) * kLongStep + 32 <= (int)kLongRing, "ring too short");
+static_assert(kLongStep == 64, "the scout warp brings in two keys per lane and step");
 
 template <int MODE>
 __global__ void __launch_bounds__(32 * kLongWarps)
 det_apply_long_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint32_t* __restrict__ V) {
-    __shared__ float terms_s[2][kLongStep][32];
+    __shared__ float terms_s[kLongBufs][kLongStep][32];
     __shared__ uint2 ring[kLongRing];
-    __shared__ uint32_t go_on;
+    __shared__ uint32_t reach_s[2][32];  // by step parity: positions of the step that reach each slot
+    __shared__ uint32_t go_on[2];        // by step parity: is there a step to add?
+    __shared__ uint32_t rec_s;
     if (a.status != nullptr && *a.status != 0) return;
     const uint32_t tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
     const uint32_t n_rec = *a.long_count < a.long_cap ? *a.long_count : a.long_cap;
     const uint32_t dst0 = (uint32_t)__cvta_generic_to_shared(&terms_s[0][0][lane]);
     constexpr uint32_t kBufBytes = kLongStep * 32 * sizeof(float);
-    constexpr int kPerWarp = kLongStep / kLongWarps;
-    for (uint32_t rec = blockIdx.x; rec < n_rec; rec += gridDim.x) {
+    constexpr int kPerCopier = (kLongStep + kLongCopiers - 1) / kLongCopiers;
+    const bool adder = w == 0, scout = w == kLongWarps - 1;
+    // Rounds differ in length by orders of magnitude: a CTA takes the next one when it is free
+    // (a.long_count[1] counts the rounds taken) instead of a fixed share.
+    for (;;) {
+        if (tid == 0) rec_s = atomicAdd(a.long_count + 1, 1u);
+        __syncthreads();  // (the barriers inside a round order this store after all reads of the last one)
+        const uint32_t rec = rec_s;
+        if (rec >= n_rec) break;
         const LongWalk* lw = a.long_walks + rec;
         const uint64_t i0 = lw->i0;
         const uint32_t j = lw->j[lane];
@@ -836,15 +853,20 @@ det_apply_long_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint32_
             if (idx >= a.nb) return make_uint2(kNoKey, 0u);
             return make_uint2(__ldg(K + idx), __ldg(V + idx));
         };
-        // This warp's quarter of the copies of the step that starts at tile-relative position `base`.
+        // This copier warp's share of the copies of the step that starts at tile-relative position `base`.
         auto issue = [&](uint32_t base, uint32_t buf) {
             const uint32_t dst = dst0 + buf * kBufBytes;
+            uint2 kv[kPerCopier];
 #pragma unroll
-            for (int q = 0; q < kPerWarp; ++q) {
-                const uint32_t t = w * kPerWarp + q;
-                const uint2 kv = ring[(base + e + t) & (kLongRing - 1)];
-                if (mine && kv.x <= j) {
-                    const float* src = a.grad_out + (kv.y + (j - kv.x));
+            for (int q = 0; q < kPerCopier; ++q) {
+                const uint32_t t = (w - 1) + q * kLongCopiers;
+                kv[q] = ring[(base + e + (t < (uint32_t)kLongStep ? t : 0u)) & (kLongRing - 1)];
+            }
+#pragma unroll
+            for (int q = 0; q < kPerCopier; ++q) {
+                const uint32_t t = (w - 1) + q * kLongCopiers;
+                if (t < (uint32_t)kLongStep && mine && kv[q].x <= j) {
+                    const float* src = a.grad_out + (kv[q].y + (j - kv[q].x));
                     asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst + t * 128u), "l"(src));
                 }
             }
@@ -861,52 +883,63 @@ det_apply_long_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint32_
             return lo;
         };
         // a step reads positions base + e + t, e < 32, t < kLongStep: [base, base + kLongStep + 32);
-        // the ring is kept filled one step further than that
-        constexpr uint32_t kAhead = 2 * kLongStep + 32;
+        // the ring is kept filled up to the end of the step kLongDepth steps ahead
+        constexpr uint32_t kAhead = (kLongDepth + 1) * kLongStep + 32;
         uint32_t base = lw->fbase;
         uint32_t ring_end = base + kAhead;
-        __syncthreads();  // the previous round's readers are done with the ring and the buffers
         for (uint32_t r = tid; r < kAhead; r += 32 * kLongWarps)
             ring[(base + r) & (kLongRing - 1)] = fetch(base + r);
+        if (tid == 0) go_on[0] = 1u;
         __syncthreads();
-        uint32_t n_cur = w == 0 ? reach(base) : 0u;
-        issue(base, 0);
+        uint2 pend0 = make_uint2(kNoKey, 0u), pend1 = pend0;  // scout: keys of ring_end + lane, + 32 + lane
+        if (scout) {
+            pend0 = fetch(ring_end + lane);
+            pend1 = fetch(ring_end + 32 + lane);
+            reach_s[0][lane] = reach(base);
+        } else if (!adder) {
+#pragma unroll
+            for (int s = 0; s < kLongDepth; ++s) issue(base + s * kLongStep, s);
+            asm volatile("cp.async.wait_group %0;" ::"n"(kLongDepth - 1) : "memory");  // step 0 is in
+        }
         for (uint32_t step = 0;; ++step) {
-            // step+1: its keys are in the ring already (ring_end = base + 2 steps + 32)
-            issue(base + kLongStep, (step + 1) & 1u);
-            uint2 fresh = make_uint2(kNoKey, 0u);
-            if (tid < (uint32_t)kLongStep) fresh = fetch(ring_end + tid);
-            uint32_t n_nxt = 0;
-            if (w == 0) {
-                n_nxt = reach(base + kLongStep);
-                const bool any_next = __ballot_sync(0xFFFFFFFFu, n_nxt != 0) != 0;
-                if (lane == 0) go_on = any_next ? 1u : 0u;
-            }
-            asm volatile("cp.async.wait_group 1;" ::: "memory");  // this thread's copies of `step`
-            __syncthreads();  // everybody's copies of `step` are in; all ring reads of step+1 are done
-            if (w == 0) {
-                const float(*buf)[32] = terms_s[step & 1u];
+            // the copies of `step` are in (every copier waited for its own) and the adds of
+            // step - 1 are done, so its buffer may be refilled; the ring holds the next keys
+            __syncthreads();
+            if (go_on[step & 1u] == 0) break;
+            if (adder) {
+                const float(*buf)[32] = terms_s[step % kLongBufs];
+                const uint32_t n_cur = reach_s[step & 1u][lane];
                 const uint32_t n_max = __reduce_max_sync(0xFFFFFFFFu, n_cur);
-                for (uint32_t t0 = 0; t0 < n_max; t0 += 8) {
-                    float x[8];
+                for (uint32_t t0 = 0; t0 < n_max; t0 += 16) {
+                    float x[16];
 #pragma unroll
-                    for (int q = 0; q < 8; ++q) x[q] = buf[t0 + q][lane];
+                    for (int q = 0; q < 16; ++q) x[q] = buf[t0 + q][lane];
 #pragma unroll
-                    for (int q = 0; q < 8; ++q)
+                    for (int q = 0; q < 16; ++q)
                         if (t0 + q < n_cur) acc = __fadd_rn(acc, x[q]);
                 }
                 if (n_cur != 0) touched = true;
+            } else if (scout) {
+                // keys: asked for a whole iteration before they are stored into the ring
+                const uint2 f0 = fetch(ring_end + kLongStep + lane);
+                const uint2 f1 = fetch(ring_end + kLongStep + 32 + lane);
+                const uint32_t n_nxt = reach(base + kLongStep);
+                reach_s[(step + 1) & 1u][lane] = n_nxt;
+                const bool any_next = __ballot_sync(0xFFFFFFFFu, n_nxt != 0) != 0;
+                if (lane == 0) go_on[(step + 1) & 1u] = any_next ? 1u : 0u;
+                ring[(ring_end + lane) & (kLongRing - 1)] = pend0;
+                ring[(ring_end + 32 + lane) & (kLongRing - 1)] = pend1;
+                pend0 = f0;
+                pend1 = f1;
+            } else {
+                issue(base + kLongDepth * kLongStep, (step + kLongDepth) % kLongBufs);
+                asm volatile("cp.async.wait_group %0;" ::"n"(kLongDepth - 1) : "memory");  // step + 1 is in
             }
-            if (tid < (uint32_t)kLongStep) ring[(ring_end + tid) & (kLongRing - 1)] = fresh;  // keys of step+2
-            const bool more = go_on != 0;
-            __syncthreads();  // adds of `step` done before its buffer is refilled; ring updated
-            if (!more) break;
             ring_end += kLongStep;
-            n_cur = n_nxt;
             base += kLongStep;
         }
         asm volatile("cp.async.wait_group 0;" ::: "memory");
-        if (w == 0 && mine && touched) commit_slot<MODE>(a, j, acc, a.target[j]);
+        if (adder && mine && touched) commit_slot<MODE>(a, j, acc, a.target[j]);
     }
 }
 
@@ -1247,7 +1280,7 @@ cudaError_t launch_backward_det(const Problem& pb, const float* grad_out, float*
     }
 
     uint32_t* long_count = (uint32_t*)(ws + L.long_count);
-    cudaMemsetAsync(long_count, 0, sizeof(uint32_t), st);
+    cudaMemsetAsync(long_count, 0, 2 * sizeof(uint32_t), st);  // [0] rounds handed over, [1] rounds taken
     ApplyArgs aa{mp, grad_out, pb.indices, target, lr, nb, pb.status, adam ? *adam : AdamState{},
                  long_count, (LongWalk*)(ws + L.long_walks), L.long_cap, nullptr, nullptr, 0};
     const WindowBuffers wb{(uint32_t*)(ws + L.bounds),
