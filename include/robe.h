@@ -64,6 +64,14 @@ typedef enum {
 #define ROBE_OPT_INDEX_TYPE 6 /* ROBE_I64 (default) | ROBE_I32: element type of `indices` in the
                                  calls that follow (offsets stay int64)                   */
 
+#define ROBE_OPT_BAG_LAYOUT 7 /* ROBE_BAGS_SAMPLE_MAJOR (default): bag k = n*T + e, out and grad_out are
+                                 [batch, T, d];  ROBE_BAGS_TABLE_MAJOR: bag k = e*batch + n - the ids of
+                                 table 0 for all samples, then table 1, ... (per-table id lists laid end
+                                 to end) - and out and grad_out are [T, batch, d].  Applies to the calls
+                                 that follow; offsets index bags in the chosen order.              */
+#define ROBE_BAGS_SAMPLE_MAJOR 0
+#define ROBE_BAGS_TABLE_MAJOR 1
+
 /* index element types */
 #define ROBE_I64 0
 #define ROBE_I32 1
@@ -132,7 +140,8 @@ int robe_get_hash_constants(robe_handle_t h, uint64_t out[9]);
  *   offsets  device pointer, int64 [batch*T + 1], offsets[0] = 0, non-decreasing,
  *            offsets[batch*T] = nnz; or NULL for one-hot (then nnz == batch*T).
  *   batch    number of samples B >= 0;  nnz >= 0 total ids.
- *   out      device pointer, fp32 [batch, T, d], fully overwritten; an empty bag gives +0.
+ *   out      device pointer, fp32 [batch, T, d] ([T, batch, d] with ROBE_BAGS_TABLE_MAJOR), fully
+ *            overwritten; an empty bag gives +0.
  * Errors: ROBE_ERR_INVALID_ARG, ROBE_ERR_NO_ARRAY, ROBE_ERR_CUDA.
  */
 int robe_forward(robe_handle_t h, const void* indices, const int64_t* offsets, int64_t batch,

@@ -166,12 +166,19 @@ static void bag_bounds(const int64_t *offsets, int64_t k, int64_t *lo, int64_t *
 
 /* One output row: E summed over the bag, sequentially, in fp32, the first term
    initialising the accumulator (empty bag -> +0). */
+/* Table of bag number `bag`.  Sample-major bags are numbered n*T + e (the default); table-major
+ * bags e*B + n, the per-table id lists laid end to end: per_table = B, the number of bags of one
+ * table, selects that numbering, per_table = 0 the default. */
+static uint64_t table_of(int64_t bag, uint64_t T, int64_t per_table) {
+    return per_table ? (uint64_t)(bag / per_table) : (uint64_t)bag % T;
+}
+
 static void forward_one_bag(const uint64_t k[9], uint64_t m, uint64_t Z, uint64_t d, uint64_t T,
                             int sign, const void *array, int dtype, const int64_t *indices,
-                            const int64_t *offsets, int64_t bag, float *row) {
+                            const int64_t *offsets, int64_t bag, int64_t per_table, float *row) {
     int64_t lo, hi;
     bag_bounds(offsets, bag, &lo, &hi);
-    uint64_t e = (uint64_t)bag % T;
+    uint64_t e = table_of(bag, T, per_table);
     for (uint64_t i = 0; i < d; ++i) row[i] = 0.0f;
     for (int64_t p = lo; p < hi; ++p) {
         uint64_t x = (uint64_t)indices[p];
@@ -191,21 +198,21 @@ static void forward_one_bag(const uint64_t k[9], uint64_t m, uint64_t Z, uint64_
 /* Forward over all bags: out[batch*T, d] (Section 3.2 forward; pooling as stated above). */
 void robe_oracle_forward(const uint64_t k[9], uint64_t m, uint64_t Z, uint64_t d, uint64_t T,
                          int sign, const void *array, int dtype, const int64_t *indices,
-                         const int64_t *offsets, int64_t batch, float *out) {
+                         const int64_t *offsets, int64_t batch, int64_t per_table, float *out) {
     int64_t nbags = batch * (int64_t)T;
 #pragma omp parallel for schedule(static)
     for (int64_t bag = 0; bag < nbags; ++bag)
-        forward_one_bag(k, m, Z, d, T, sign, array, dtype, indices, offsets, bag, out + bag * d);
+        forward_one_bag(k, m, Z, d, T, sign, array, dtype, indices, offsets, bag, per_table, out + bag * d);
 }
 
 /* Forward for a chosen list of bags only: out[nsel, d]. */
 void robe_oracle_forward_bags(const uint64_t k[9], uint64_t m, uint64_t Z, uint64_t d, uint64_t T,
                               int sign, const void *array, int dtype, const int64_t *indices,
                               const int64_t *offsets, const int64_t *bags, int64_t nsel,
-                              float *out) {
+                              int64_t per_table, float *out) {
 #pragma omp parallel for schedule(static)
     for (int64_t s = 0; s < nsel; ++s)
-        forward_one_bag(k, m, Z, d, T, sign, array, dtype, indices, offsets, bags[s], out + s * d);
+        forward_one_bag(k, m, Z, d, T, sign, array, dtype, indices, offsets, bags[s], per_table, out + s * d);
 }
 
 /* The slots idx(e,x,i) of one embedding, for tests that need the mapping itself. */
@@ -224,14 +231,14 @@ void robe_oracle_locate(const uint64_t k[9], uint64_t m, uint64_t Z, uint64_t d,
    L1 mass l1[j-j0] = sum |dE| over the same contributions.  Both are ADDED to. */
 void robe_oracle_backward_f64(const uint64_t k[9], uint64_t m, uint64_t Z, uint64_t d, uint64_t T,
                               int sign, const float *grad_out, const int64_t *indices,
-                              const int64_t *offsets, int64_t batch, uint64_t j0, uint64_t jn,
-                              double *delta64, double *l1) {
+                              const int64_t *offsets, int64_t batch, int64_t per_table, uint64_t j0,
+                              uint64_t jn, double *delta64, double *l1) {
     int64_t nbags = batch * (int64_t)T;
     uint64_t nchunks = blocks_per_id(Z, d);
     for (int64_t bag = 0; bag < nbags; ++bag) {
         int64_t lo, hi;
         bag_bounds(offsets, bag, &lo, &hi);
-        uint64_t e = (uint64_t)bag % T;
+        uint64_t e = table_of(bag, T, per_table);
         const float *grow = grad_out + bag * (int64_t)d;
         for (int64_t p = lo; p < hi; ++p) {
             uint64_t x = (uint64_t)indices[p];
@@ -271,7 +278,8 @@ static int block_key_cmp(const void *a, const void *b) {
 int robe_oracle_backward_canonical(const uint64_t k[9], uint64_t m, uint64_t Z, uint64_t d,
                                    uint64_t T, int sign, const float *grad_out,
                                    const int64_t *indices, const int64_t *offsets, int64_t batch,
-                                   uint64_t j0, uint64_t jn, float *delta, uint8_t *touched) {
+                                   int64_t per_table, uint64_t j0, uint64_t jn, float *delta,
+                                   uint8_t *touched) {
     int64_t nbags = batch * (int64_t)T;
     uint64_t nchunks = blocks_per_id(Z, d);
     int64_t nnz = offsets ? offsets[nbags] : nbags;
@@ -286,7 +294,7 @@ int robe_oracle_backward_canonical(const uint64_t k[9], uint64_t m, uint64_t Z, 
     for (int64_t bag = 0; bag < nbags; ++bag) {
         int64_t lo, hi;
         bag_bounds(offsets, bag, &lo, &hi);
-        uint64_t e = (uint64_t)bag % T;
+        uint64_t e = table_of(bag, T, per_table);
         for (int64_t p = lo; p < hi; ++p) {
             bag_of[p] = bag;
             for (uint64_t c = 0; c < nchunks; ++c) {
@@ -304,7 +312,7 @@ int robe_oracle_backward_canonical(const uint64_t k[9], uint64_t m, uint64_t Z, 
     for (uint64_t b = 0; b < nblocks; ++b) {
         uint64_t p = keys[b].q / nchunks, c = keys[b].q % nchunks;
         int64_t bag = bag_of[p];
-        uint64_t e = (uint64_t)bag % T;
+        uint64_t e = table_of(bag, T, per_table);
         uint64_t x = (uint64_t)indices[p];
         const float *grow = grad_out + bag * (int64_t)d;
         for (uint64_t o = 0; o < block_len(Z, d, c); ++o) {

@@ -47,13 +47,13 @@ def lib() -> C.CDLL:
         _lib.robe_oracle_g.argtypes = [p, u64, u64, u64]
         _lib.robe_oracle_g.restype = C.c_int
         _lib.robe_oracle_locate.argtypes = [p, u64, u64, u64, u64, u64, p]
-        _lib.robe_oracle_forward.argtypes = [p, u64, u64, u64, u64, C.c_int, p, C.c_int, p, p, i64, p]
+        _lib.robe_oracle_forward.argtypes = [p, u64, u64, u64, u64, C.c_int, p, C.c_int, p, p, i64, i64, p]
         _lib.robe_oracle_forward_bags.argtypes = [p, u64, u64, u64, u64, C.c_int, p, C.c_int, p, p,
-                                                  p, i64, p]
+                                                  p, i64, i64, p]
         _lib.robe_oracle_backward_f64.argtypes = [p, u64, u64, u64, u64, C.c_int, p, p, p, i64,
-                                                  u64, u64, p, p]
+                                                  i64, u64, u64, p, p]
         _lib.robe_oracle_backward_canonical.argtypes = [p, u64, u64, u64, u64, C.c_int, p, p, p,
-                                                        i64, u64, u64, p, p]
+                                                        i64, i64, u64, u64, p, p]
         _lib.robe_oracle_backward_canonical.restype = C.c_int
         _lib.robe_oracle_sgd_apply.argtypes = [p, p, p, u64, C.c_float]
         _lib.robe_oracle_accumulate.argtypes = [p, p, p, u64]
@@ -85,11 +85,17 @@ def hash_constants(seed: int) -> np.ndarray:
 class Oracle:
     """The ROBE-Z mapping for one (M, Z, d, T, constants, sign) setting."""
 
-    def __init__(self, M, Z, d, num_tables, consts, sign=False):
+    def __init__(self, M, Z, d, num_tables, consts, sign=False, table_major=False):
+        """table_major: bags are numbered e*B + n (per-table id lists laid end to end) and the
+        outputs and gradients are [T, B, d]; default: bags n*T + e, [B, T, d]."""
         self.M, self.Z, self.d, self.T = int(M), int(Z), int(d), int(num_tables)
         self.k = np.ascontiguousarray(consts, dtype=np.uint64)
         assert self.k.shape == (9,)
         self.sign = 1 if sign else 0
+        self.table_major = bool(table_major)
+
+    def _per_table(self, batch) -> int:
+        return int(batch) if self.table_major else 0
 
     # -- mapping -------------------------------------------------------------
     def h(self, e, x, c) -> int:
@@ -121,17 +127,19 @@ class Oracle:
         indices, offsets = _i64(indices), _i64(offsets)
         out = np.empty((batch * self.T, self.d), dtype=np.float32)
         lib().robe_oracle_forward(_ptr(self.k), self.M, self.Z, self.d, self.T, self.sign,
-                                  _ptr(array), dt, _ptr(indices), _ptr(offsets), batch, _ptr(out))
-        return out.reshape(batch, self.T, self.d)
+                                  _ptr(array), dt, _ptr(indices), _ptr(offsets), batch,
+                                  self._per_table(batch), _ptr(out))
+        return out.reshape((self.T, batch, self.d) if self.table_major else (batch, self.T, self.d))
 
-    def forward_bags(self, array, indices, offsets, bags) -> np.ndarray:
+    def forward_bags(self, array, indices, offsets, bags, batch=None) -> np.ndarray:
+        assert batch is not None or not self.table_major, "table-major bags need the batch size"
         array, dt = self._array_args(array)
         assert array.shape[0] == self.M
         indices, offsets, bags = _i64(indices), _i64(offsets), _i64(bags)
         out = np.empty((len(bags), self.d), dtype=np.float32)
         lib().robe_oracle_forward_bags(_ptr(self.k), self.M, self.Z, self.d, self.T, self.sign,
                                        _ptr(array), dt, _ptr(indices), _ptr(offsets), _ptr(bags),
-                                       len(bags), _ptr(out))
+                                       len(bags), self._per_table(batch or 0), _ptr(out))
         return out
 
     # -- backward ------------------------------------------------------------
@@ -143,7 +151,7 @@ class Oracle:
         l1 = np.zeros(jn, dtype=np.float64)
         lib().robe_oracle_backward_f64(_ptr(self.k), self.M, self.Z, self.d, self.T, self.sign,
                                        _ptr(grad_out), _ptr(indices), _ptr(offsets), batch,
-                                       j0, jn, _ptr(delta), _ptr(l1))
+                                       self._per_table(batch), j0, jn, _ptr(delta), _ptr(l1))
         return delta, l1
 
     def backward_canonical(self, grad_out, indices, offsets, batch, j0=0, jn=None):
@@ -154,8 +162,8 @@ class Oracle:
         touched = np.empty(jn, dtype=np.uint8)
         rc = lib().robe_oracle_backward_canonical(_ptr(self.k), self.M, self.Z, self.d, self.T,
                                                   self.sign, _ptr(grad_out), _ptr(indices),
-                                                  _ptr(offsets), batch, j0, jn, _ptr(delta),
-                                                  _ptr(touched))
+                                                  _ptr(offsets), batch, self._per_table(batch), j0, jn,
+                                                  _ptr(delta), _ptr(touched))
         if rc != 0:
             raise MemoryError("oracle could not allocate its key list")
         return delta, touched

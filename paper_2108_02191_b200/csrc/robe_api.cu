@@ -28,6 +28,7 @@ struct robe_ctx {
     int bwd_variant;
     int32_t* status_word;
     int index_type;
+    int bag_layout;
     // second stream of the deterministic backward, made at the first call that can use it
     bool side_tried;
     cudaStream_t side;
@@ -80,6 +81,7 @@ bool check_sizes(robe_ctx* h, const void* indices, const int64_t* offsets, int64
     const int64_t nbags = batch * (int64_t)h->T;
     if (batch != 0 && nbags / batch != (int64_t)h->T) return false;  // overflow
     if (offsets == nullptr && nnz != nbags) return false;
+    if (h->bag_layout == ROBE_BAGS_TABLE_MAJOR && batch >= (1ll << 32)) return false;  // B is kept in 32 bits
     return true;
 }
 
@@ -87,6 +89,10 @@ Problem make_problem(robe_ctx* h, const void* indices, const int64_t* offsets, i
                      int64_t nnz) {
     Problem pb;
     pb.mp = h->mp;
+    if (h->bag_layout == ROBE_BAGS_TABLE_MAJOR && batch > 0) {  // bag k belongs to table k / batch
+        pb.mp.B = (uint32_t)batch;  // (below 2^32: checked with the other sizes)
+        pb.mp.bmagic = 0xFFFFFFFFFFFFFFFFull / (uint64_t)batch + 1;
+    }
     pb.array = h->array;
     pb.dtype = h->dtype;
     pb.sign = h->sign;
@@ -187,6 +193,8 @@ int robe_create(robe_handle_t* out, uint64_t M, uint32_t Z, uint32_t d, uint32_t
         mp.log2Z = l;
     }
     mp.tmagic = 0xFFFFFFFFFFFFFFFFull / num_tables + 1;
+    mp.bmagic = 0;
+    mp.B = 0;
     h->array = nullptr;
     h->dtype = ROBE_F32;
     h->sign = 0;
@@ -196,6 +204,7 @@ int robe_create(robe_handle_t* out, uint64_t M, uint32_t Z, uint32_t d, uint32_t
     h->bwd_variant = 0;
     h->status_word = nullptr;
     h->index_type = ROBE_I64;
+    h->bag_layout = ROBE_BAGS_SAMPLE_MAJOR;
     h->side_tried = false;
     h->side = nullptr;
     h->fork_event = h->join_event = nullptr;
@@ -238,6 +247,10 @@ int robe_set_option(robe_handle_t h, int key, int64_t value) {
         case ROBE_OPT_INDEX_TYPE:
             if (value != ROBE_I64 && value != ROBE_I32) return ROBE_ERR_INVALID_ARG;
             h->index_type = (int)value;
+            return ROBE_OK;
+        case ROBE_OPT_BAG_LAYOUT:
+            if (value != ROBE_BAGS_SAMPLE_MAJOR && value != ROBE_BAGS_TABLE_MAJOR) return ROBE_ERR_INVALID_ARG;
+            h->bag_layout = (int)value;
             return ROBE_OK;
         case ROBE_OPT_BWD_KERNEL:
             if (value < 0 || value > 2) return ROBE_ERR_INVALID_ARG;

@@ -42,6 +42,8 @@ struct MapParams {
     uint32_t C;        // blocks per embedding = ceil(d / Z)
     uint32_t log2Z;    // valid when Z is a power of two, else 0xFFFFFFFF
     uint64_t tmagic;   // floor((2^64 - 1) / T) + 1, for k mod T with k < 2^32
+    uint64_t bmagic;   // table-major bags: floor((2^64 - 1) / B) + 1, for k / B with k < 2^32
+    uint32_t B;        // table-major bags: the batch size B of the call; 0 = sample-major bags
 };
 
 // (hi * 2^64 + lo) mod P for hi < 2^61.
@@ -84,8 +86,15 @@ __device__ __forceinline__ uint32_t mod_m(uint64_t t, uint32_t m, uint64_t mu) {
     return (uint32_t)(r >= m ? r - m : r);
 }
 
-// k mod T for k < 2^32 (Lemire's fastmod with a 64-bit magic number).
+// Table of bag k.  Sample-major bags (k = n T + e): k mod T, by Lemire's fastmod with a 64-bit
+// magic number for k < 2^32.  Table-major bags (k = e B + n, mp.B = B != 0): k / B, by the
+// matching fastdiv.
 __device__ __forceinline__ uint32_t table_of_bag(uint64_t k, const MapParams& mp) {
+    if (mp.B != 0) {
+        if (mp.B == 1) return (uint32_t)k;
+        if (k >> 32) return (uint32_t)(k / mp.B);
+        return (uint32_t)__umul64hi(mp.bmagic, k);
+    }
     if (k >> 32) return (uint32_t)(k % mp.T);
     uint64_t low = mp.tmagic * (uint32_t)k;
     return (uint32_t)__umul64hi(low, (uint64_t)mp.T);

@@ -426,6 +426,78 @@ def test_adjoint_identity(sign, bags):
     assert lhs == rhs
 
 
+def _renumber_table_major(ids, offsets, B, T):
+    """The same bags numbered e*B + n instead of n*T + e: ids, offsets, and old bag of every new one."""
+    old_of_new = np.array([n * T + e for e in range(T) for n in range(B)], dtype=np.int64)
+    if offsets is None:
+        return ids[old_of_new], None, old_of_new
+    pieces = [ids[offsets[k]:offsets[k + 1]] for k in old_of_new]
+    lengths = np.diff(offsets)[old_of_new]
+    return (np.concatenate(pieces) if pieces else ids[:0],
+            np.concatenate([[0], np.cumsum(lengths)]).astype(np.int64), old_of_new)
+
+
+@pytest.mark.parametrize("sign", [False, True])
+@pytest.mark.parametrize("bags", [False, True])
+def test_table_major_bags_are_the_same_bags_renumbered(sign, bags):
+    # Numbering the bags table by table changes which row of the output a bag is, nothing else:
+    # forward rows and (on integer data, where no order matters) gradient sums are those of the
+    # default numbering.
+    m, Z, d, T, B = 307, 4, 12, 3, 17
+    k = orc.hash_constants(21)
+    o = orc.Oracle(m, Z, d, T, k, sign=sign)
+    otm = orc.Oracle(m, Z, d, T, k, sign=sign, table_major=True)
+    rng = np.random.default_rng(5)
+    arr = (rng.standard_normal(m) * 0.01).astype(np.float32)
+    G = rng.integers(-8, 9, size=(B, T, d)).astype(np.float32)
+    if bags:
+        lengths = rng.integers(0, 5, size=B * T)
+        offsets = np.concatenate([[0], np.cumsum(lengths)]).astype(np.int64)
+        ids = rng.integers(0, 60, size=int(offsets[-1]))
+    else:
+        offsets, ids = None, rng.integers(0, 60, size=B * T)
+    ids_tm, offs_tm, old_of_new = _renumber_table_major(ids, offsets, B, T)
+    want = o.forward(arr, ids, offsets, B).reshape(B * T, d)[old_of_new]
+    got = otm.forward(arr, ids_tm, offs_tm, B)
+    assert got.shape == (T, B, d)
+    np.testing.assert_array_equal(got.reshape(B * T, d).view(np.uint32), want.view(np.uint32))
+    some = np.array([0, 5, B, B * T - 1], dtype=np.int64)
+    np.testing.assert_array_equal(otm.forward_bags(arr, ids_tm, offs_tm, some, batch=B).view(np.uint32),
+                                  want[some].view(np.uint32))
+    G_tm = G.reshape(B * T, d)[old_of_new].reshape(T, B, d)
+    d_sm, l1_sm = o.backward_f64(G, ids, offsets, B)
+    d_tm, l1_tm = otm.backward_f64(G_tm, ids_tm, offs_tm, B)
+    np.testing.assert_array_equal(d_tm, d_sm)
+    np.testing.assert_array_equal(l1_tm, l1_sm)
+    can, touched = otm.backward_canonical(G_tm, ids_tm, offs_tm, B)
+    np.testing.assert_array_equal(can.astype(np.float64), d_sm)
+    assert not np.any(~touched.astype(bool) & (l1_sm > 0))  # every slot that got mass is marked
+    np.testing.assert_array_equal(touched, o.backward_canonical(G, ids, offsets, B)[1])
+
+
+def test_table_major_canonical_order_follows_the_position_in_that_numbering():
+    # Four one-element embeddings on ONE slot: with A_h = B_h = 1 the ids 5 of table 0 and 4 of
+    # table 1 hash alike.  Equal block starts are added in the order of their position in the id
+    # array, which the bag numbering fixes.  Gradients (n, e): (0,0) 1e8, (0,1) 1, (1,0) -1e8,
+    # (1,1) 1; in fp32 1e8 + 1 = 1e8.
+    #   default numbering, positions (0,0) (0,1) (1,0) (1,1): ((1e8 + 1) - 1e8) + 1 = 1
+    #   table by table,    positions (0,0) (1,0) (0,1) (1,1): ((1e8 - 1e8) + 1) + 1 = 2
+    m, T, B = 97, 2, 2
+    kk = consts()
+    G = np.array([[[1e8], [1.0]], [[-1e8], [1.0]]], dtype=np.float32)  # [B, T, 1]
+    ids = np.array([5, 4, 5, 4], dtype=np.int64)                       # (n, e) = (0,0) (0,1) (1,0) (1,1)
+    o = orc.Oracle(m, 1, 1, T, kk)
+    slot = o.idx(0, 5, 0)
+    assert slot == o.idx(1, 4, 0)
+    can, _ = o.backward_canonical(G, ids, None, B)
+    assert can[slot] == np.float32(1.0)
+    otm = orc.Oracle(m, 1, 1, T, kk, table_major=True)
+    ids_tm, _, old_of_new = _renumber_table_major(ids, None, B, T)
+    G_tm = G.reshape(B * T, 1)[old_of_new].reshape(T, B, 1)
+    can_tm, _ = otm.backward_canonical(G_tm, ids_tm, None, B)
+    assert can_tm[slot] == np.float32(2.0)
+
+
 def test_gradient_mass_is_conserved():
     m, Z, d, T, B = 500, 8, 16, 2, 30
     o = orc.Oracle(m, Z, d, T, orc.hash_constants(13))
