@@ -271,8 +271,10 @@ def run_ours(args, w):
     B, T, d = w.batch, w.num_tables, w.d
     nbags = B * T
     batches = []
+    table_major = args.bag_layout == "table-major"
     for v in rank_batch_variants(rank, NB):
-        batches.append(synth.make_ids(w, B, variant=v))
+        ids_v = synth.make_ids(w, B, variant=v)
+        batches.append(synth.to_table_major(ids_v[0], ids_v[1], B, T) if table_major else ids_v)
     array = synth.make_array(w, dev)
     gen = torch.Generator(device=dev)
     gen.manual_seed(w.data_seed + 17 * rank)
@@ -285,6 +287,8 @@ def run_ours(args, w):
 
     h = robe.robe_create(w.M, w.Z, w.d, T, w.hash_seed)
     robe.robe_attach_array(h, array)
+    if table_major:
+        robe.robe_set_option(h, robe.ROBE_OPT_BAG_LAYOUT, robe.ROBE_BAGS_TABLE_MAJOR)
     lr = 1.0  # the paper trains its DLRM with plain SGD at learning rate 1.0 (Section 5)
     ws = None
     bwd_launches = 1
@@ -467,7 +471,7 @@ def run_ours(args, w):
         "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": w.name, "num_tables": T, "d": d, "Z": w.Z, "M": w.M, "batch_per_gpu": B,
-                   "ids_per_step_per_gpu": nnz_per_step, "ids": args.ids, "bags": bags, "backward": {"atomic": "atomic", "det": "deterministic", "binned": "binned atomic"}[args.backward] +
+                   "ids_per_step_per_gpu": nnz_per_step, "ids": args.ids, "bags": bags, "bag_layout": args.bag_layout, "backward": {"atomic": "atomic", "det": "deterministic", "binned": "binned atomic"}[args.backward] +
                    (", SGD fused" if dense is None else ", dense fp32 gradient"),
                    "block_starts": ("hashed once per step: kept by the forward for the backward" if share_keys
                                     else "hashed by the forward and again by the backward"),
@@ -511,6 +515,8 @@ def main():
                     help="backward variant of the step; auto = binned atomic adds when the array lives in "
                          "HBM and is touched several times per step, else plain atomic adds")
     ap.add_argument("--ids", default="int64", choices=["int64", "int32"], help="element type of the id arrays")
+    ap.add_argument("--bag-layout", default="sample-major", choices=["sample-major", "table-major"],
+                    help="bag numbering of the inputs: n*T + e (default) or e*B + n (per-table id lists end to end)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-share-keys", dest="share_keys", action="store_false",
                     help="hash the ids in the backward again (robe_forward + robe_backward) instead of "

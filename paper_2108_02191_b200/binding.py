@@ -34,6 +34,9 @@ ROBE_OPT_INDEX_TYPE = 6
 
 ROBE_I64 = 0
 ROBE_I32 = 1
+ROBE_OPT_BAG_LAYOUT = 7
+ROBE_BAGS_SAMPLE_MAJOR = 0
+ROBE_BAGS_TABLE_MAJOR = 1
 
 ROBE_BWD_ATOMIC = 0
 ROBE_BWD_DETERMINISTIC = 1

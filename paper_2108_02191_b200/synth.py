@@ -173,6 +173,21 @@ def array_values_at(w: RobeWorkload, j: torch.Tensor) -> torch.Tensor:
     raise ValueError(w.array_init)
 
 
+def to_table_major(indices: np.ndarray, offsets: Optional[np.ndarray], batch: int, num_tables: int):
+    """The ids of make_ids with the bags renumbered table by table (bag e*B + n instead of
+    n*T + e): the per-table id lists laid end to end.  Returns (indices, offsets)."""
+    old_of_new = (np.arange(batch, dtype=np.int64)[None, :] * num_tables
+                  + np.arange(num_tables, dtype=np.int64)[:, None]).reshape(-1)
+    if offsets is None:
+        return np.ascontiguousarray(indices[old_of_new]), None
+    lengths = np.diff(offsets)[old_of_new]
+    new_offsets = np.concatenate([[0], np.cumsum(lengths)]).astype(np.int64)
+    starts = offsets[:-1][old_of_new]
+    # position of every id of the new order in the old one
+    src = np.repeat(starts - new_offsets[:-1], lengths) + np.arange(int(new_offsets[-1]), dtype=np.int64)
+    return np.ascontiguousarray(indices[src]), new_offsets
+
+
 def make_array(w: RobeWorkload, device="cpu", chunk: int = 1 << 25) -> torch.Tensor:
     """The full array [M] on ``device``: fp32, or bf16 (round-to-nearest-even of the fp32 value)."""
     dtype = torch.float32 if w.array_dtype == "f32" else torch.bfloat16

@@ -14,13 +14,15 @@ class Case:
     """One workload instantiated on the device, with its oracle twin."""
 
     def __init__(self, w: synth.RobeWorkload, batch=None, sign=False, variant=0, array=None,
-                 ids=None, host_array=True):
+                 ids=None, host_array=True, table_major=False):
         self.w = w
         self.B = w.batch if batch is None else batch
         self.T = w.num_tables
         self.dev = torch.device("cuda:0")
         if ids is None:
             ids = synth.make_ids(w, self.B, variant)
+        if table_major:  # the same bags, numbered table by table
+            ids = synth.to_table_major(ids[0], ids[1], self.B, self.T)
         self.indices_h, self.offsets_h = ids
         self.nbags = self.B * self.T
         self.indices = torch.from_numpy(self.indices_h).to(self.dev)
@@ -29,13 +31,17 @@ class Case:
         self.array_h = synth.array_to_numpy(self.array) if host_array else None
         self.h = robe.robe_create(w.M, w.Z, w.d, w.num_tables, w.hash_seed)
         robe.robe_attach_array(self.h, self.array)
+        self.table_major = table_major
+        if table_major:
+            robe.robe_set_option(self.h, robe.ROBE_OPT_BAG_LAYOUT, robe.ROBE_BAGS_TABLE_MAJOR)
         self.sign = sign
         if sign:
             robe.robe_set_option(self.h, robe.ROBE_OPT_SIGN, 1)
         k = np.array(robe.robe_get_hash_constants(self.h), dtype=np.uint64)
         # the oracle draws its own constants; the library's must be the same numbers
         np.testing.assert_array_equal(k, orc.hash_constants(w.hash_seed))
-        self.oracle = orc.Oracle(w.M, w.Z, w.d, w.num_tables, orc.hash_constants(w.hash_seed), sign)
+        self.oracle = orc.Oracle(w.M, w.Z, w.d, w.num_tables, orc.hash_constants(w.hash_seed), sign,
+                                 table_major=table_major)
 
     def close(self):
         if self.h is not None:
@@ -101,7 +107,7 @@ class Case:
         return self.oracle.forward(self.array_h, self.indices_h, self.offsets_h, self.B)
 
     def oracle_forward_bags(self, bags):
-        return self.oracle.forward_bags(self.array_h, self.indices_h, self.offsets_h, bags)
+        return self.oracle.forward_bags(self.array_h, self.indices_h, self.offsets_h, bags, batch=self.B)
 
 
 def assert_bits_equal(a: np.ndarray, b: np.ndarray, what=""):

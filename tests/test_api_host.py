@@ -60,13 +60,15 @@ def test_options_and_errors_without_device():
     h = robe.robe_create(4096, 4, 16, 4, 7)
     for key, val in [(robe.ROBE_OPT_SIGN, 2), (robe.ROBE_OPT_BWD_MODE, 5), (99, 0),
                      (robe.ROBE_OPT_VALIDATE, -1), (robe.ROBE_OPT_FWD_KERNEL, 3),
-                     (robe.ROBE_OPT_INDEX_TYPE, 2)]:
+                     (robe.ROBE_OPT_INDEX_TYPE, 2), (robe.ROBE_OPT_BAG_LAYOUT, 2)]:
         with pytest.raises(robe.RobeError):
             robe.robe_set_option(h, key, val)
     robe.robe_set_option(h, robe.ROBE_OPT_SIGN, 1)
     robe.robe_set_option(h, robe.ROBE_OPT_SIGN, 0)
     robe.robe_set_option(h, robe.ROBE_OPT_INDEX_TYPE, robe.ROBE_I32)
     robe.robe_set_option(h, robe.ROBE_OPT_INDEX_TYPE, robe.ROBE_I64)
+    robe.robe_set_option(h, robe.ROBE_OPT_BAG_LAYOUT, robe.ROBE_BAGS_TABLE_MAJOR)
+    robe.robe_set_option(h, robe.ROBE_OPT_BAG_LAYOUT, robe.ROBE_BAGS_SAMPLE_MAJOR)
     lib = robe.binding.raw()
     # forward before attach: no array (dummy non-null pointers are never dereferenced)
     dummy = C.c_void_p(0x1000)

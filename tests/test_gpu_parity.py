@@ -376,6 +376,41 @@ def test_step_sharing_block_starts_int32_ids_and_workspace_check():
         assert ei.value.status == robe.ROBE_ERR_WORKSPACE
 
 
+# Table-major bags (bag e*B + n: the per-table id lists laid end to end; out and grad_out are
+# [T, B, d]).  Every kernel takes the table of a bag from the same helper, so each kernel family
+# is run once: both forward kernels, the atomic, binned and deterministic backward (window and
+# position-tile apply), the step that shares block starts, Adam; one-hot and pooled input.
+@pytest.mark.parametrize("bags", [None, (3, 0, 9)])
+@pytest.mark.parametrize("d,Z,M,batch", [(16, 4, 4096, 61), (64, 16, 300_007, 700), (130, 2, 1000, 33),
+                                         (128, 128, 1280, 1), (16, 64, 1000, 50), (32, 8, 2_000_003, 90)])
+def test_table_major_bags(d, Z, M, batch, bags):
+    w = small(d=d, Z=Z, M=M, bag_rule=bags, batch=batch)
+    for sign in (False, True):
+        with Case(w, sign=sign, table_major=True) as c, Case(w, sign=sign) as ref:
+            want = c.oracle_forward()  # [T, B, d]
+            for kernel in ([0, 1, 2] if d <= 128 else [0, 1]):
+                assert_bits_equal(c.forward(kernel).cpu().numpy().reshape(want.shape), want,
+                                  f"table-major forward k={kernel} d={d} Z={Z}")
+            # the same rows as the default numbering gives, at other places (not through the oracle)
+            rows_ref = ref.forward().cpu().numpy().reshape(c.B, c.T, d).transpose(1, 0, 2)
+            assert_bits_equal(c.forward().cpu().numpy().reshape(c.T, c.B, d), rows_ref, "rows renumbered")
+            g_h = np.random.default_rng(31).standard_normal((c.T, c.B, d)).astype(np.float32)
+            g_d = torch.from_numpy(g_h).to(c.dev)
+            delta64, l1 = c.oracle.backward_f64(g_h, c.indices_h, c.offsets_h, c.B)
+            can, touched = c.oracle.backward_canonical(g_h, c.indices_h, c.offsets_h, c.B)
+            assert_within_l1(c.backward(g_d, "atomic").cpu().numpy(), delta64, l1, what="table-major atomic")
+            assert_within_l1(c.backward(g_d, "binned").cpu().numpy(), delta64, l1, what="table-major binned")
+            assert_bits_equal(c.backward(g_d, "det").cpu().numpy(), can, f"table-major det d={d} Z={Z} sign={sign}")
+            out, detk = c.step_sharing_keys(g_d, "det")
+            assert_bits_equal(out.cpu().numpy().reshape(want.shape), want, "table-major forward that keeps")
+            assert_bits_equal(detk.cpu().numpy(), can, "table-major det on kept starts")
+            before = c.array_h.copy()
+            c.backward(g_d, "det", sgd=True, lr=0.5)
+            wanted = before.copy()
+            orc.sgd_apply(wanted, can, touched, 0.5)
+            assert_bits_equal(c.array.cpu().numpy(), wanted, "table-major det SGD")
+
+
 def test_backward_empty_inputs():
     w = small(bag_rule=(2, 0, 5))
     with Case(w, batch=4) as c:

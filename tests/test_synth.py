@@ -67,3 +67,18 @@ def test_grad_out_is_standard_normal():
     g = synth.make_grad_out(w)
     assert g.shape == (256, 4, 16) and g.dtype == np.float32
     assert abs(g.mean()) < 0.03 and abs(g.std() - 1) < 0.03
+
+
+def test_to_table_major_moves_whole_bags():
+    w = synth.RobeWorkload("t", 3, "list", (50, 7, 1000), 8, 4, 1000, 5, "normal0.01", "f32", "uniform",
+                           (3, 0, 6), 1, 2)
+    ids, offs = synth.make_ids(w)
+    ids_tm, offs_tm = synth.to_table_major(ids, offs, w.batch, w.num_tables)
+    assert offs_tm[0] == 0 and offs_tm[-1] == len(ids) and len(offs_tm) == len(offs)
+    for e in range(w.num_tables):
+        for n in range(w.batch):
+            old, new = n * w.num_tables + e, e * w.batch + n
+            np.testing.assert_array_equal(ids_tm[offs_tm[new]:offs_tm[new + 1]], ids[offs[old]:offs[old + 1]])
+    one, none = synth.to_table_major(np.arange(15), None, 5, 3)
+    assert none is None
+    np.testing.assert_array_equal(one.reshape(3, 5), np.arange(15).reshape(5, 3).T)
