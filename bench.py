@@ -42,9 +42,9 @@ NCU_TRAFFIC_BYTES = {
     # (workload, backward variant, block starts shared between forward and backward)
     ("cfg4_multihot", "atomic", False): {"forward": 4_197_885_696, "backward": 7_509_030_400},
     # the forward also writes the block starts; backward = count, scan, scatter, binned_apply
-    ("cfg4_multihot", "binned", True): {"forward": 4_432_388_498, "backward": 4_824_968_027},
+    ("cfg4_multihot", "binned", True): {"forward": 4_432_575_140, "backward": 4_824_216_228},
     # backward = four sort passes, window bounds and classes, the four apply kernels
-    ("cfg4_multihot", "det", True): {"forward": 4_432_199_990, "backward": 7_244_786_340},
+    ("cfg4_multihot", "det", True): {"forward": 4_432_391_881, "backward": 7_245_764_406},
 }
 
 
