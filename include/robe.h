@@ -98,17 +98,22 @@ typedef enum {
  *               piece [(x mod R) d, (x mod R) d + d) of it.
  *   d           embedding dimension (one d per handle; several handles may share
  *               one array, Section 3.1 "Multiple embedding tables").
- *   num_tables  T >= 1; the table id e of bag k is k mod T.
+ *   num_tables  T >= 1; the table id e of bag k is k mod T (k / batch after
+ *               ROBE_OPT_BAG_LAYOUT = ROBE_BAGS_TABLE_MAJOR).
  *   hash_seed   seeds the draw of the hash constants: P = 2^61 - 1 and, from a
  *               SplitMix64 stream, A_h B_h C_h D_h A_g B_g C_g D_g (61-bit draws,
  *               redrawn when outside [1,P-1] for multipliers / [0,P-1] for the
  *               additive terms), as the paper's hash family requires.
+ * A handle holds options and, after the first deterministic backward, a CUDA stream and two
+ * events of its own (no device memory): calls on ONE handle must not overlap in time on the
+ * host; different handles are independent.
  * Errors: ROBE_ERR_INVALID_ARG.
  */
 int robe_create(robe_handle_t* out, uint64_t M, uint32_t Z, uint32_t d, uint32_t num_tables,
                 uint64_t hash_seed);
 
-/* robe_destroy - free the host handle.  Device buffers stay the caller's. */
+/* robe_destroy - free the host handle (waits for the handle's own stream, if it has one).  Device
+ * buffers stay the caller's. */
 int robe_destroy(robe_handle_t h);
 
 /* robe_set_option - see the ROBE_OPT_* keys.  ROBE_ERR_INVALID_ARG on a bad key/value. */
