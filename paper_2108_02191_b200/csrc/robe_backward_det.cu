@@ -374,10 +374,10 @@ __device__ __forceinline__ void commit_slot(const ApplyArgs& a, uint32_t j, floa
 // position, UN positions per step (4 in the first step, then 8): ring reads, then the gradient
 // loads, then the adds in sorted order; the next 32 positions are fetched one step ahead of
 // their first use.  A walk that is still going after 64 positions (an id that occurs many
-// times in the batch) goes on 16 positions per step, with the gradient rows of the positions
-// after those asked into L2 ahead of time; one that is still going after 256 positions is
-// handed, with its sums so far, to the long-walk kernel below (or finished here if the list of
-// handed-over rounds is full).
+// times in the batch) is handed, with its sums so far, to the long-walk kernel below, whose
+// division of labour adds such a chain several times faster.  Only if the list of handed-over
+// rounds is full does it go on here, 16 positions per step, with the gradient rows of the
+// positions after those asked into L2 ahead of time.
 constexpr uint32_t kRing = 128;
 // window apply: the array is cut into windows of 2^8 .. 2^11 slots, one CTA each
 constexpr uint32_t kWinLog2Min = 9, kWinLog2Max = 11;
@@ -524,8 +524,9 @@ __global__ void __launch_bounds__(256)
 det_apply_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint32_t* __restrict__ V,
                  const uint32_t* __restrict__ bag_of) {
     constexpr int UN = 8;
-    constexpr uint32_t kDeepAfter = 64;       // positions after which a walk takes 16 per step
-    constexpr uint32_t kHandOverAfter = 256;  // ... and after which it goes to the long-walk kernel
+    constexpr uint32_t kDeepAfter = 64;       // positions after which a walk takes 16 per step, if it stays here
+    constexpr uint32_t kHandOverAfter = 64;   // positions after which it goes to the long-walk kernel (128 and 256
+                                              // measured slower on Zipf ids, 32 no faster)
     __shared__ uint2 ring_s[8][kRing];
     if (a.status != nullptr && *a.status != 0) return;
     if (a.any_left != nullptr && *a.any_left == 0) return;  // the window kernel served every slot
