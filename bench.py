@@ -3,7 +3,8 @@
 
 One step = one pass of the whole path over one batch: robe_forward (hash -> offset -> circular
 block gather -> bag sum-pool) followed by robe_backward (block scatter-add of the output
-gradient with the SGD step fused in).  The default workload is the multi-hot pooled
+gradient with the SGD step fused in) - called as robe_forward_keep / robe_backward_kept when
+the backward sorts the blocks, so that every id is hashed once per step.  The default workload is the multi-hot pooled
 configuration whose 1 GB array does not fit in L2 (26 tables, d=64, Z=16, batch 16384, bags of
 about 20 ids).
 
