@@ -462,6 +462,11 @@ def test_cfg3_forward_backward_full_size(Z):
         det = c.backward(g_d, "det").cpu().numpy()
         assert_within_l1(det, delta64, l1, what=f"cfg3 Z={Z} det vs fp64")
         assert_bits_equal(c.backward(g_d, "det").cpu().numpy(), det, "cfg3 det repeat")
+        # the same step with the forward's block starts: same bits (window, position-tile and
+        # long-walk kernels all take part at this size)
+        _, detk = c.step_sharing_keys(g_d, "det")
+        assert_bits_equal(detk.cpu().numpy(), det, "cfg3 det on kept starts")
+        del detk
         if Z == 128:
             can, touched = c.oracle.backward_canonical(g_h, c.indices_h, c.offsets_h, c.B)
             assert_bits_equal(det, can, "cfg3 Z=128 det vs canonical")
