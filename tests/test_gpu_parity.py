@@ -420,6 +420,9 @@ def test_backward_empty_inputs():
         for mode in ("atomic", "det"):
             ga = c.backward(g_d, mode).cpu().numpy()
             assert np.all(ga == 0)
+        for mode in ("binned", "det"):  # and through the calls that share the block starts
+            out, ga = c.step_sharing_keys(g_d, mode)
+            assert not out.any() and not ga.any()
 
 
 # ---------------------------------------------------------------------------------------
