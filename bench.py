@@ -36,16 +36,13 @@ from paper_2108_02191_b200 import synth  # noqa: E402
 METRIC = "robe_lookups_per_s_fwd_bwd"
 UNIT = "ids/s"
 
-# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu capture of the
-# full-size default workload (summaries of those captures are kept under profiles/); None = not
-# captured for that workload or backward variant.
-NCU_TRAFFIC_BYTES = {
-    # (workload, backward variant, block starts shared between forward and backward)
-    ("cfg4_multihot", "atomic", False): {"forward": 4_197_885_696, "backward": 7_509_030_400},
-    # the forward also writes the block starts; backward = count, scan, scatter, binned_apply
-    ("cfg4_multihot", "binned", True): {"forward": 4_432_575_140, "backward": 4_824_216_228},
-    # backward = four sort passes, window bounds and classes, the four apply kernels
-    ("cfg4_multihot", "det", True): {"forward": 4_432_391_881, "backward": 7_245_764_406},
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) recorded from one-pass ncu
+# captures of the full-size workload; the summaries under profiles/ hold the commands.  A record
+# applies only to the exact configuration it was captured on (workload, backward variant, shared
+# block starts, id type, bag layout, workload's own batch): any other run reports traffic = null.
+# Records go stale when a kernel changes: they are re-captured with the kernel, never edited.
+NCU_TRAFFIC_RECORDS = {
+    # (workload, backward variant, block starts shared, id type, bag layout)
 }
 
 
@@ -90,9 +87,10 @@ def forward_byte_models(w, nbags, nnz, bags, id_bytes=8):
 class ClockSampler:
     """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
 
-    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+    Q = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
          "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    PERIOD_MS = 10
 
     def __init__(self, gpu_index: int):
         self.gpu = gpu_index
@@ -104,12 +102,22 @@ class ClockSampler:
             fd, self.path = tempfile.mkstemp(suffix=".csv")
             os.close(fd)
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "50",
-                 "-i", str(self.gpu)], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms",
+                 str(self.PERIOD_MS), "-i", str(self.gpu)], stdout=open(self.path, "w"),
+                stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
-    def stop(self):
+    @staticmethod
+    def _stamp(text):
+        """Seconds since the epoch of an nvidia-smi timestamp (local time, milliseconds)."""
+        import datetime
+        return datetime.datetime.strptime(text, "%Y/%m/%d %H:%M:%S.%f").timestamp()
+
+    def stop(self, window=None):
+        """Stops sampling.  window = (t0, t1) in time.time() seconds keeps only the samples taken
+        inside the timed region (the sampler itself is started before the warm-up so that it is
+        already delivering when the region begins)."""
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
         if self.proc is None:
             return out
@@ -125,6 +133,10 @@ class ClockSampler:
                 if len(f) < 9:
                     continue
                 try:
+                    if window is not None:
+                        ts = self._stamp(f[0])
+                        if ts < window[0] or ts > window[1]:
+                            continue
                     sm.append(float(f[1]))
                     mx.append(float(f[2]))
                 except ValueError:
@@ -223,9 +235,17 @@ def run_reference(args, w):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return 0
-    sample_batch = max(1, w.batch // 16)
     array_h = synth.array_to_numpy(synth.make_array(w, "cpu"))
-    for i in range(args.warmup):
+    # Every step runs the oracle on the workload's whole batch - the sample the cpu_baseline leg of
+    # the other arm times - unless the first (warm-up) step shows that steps + warmup such steps
+    # would take more than about three minutes; then the batch is cut by a power of two.
+    sample_batch = w.batch
+    _, _, _, t_full = oracle_step_rate(w, sample_batch, array_h, variant=0)
+    planned = (args.steps + args.warmup) * t_full
+    while planned > 200.0 and sample_batch > 64:
+        sample_batch //= 2
+        planned /= 2
+    for i in range(1, args.warmup):
         oracle_step_rate(w, sample_batch, array_h, variant=i)
     total_ids, total_t, threads = 0, 0.0, 1
     for i in range(args.steps):
@@ -307,6 +327,13 @@ def run_ours(args, w):
     # a bf16 array is read-only for the library: its gradient goes to a dense fp32 array instead
     # of the fused SGD step (the array stays as it is)
     dense = torch.zeros(w.M, dtype=torch.float32, device=dev) if w.array_dtype != "f32" else None
+    # Data-parallel training step (more than one rank, fp32 array): the replicas must apply the
+    # SAME update, so the fused step gives way to backward into a dense gradient -> all-reduce
+    # (sum over ranks, 4 M bytes) -> robe_apply_sgd.  One rank needs no exchange and keeps the
+    # fused step unless --dp-step on asks for the three-phase step.
+    dp_step = w.array_dtype == "f32" and (args.dp_step == "on" or (args.dp_step == "auto" and world > 1))
+    if dp_step:
+        dense = torch.zeros(w.M, dtype=torch.float32, device=dev)
     if args.backward == "det":
         robe.robe_set_option(h, robe.ROBE_OPT_BWD_MODE, robe.ROBE_BWD_DETERMINISTIC)
         ws = torch.empty(robe.robe_backward_workspace_bytes(h, B, max(len(b[0]) for b in batches)),
@@ -328,6 +355,11 @@ def run_ours(args, w):
     if share_keys and w.d <= 128:
         bwd_launches -= (1 if bags else 0) + 1
 
+    def exchange_and_apply():
+        if dist is not None:
+            dist.all_reduce(dense, op=dist.ReduceOp.SUM)
+        robe.robe_apply_sgd(h, dense, lr / world, True)  # mean of the ranks' gradients
+
     def step(i, events=None):
         k = i % NB
         if events is not None:
@@ -344,30 +376,39 @@ def run_ours(args, w):
             robe.robe_backward(h, grad_out, d_ids[k], d_offs[k], B, dense, lr, ws)
         if events is not None:
             events[2].record()
+        if dp_step:
+            exchange_and_apply()
+            if events is not None:
+                events[3].record()
 
     def barrier():
         if dist is not None:
             dist.barrier()
         torch.cuda.synchronize()
 
+    sampler = ClockSampler(visible_gpu_index(local_rank))
+    sampler.start()  # before the warm-up, so that samples are already coming when the timing starts
     for i in range(args.warmup):
         step(i)
     barrier()
-    sampler = ClockSampler(visible_gpu_index(local_rank))
-    sampler.start()
-    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
     barrier()
     t_start = torch.cuda.Event(enable_timing=True)
     t_end = torch.cuda.Event(enable_timing=True)
+    wall0 = time.time()
     t_start.record()
     for i in range(args.steps):
         step(args.warmup + i, evs[i])
     t_end.record()
     barrier()
-    clocks = sampler.stop()
+    wall1 = time.time()
+    clocks = sampler.stop((wall0, wall1))
     total_ms = t_start.elapsed_time(t_end)
     fwd_ms = float(np.mean([e[0].elapsed_time(e[1]) for e in evs]))
     bwd_ms = float(np.mean([e[1].elapsed_time(e[2]) for e in evs]))
+    apply_ms = float(np.mean([e[2].elapsed_time(e[3]) for e in evs])) if dp_step else 0.0
+    if dp_step and not robe.dp.replicas_identical(array):
+        raise RuntimeError("the replicas of the array differ after the data-parallel steps")
     nnz_per_step = float(np.mean([len(batches[(args.warmup + i) % NB][0]) for i in range(args.steps)]))
 
     # ---- end to end: host buffers in, result out, every step ------------------------------
@@ -408,6 +449,9 @@ def run_ours(args, w):
         else:
             robe.robe_forward(h, ids_d, e_offs[b], B, e_out[b], stream=s_comp)
             robe.robe_backward(h, e_grad[b], ids_d, e_offs[b], B, dense, lr, ws, stream=s_comp)
+        if dp_step:
+            with torch.cuda.stream(s_comp):
+                exchange_and_apply()
         ev_comp[b].record(s_comp)
         with torch.cuda.stream(s_out):
             s_out.wait_event(ev_comp[b])
@@ -432,8 +476,8 @@ def run_ours(args, w):
     d2h = int(4 * nbags * d)
 
     # ---- max over ranks --------------------------------------------------------------------
-    (total_ms, e2e_ms, fwd_ms, bwd_ms), (job_ids, job_e2e_ids) = aggregate_over_ranks(
-        dist, dev, [total_ms, e2e_ms, fwd_ms, bwd_ms],
+    (total_ms, e2e_ms, fwd_ms, bwd_ms, apply_ms), (job_ids, job_e2e_ids) = aggregate_over_ranks(
+        dist, dev, [total_ms, e2e_ms, fwd_ms, bwd_ms, apply_ms],
         [nnz_per_step * args.steps, e2e_nnz * e2e_steps])
 
     robe.robe_destroy(h)
@@ -444,20 +488,45 @@ def run_ours(args, w):
 
     peak, peak_kind = measured_peaks()
     fwd_bytes, bwd_bytes = algorithmic_bytes(w, nbags, nnz_per_step, bags, id_bytes)
-    dominant = "backward" if bwd_ms >= fwd_ms else "forward"
-    bwd_label = {"atomic": "backward (bwd_atomic_staged_kernel)",
-                 "binned": "backward (keys, count, scan, scatter, binned_apply kernels together)",
-                 "det": "backward (keys, sort passes, apply kernels together)"}[args.backward]
+    fwd_kernel = "fwd_staged_kernel" if d <= 128 else "fwd_direct_kernel"
+    bwd_label = {"atomic": "bwd_atomic_staged_kernel" if d <= 128 else "bwd_atomic_direct_kernel",
+                 "binned": "composite: keys, sort_count, sort_scan, sort_scatter, binned_apply kernels",
+                 "det": "composite: keys, sort passes, window bounds/classes, apply kernels"}[args.backward]
     if share_keys:
-        bwd_label = bwd_label.replace("(keys, ", "(")
-    dom_bytes, dom_ms = (bwd_bytes, bwd_ms) if dominant == "backward" else (fwd_bytes, fwd_ms)
-    traffic = NCU_TRAFFIC_BYTES.get((w.name, args.backward, bool(share_keys)), {}) if args.ids == "int64" else {}
+        bwd_label = bwd_label.replace("keys, ", "")
+    # a traffic record applies to the configuration it was captured on, and to no other
+    own_batch = args.batch == 0
+    rec = NCU_TRAFFIC_RECORDS.get((w.name, args.backward, bool(share_keys), args.ids, args.bag_layout)) \
+        if (own_batch and not dp_step and world == 1) else None
+    sm_mhz = clocks.get("sm_mhz")
 
-    def roof(nbytes, ms, which):
+    def roof(nbytes, ms, kernel, which):
         ach = nbytes / (ms * 1e-3) / 1e9
-        return {"kernel": which, "bound": "hbm", "achieved": ach, "peak": peak, "unit": "GB/s",
-                "frac": ach / peak, "peak_kind": f"of {peak_kind}", "traffic": traffic.get(which),
-                "ms_per_launch": ms, "algorithmic_bytes": int(nbytes)}
+        r = {"kernel": kernel, "bound": "hbm", "achieved": ach, "peak": peak, "unit": "GB/s",
+             "frac": ach / peak, "peak_kind": f"of {peak_kind}",
+             "traffic": rec[which] if rec else None,
+             "traffic_source": rec["source"] if rec else None,
+             "ms_per_launch": ms, "algorithmic_bytes": int(nbytes)}
+        if sm_mhz:
+            r["ms_x_sm_mhz"] = ms * sm_mhz
+        return r
+
+    # The binned and the deterministic backward are built to keep the array's read-modify-write in
+    # L2, so next to the survey's model (every add reads and writes its slot in HBM) they are also
+    # read against the bytes such a path must move: ids, the block starts and payloads written and
+    # read once per sort pass, one read and one write of the touched part of the array, and the
+    # gradient elements once per id.
+    touched = min(float(w.M), nnz_per_step * d) * 4
+    npass_keys = {"atomic": 0, "binned": 1, "det": -(-max(1, (w.M - 1).bit_length()) // 8)}[args.backward]
+    blocks = nnz_per_step * (-(-d // min(w.Z, d)))
+    # per block: start and payload written once (8 B) and read by the apply (8 B); per sort pass
+    # the starts read by the count (4 B), both read (8 B) and written (8 B) by the scatter
+    key_bytes = blocks * (16 + 20 * npass_keys) if npass_keys else 0
+    l2_rmw_bytes = (id_bytes * nnz_per_step + (8 * (nbags + 1) if bags else 0) + 2 * touched
+                    + 4 * d * nnz_per_step + key_bytes)
+    roof_b = roof(bwd_bytes, bwd_ms, bwd_label, "backward")
+    roof_b["algorithmic_bytes_l2_rmw"] = int(l2_rmw_bytes)
+    roof_b["frac_l2_rmw"] = l2_rmw_bytes / (bwd_ms * 1e-3) / 1e9 / peak
 
     value = job_ids / (total_ms * 1e-3)
     array_mb = w.M * (4 if w.array_dtype == "f32" else 2) / 1e6
@@ -467,32 +536,44 @@ def run_ours(args, w):
     else:
         l2_note = (f"{array_mb:.0f} MB array stays L2-warm on purpose (steady state of a model that fits L2); "
                    f"the {stream_mb:.0f} MB of ids, output and gradient streamed per step exceed L2; no flush")
+    if dp_step:
+        parallelism = f"dp{world}, all-reduce of the dense gradient ({4 * w.M} bytes per rank and step), dense SGD apply"
+    else:
+        parallelism = f"dp{world}: one replica, fused SGD, nothing to exchange" if world == 1 else \
+            f"dp{world} replicas, no collective"
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": w.name, "num_tables": T, "d": d, "Z": w.Z, "M": w.M, "batch_per_gpu": B,
-                   "ids_per_step_per_gpu": nnz_per_step, "ids": args.ids, "bags": bags, "bag_layout": args.bag_layout, "backward": {"atomic": "atomic", "det": "deterministic", "binned": "binned atomic"}[args.backward] +
-                   (", SGD fused" if dense is None else ", dense fp32 gradient"),
+                   "ids_per_step_per_gpu": nnz_per_step, "ids": args.ids, "bags": bags, "bag_layout": args.bag_layout,
+                   "backward": {"atomic": "atomic", "det": "deterministic", "binned": "binned atomic"}[args.backward] +
+                   (", SGD fused" if dense is None else (", dense fp32 gradient, all-reduce, dense SGD apply" if dp_step
+                                                         else ", dense fp32 gradient")),
                    "block_starts": ("hashed once per step: kept by the forward for the backward" if share_keys
                                     else "hashed by the forward and again by the backward"),
                    "l2": l2_note,
-                   "parallelism": f"dp{world} replicas, no collective"},
+                   "parallelism": parallelism},
         "clocks": clocks,
         "e2e": {"value": job_e2e_ids / (e2e_ms * 1e-3), "unit": UNIT,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
                 "ms_per_step": e2e_ms / e2e_steps},
-        "gpu_launches": (1 + bwd_launches) * args.steps,
-        "roofline": roof(dom_bytes, dom_ms, dominant),
-        "roofline_forward": roof(fwd_bytes, fwd_ms, "forward"),
-        "roofline_backward": roof(bwd_bytes, bwd_ms, "backward"),
-        "kernels": {"forward": "fwd_staged_kernel", "backward": bwd_label},
+        "gpu_launches": (1 + bwd_launches + (1 if dp_step else 0)) * args.steps,
+        # ONE kernel: the forward gather (the largest single kernel of the step by the ncu launch
+        # list under profiles/, and the kernel the >= 0.60 target is stated for)
+        "roofline": roof(fwd_bytes, fwd_ms, fwd_kernel, "forward"),
+        "roofline_backward": roof_b,
         "forward_models": {k: {"bytes": int(v), "GB/s": v / (fwd_ms * 1e-3) / 1e9,
                                "frac": v / (fwd_ms * 1e-3) / 1e9 / peak}
                            for k, v in forward_byte_models(w, nbags, nnz_per_step, bags, id_bytes).items()},
         "forward_only": {"value": world * nnz_per_step / (fwd_ms * 1e-3), "unit": UNIT,
                          "bags_per_s": world * nbags / (fwd_ms * 1e-3), "ms": fwd_ms},
     }
+    if dp_step:
+        # all-reduce + apply together (the collective runs in the process group's own stream between
+        # two events of the compute stream); the apply alone moves 12 bytes per slot
+        line["exchange_and_apply"] = {"ms": apply_ms, "apply_algorithmic_bytes": 12 * w.M,
+                                      "allreduce_bytes_per_rank": 4 * w.M}
     if not args.no_cpu_baseline and world == 1:
         sample_batch = w.batch  # about 10 s of host work on the default workload
         rate, n, threads, dt = oracle_step_rate(w, sample_batch, synth.array_to_numpy(array), variant=7)
@@ -519,6 +600,9 @@ def main():
     ap.add_argument("--bag-layout", default="sample-major", choices=["sample-major", "table-major"],
                     help="bag numbering of the inputs: n*T + e (default) or e*B + n (per-table id lists end to end)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--dp-step", default="auto", choices=["auto", "on", "off"],
+                    help="data-parallel step (backward into a dense gradient, all-reduce over the ranks, dense "
+                         "SGD apply) instead of the fused SGD step; auto = on with more than one rank")
     ap.add_argument("--no-share-keys", dest="share_keys", action="store_false",
                     help="hash the ids in the backward again (robe_forward + robe_backward) instead of "
                          "keeping the forward's block starts (robe_forward_keep + robe_backward_kept)")

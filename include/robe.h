@@ -56,7 +56,13 @@ typedef enum {
 #define ROBE_OPT_BWD_MODE 2 /* ROBE_BWD_ATOMIC (default) | ROBE_BWD_DETERMINISTIC | ROBE_BWD_BINNED */
 #define ROBE_OPT_VALIDATE 3 /* 0 (default) | 1: range-check ids/offsets on the device and
                                record the first violation in a status word instead of
-                               using the bad value                                        */
+                               using the bad value.  The word is sticky: while it is
+                               non-zero EVERY kernel of EVERY later call on the handle
+                               returns at once - robe_forward leaves `out` as it was
+                               (not overwritten), robe_forward_keep keeps nothing, the
+                               backward calls add nothing - and the host call still
+                               returns ROBE_OK.  Read it with robe_last_device_status
+                               and zero it yourself before going on.                      */
 #define ROBE_OPT_FWD_KERNEL 4 /* 0 = automatic (default); other values pick one forward
                                  kernel variant, for benchmarking only                    */
 #define ROBE_OPT_BWD_KERNEL 5 /* same for the atomic backward                             */
@@ -105,8 +111,10 @@ typedef enum {
  *               redrawn when outside [1,P-1] for multipliers / [0,P-1] for the
  *               additive terms), as the paper's hash family requires.
  * A handle holds options and, after the first deterministic backward, a CUDA stream and two
- * events of its own (no device memory): calls on ONE handle must not overlap in time on the
- * host; different handles are independent.
+ * events of its own (no device memory) on the device that was current at that call; a
+ * deterministic backward made later with another device current runs in the caller's stream
+ * alone.  Calls on ONE handle must not overlap in time on the host; different handles are
+ * independent.
  * Errors: ROBE_ERR_INVALID_ARG.
  */
 int robe_create(robe_handle_t* out, uint64_t M, uint32_t Z, uint32_t d, uint32_t num_tables,
@@ -120,8 +128,8 @@ int robe_destroy(robe_handle_t h);
 int robe_set_option(robe_handle_t h, int key, int64_t value);
 
 /*
- * robe_attach_array - name the parameter array M (Section 3: "a single array for
- * learned parameters" shared by all tables).
+ * robe_attach_array - name the parameter array M (Section 3: the one array that holds the
+ * learned parameters of all tables).
  *   dev_array  device pointer to M elements of `dtype`, 16-byte aligned, owned by the
  *              caller, read by forward and updated in place by the fused-SGD backward.
  *   dtype      ROBE_F32 or ROBE_BF16 (bf16 is read-only: widened exactly to fp32).
@@ -239,6 +247,24 @@ int robe_backward_adam(robe_handle_t h, const float* grad_out, const void* indic
                        size_t workspace_bytes, void* stream);
 
 /*
+ * robe_apply_sgd - the dense SGD apply of a data-parallel training step (Section 1 of the
+ * paper, implications of the compression: the whole model fits every GPU, so training is plain
+ * data-parallel and the ranks exchange one gradient the size of the array; Section 5: SGD).
+ * A rank runs robe_backward with a dense grad_array on its shard of the batch, the caller
+ * sums grad_array over the ranks (an all-reduce: 4 M bytes), and this call applies the sum
+ *     M[j] <- fma(-lr, grad_array[j], M[j])       for every j < M
+ * to the attached fp32 array in one streaming pass.  On one rank it gives the bits of the
+ * fused step (robe_backward with grad_array == NULL) when grad_array held +0 before the
+ * deterministic backward ran.
+ *   grad_array  device pointer, fp32 [M], 16-byte aligned; with zero_grad = 1 it is left
+ *               holding +0 everywhere, ready for the next step's robe_backward.
+ *   zero_grad   0 or 1.
+ * Errors: ROBE_ERR_INVALID_ARG (null or misaligned pointer, bf16 array), ROBE_ERR_NO_ARRAY,
+ * ROBE_ERR_CUDA.
+ */
+int robe_apply_sgd(robe_handle_t h, float* grad_array, float lr, int zero_grad, void* stream);
+
+/*
  * robe_backward_deterministic_static - the deterministic robe_backward for callers that
  * cannot supply scratch memory.  (The paper has no counterpart: this is a convenience of
  * this library, not part of the method.)
@@ -260,7 +286,8 @@ int robe_backward_adam(robe_handle_t h, const float* grad_out, const void* indic
  *
  * Limit: the call must fit the fixed array, i.e. the value robe_backward_workspace_bytes
  * reports for it in deterministic mode (about 19 bytes per block, nnz * ceil(d/Z) blocks,
- * plus 4 bytes per id and 0.7 MB of counters and lists) must not exceed
+ * plus 4 bytes per id, 0.7 MB of counters and lists, and the window bounds of the array:
+ * M/57 bytes for arrays under 2 M slots, M/228 bytes above) must not exceed
  * ROBE_STATIC_SCRATCH_BYTES; a larger call returns ROBE_ERR_WORKSPACE and launches nothing.
  *
  * First call on a device: the function looks up the device address of the array once per
@@ -284,7 +311,10 @@ int robe_backward_deterministic_static(robe_handle_t h, const float* grad_out,
 
 /*
  * robe_set_status_word - give the handle a device int32 (caller-owned, zeroed by the
- * caller) that kernels write a ROBE_DEV_* code into when ROBE_OPT_VALIDATE is on.
+ * caller) that kernels write a ROBE_DEV_* code into when ROBE_OPT_VALIDATE is on.  Only the
+ * first violation is recorded (compare-and-swap from ROBE_DEV_OK), and a non-zero word turns
+ * all later launches on the handle into no-ops until the caller zeroes it (see
+ * ROBE_OPT_VALIDATE).
  * robe_last_device_status - synchronise `stream`, read that word (device-to-host copy)
  * and return it (>= 0), or a negative robe_status.
  */

@@ -20,15 +20,15 @@
  *     of Section 3.2 has a misplaced parenthesis).
  *   - "(..) mod P mod |M|" is ((..) mod P) mod |M|.
  *   - e, x, c and i are 0-based.
- *   - P = 2^61 - 1 (the paper only says "a large prime"); the multipliers are in
- *     [1, P-1], the additive terms in [0, P-1] (Section 3.2 statement).
+ *   - P = 2^61 - 1 (Section 3.2 asks for a large prime and names none); the
+ *     multipliers are in [1, P-1], the additive terms in [0, P-1] (Section 3.2).
  *   - the sign hash g is optional and off by default (Section 4.1 and the
  *     appendix both say it is not used in practice).
  *   - pooling over a bag is a sequential fp32 sum in bag order (the paper's data
  *     are one-hot, so this part is a definition of this library, not the paper's).
- *   - Z > d (Section 3.2, last paragraph: "clubbing multiple embeddings together
- *     in a chunk"; the appendix cuts the row-wise flattened table into chunks of
- *     Z) is taken for d dividing Z: R = Z/d consecutive rows of a table share one
+ *   - Z > d (Section 3.2, last paragraph: a chunk may span several embeddings;
+ *     the appendix cuts the row-wise flattened table into chunks of Z) is taken
+ *     for d dividing Z: R = Z/d consecutive rows of a table share one
  *     block, row x is the piece [(x mod R) d, (x mod R) d + d) of the block that
  *     starts at h(e, floor(x/R), 0).
  *
@@ -57,7 +57,7 @@ typedef unsigned __int128 u128;
 /* Index layout of the nine constants every function takes. */
 enum { K_P = 0, K_AH, K_BH, K_CH, K_DH, K_AG, K_BG, K_CG, K_DG };
 
-/* ---- constants (Section 3.2: P a large prime, A,B,C in 1..P-1, D in 0..P-1) ---- */
+/* ---- constants (Section 3.2: P prime and large, A,B,C in 1..P-1, D in 0..P-1) ---- */
 
 static uint64_t mix_next(uint64_t *state) {
     /* SplitMix64 step (published generator by Steele, Lea, Flood). */
@@ -336,6 +336,13 @@ void robe_oracle_sgd_apply(float *array, const float *delta, const uint8_t *touc
                            float lr) {
     for (uint64_t j = 0; j < n; ++j)
         if (touched[j]) array[j] = fmaf(-lr, delta[j], array[j]);
+}
+
+/* Dense SGD apply of the data-parallel step (Section 1: the compressed model is trained
+   data-parallel, the ranks exchanging one gradient the size of the array; Section 5: SGD):
+   M[j] <- fma(-lr, g[j], M[j]) for EVERY slot, g being the gradient summed over the ranks. */
+void robe_oracle_dense_sgd_apply(float *array, const float *grad, uint64_t n, float lr) {
+    for (uint64_t j = 0; j < n; ++j) array[j] = fmaf(-lr, grad[j], array[j]);
 }
 
 /* Dense accumulation used by the deterministic variant: ga[j] <- ga[j] + delta[j]

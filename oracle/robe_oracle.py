@@ -57,6 +57,7 @@ def lib() -> C.CDLL:
         _lib.robe_oracle_backward_canonical.restype = C.c_int
         _lib.robe_oracle_sgd_apply.argtypes = [p, p, p, u64, C.c_float]
         _lib.robe_oracle_accumulate.argtypes = [p, p, p, u64]
+        _lib.robe_oracle_dense_sgd_apply.argtypes = [p, p, u64, C.c_float]
         _lib.robe_oracle_adam_apply.argtypes = [p, p, p, p, p, u64] + [C.c_float] * 6
     return _lib
 
@@ -173,6 +174,12 @@ def sgd_apply(array, delta, touched, lr) -> None:
     """In place: array[j] = fma(-lr, delta[j], array[j]) on touched slots."""
     assert array.dtype == np.float32 and delta.dtype == np.float32 and touched.dtype == np.uint8
     lib().robe_oracle_sgd_apply(_ptr(array), _ptr(delta), _ptr(touched), len(delta), C.c_float(lr))
+
+
+def dense_sgd_apply(array, grad, lr) -> None:
+    """In place: array[j] = fma(-lr, grad[j], array[j]) on every slot (data-parallel step)."""
+    assert array.dtype == np.float32 and grad.dtype == np.float32 and len(array) == len(grad)
+    lib().robe_oracle_dense_sgd_apply(_ptr(array), _ptr(grad), len(array), C.c_float(lr))
 
 
 def accumulate(grad_array, delta, touched) -> None:

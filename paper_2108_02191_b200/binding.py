@@ -49,7 +49,7 @@ EXPORTS = [
     "robe_get_hash_constants", "robe_forward", "robe_backward_workspace_bytes", "robe_backward",
     "robe_set_status_word", "robe_last_device_status", "robe_status_string",
     "robe_backward_deterministic_static", "robe_backward_adam",
-    "robe_forward_keep", "robe_backward_kept",
+    "robe_forward_keep", "robe_backward_kept", "robe_apply_sgd",
 ]
 
 if not os.path.exists(LIB_PATH):
@@ -74,6 +74,7 @@ _lib.robe_backward_kept.argtypes = list(_lib.robe_backward.argtypes)
 _lib.robe_backward_deterministic_static.argtypes = [_vp, _vp, _vp, _vp, _i64, _i64, _vp, C.c_float, _vp]
 _lib.robe_backward_adam.argtypes = [_vp, _vp, _vp, _vp, _i64, _i64, _vp, _vp, C.c_float, C.c_float,
                                     C.c_float, C.c_float, _i64, _vp, C.c_size_t, _vp]
+_lib.robe_apply_sgd.argtypes = [_vp, _vp, C.c_float, C.c_int, _vp]
 _lib.robe_set_status_word.argtypes = [_vp, _vp]
 _lib.robe_last_device_status.argtypes = [_vp, _vp]
 _lib.robe_status_string.argtypes = [C.c_int]
@@ -226,6 +227,12 @@ def robe_backward_adam(h, grad_out, indices, offsets, batch: int, m1, m2, lr: fl
         step, _dev_ptr(workspace), ws_bytes, _stream_ptr(stream)), "robe_backward_adam")
 
 
+def robe_apply_sgd(h, grad_array, lr: float, zero_grad: bool = True, stream=None) -> None:
+    """Dense SGD apply of the data-parallel step: array <- fma(-lr, grad_array, array)."""
+    _check(_lib.robe_apply_sgd(h, _dev_ptr(grad_array, torch.float32), lr, 1 if zero_grad else 0,
+                               _stream_ptr(stream)), "robe_apply_sgd")
+
+
 def robe_set_status_word(h, word) -> None:
     _check(_lib.robe_set_status_word(h, _dev_ptr(word, torch.int32)), "robe_set_status_word")
 
@@ -234,8 +241,7 @@ def robe_last_device_status(h, stream=None) -> int:
     return int(_lib.robe_last_device_status(h, _stream_ptr(stream)))
 
 
-# Host-pointer variants of forward/backward calls for callers that drive the C ABI with raw
-# addresses (the benchmark's end-to-end leg uses torch tensors like everything else).
 def raw():
-    """The ctypes library object itself."""
+    """The ctypes library object itself, for callers that drive the C ABI with raw addresses
+    (the host-side argument tests do)."""
     return _lib

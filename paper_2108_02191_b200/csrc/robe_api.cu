@@ -31,6 +31,7 @@ struct robe_ctx {
     int bag_layout;
     // second stream of the deterministic backward, made at the first call that can use it
     bool side_tried;
+    int side_device;  // the device the stream and events below belong to
     cudaStream_t side;
     cudaEvent_t fork_event, join_event;
 };
@@ -109,8 +110,14 @@ Problem make_problem(robe_ctx* h, const void* indices, const int64_t* offsets, i
 // caller's stream by events.  Made once per handle; if that fails the kernels run one after the
 // other in the caller's stream.
 void lend_side_stream(robe_ctx* h, Problem& pb) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return;
+    }
     if (!h->side_tried) {
         h->side_tried = true;
+        h->side_device = dev;
         int least = 0, greatest = 0;
         cudaStream_t s = nullptr;
         cudaEvent_t e0 = nullptr, e1 = nullptr;
@@ -127,6 +134,9 @@ void lend_side_stream(robe_ctx* h, Problem& pb) {
             (void)cudaGetLastError();
         }
     }
+    // a stream belongs to the device it was made on: a call made with another device current
+    // runs everything in the caller's stream
+    if (dev != h->side_device) return;
     pb.side = h->side;
     pb.fork_event = h->fork_event;
     pb.join_event = h->join_event;
@@ -206,6 +216,7 @@ int robe_create(robe_handle_t* out, uint64_t M, uint32_t Z, uint32_t d, uint32_t
     h->index_type = ROBE_I64;
     h->bag_layout = ROBE_BAGS_SAMPLE_MAJOR;
     h->side_tried = false;
+    h->side_device = -1;
     h->side = nullptr;
     h->fork_event = h->join_event = nullptr;
     *out = h;
@@ -241,7 +252,7 @@ int robe_set_option(robe_handle_t h, int key, int64_t value) {
             h->validate = (int)value;
             return ROBE_OK;
         case ROBE_OPT_FWD_KERNEL:
-            if (value < 0 || value > 2) return ROBE_ERR_INVALID_ARG;
+            if (value < 0 || value > 3) return ROBE_ERR_INVALID_ARG;
             h->fwd_variant = (int)value;
             return ROBE_OK;
         case ROBE_OPT_INDEX_TYPE:
@@ -468,6 +479,18 @@ int robe_backward_adam(robe_handle_t h, const float* grad_out, const void* indic
     if (launch_validate(pb, st) != cudaSuccess) return ROBE_ERR_CUDA;
     if (launch_backward_det(pb, grad_out, (float*)h->array, 2, lr, &ad, workspace, workspace_bytes,
                             st) != cudaSuccess)
+        return ROBE_ERR_CUDA;
+    return ROBE_OK;
+}
+
+int robe_apply_sgd(robe_handle_t h, float* grad_array, float lr, int zero_grad, void* stream) {
+    if (h == nullptr || grad_array == nullptr) return ROBE_ERR_INVALID_ARG;
+    if (zero_grad != 0 && zero_grad != 1) return ROBE_ERR_INVALID_ARG;
+    if (h->array == nullptr) return ROBE_ERR_NO_ARRAY;
+    if (h->dtype != ROBE_F32) return ROBE_ERR_INVALID_ARG;
+    if (((uintptr_t)grad_array & 15u) != 0) return ROBE_ERR_INVALID_ARG;
+    if (launch_dense_sgd_apply((float*)h->array, grad_array, h->M, lr, zero_grad != 0,
+                               (cudaStream_t)stream) != cudaSuccess)
         return ROBE_ERR_CUDA;
     return ROBE_OK;
 }

@@ -218,6 +218,163 @@ fwd_staged_kernel(FwdArgs a, uint32_t ids_per_batch, uint32_t cmagic) {
     }
 }
 
+// Vector kernel: fp32 array, d, Z and m multiples of four, d <= 128.  The staging and the hash
+// phase are those of the staged kernel; the gather reads 16 bytes per load.  A block starts at
+// an arbitrary element, so its elements 4k .. 4k+3 (output vector k of the row) lie in the two
+// ALIGNED 16-byte pieces around them: the lane loads both (only the first when the block start is
+// itself a multiple of four) and shifts the eight values by (start mod 4) in registers.  m is a
+// multiple of four, so an aligned piece never straddles the end of the array and the wrap-around
+// is a subtraction on the piece's slot number.  d/4 lanes serve one id; with d <= 64 the warp
+// serves 32 / (d/4) ids per load instruction, and the pooled sum still adds the ids in bag order:
+// the lanes of the first id hold the sum and fetch the other ids' vectors by shuffle, in order.
+__device__ __forceinline__ float4 ldg_f4_64B(const float* p) {
+    float4 v;
+    asm("ld.global.nc.L2::64B.v4.f32 {%0, %1, %2, %3}, [%4];"
+        : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+        : "l"(p));
+    return v;
+}
+
+// elements r .. r+3 of the eight values (lo, hi), r = 0 .. 3
+__device__ __forceinline__ float4 realign4(const float4 lo, const float4 hi, uint32_t r) {
+    float e0 = lo.x, e1 = lo.y, e2 = lo.z, e3 = lo.w, e4 = hi.x, e5 = hi.y, e6 = hi.z;
+    if (r & 2u) { e0 = e2; e1 = e3; e2 = e4; e3 = e5; e4 = e6; }
+    if (r & 1u) { e0 = e1; e1 = e2; e2 = e3; e3 = e4; }
+    return make_float4(e0, e1, e2, e3);
+}
+
+template <bool BAGS, bool WRAP, int U>
+__device__ __forceinline__ void vec_gather_batch(const FwdArgs& a, const uint32_t* col, uint32_t o,
+                                                 uint32_t cnt, int64_t p0, uint32_t lpi, uint32_t ipi,
+                                                 uint32_t grp, uint32_t k, bool lane_on, float4& acc) {
+    const MapParams& mp = a.mp;
+    const float* array = (const float*)a.array;
+    for (uint32_t g0 = 0; g0 < cnt; g0 += ipi * U) {
+        float4 v[U];
+#pragma unroll
+        for (int gg = 0; gg < U; ++gg) {
+            const uint32_t t = g0 + gg * ipi + grp;
+            v[gg] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+            if (lane_on && t < cnt) {
+                const uint32_t pos = col[t] + o;  // first slot of the vector, < m + d <= 2^32
+                const uint32_t r = pos & 3u;
+                uint32_t a0 = pos & ~3u;
+                if (WRAP && a0 >= mp.m) a0 -= mp.m;
+                const float4 lo = ldg_f4_64B(array + a0);
+                float4 hi = lo;
+                if (r != 0) {
+                    uint32_t a1 = a0 + 4u;
+                    if (WRAP && a1 >= mp.m) a1 -= mp.m;
+                    hi = ldg_f4_64B(array + a1);
+                }
+                v[gg] = realign4(lo, hi, r);
+            }
+        }
+        if (BAGS) {
+#pragma unroll
+            for (int gg = 0; gg < U; ++gg) {
+                for (uint32_t gs = 0; gs < ipi; ++gs) {
+                    if (g0 + gg * ipi + gs >= cnt) break;  // warp-uniform
+                    float4 x = v[gg];
+                    if (gs != 0) {  // the vector of a later id of this load: from its lanes
+                        const int src = (int)(k + gs * lpi);
+                        x.x = __shfl_sync(0xFFFFFFFFu, v[gg].x, src);
+                        x.y = __shfl_sync(0xFFFFFFFFu, v[gg].y, src);
+                        x.z = __shfl_sync(0xFFFFFFFFu, v[gg].z, src);
+                        x.w = __shfl_sync(0xFFFFFFFFu, v[gg].w, src);
+                    }
+                    acc.x = acc.x + x.x;
+                    acc.y = acc.y + x.y;
+                    acc.z = acc.z + x.z;
+                    acc.w = acc.w + x.w;
+                }
+            }
+        } else {
+#pragma unroll
+            for (int gg = 0; gg < U; ++gg) {
+                const uint32_t t = g0 + gg * ipi + grp;
+                if (lane_on && t < cnt)
+                    __stcs(reinterpret_cast<float4*>(a.out + (p0 + t) * (int64_t)mp.d) + k, v[gg]);
+            }
+        }
+    }
+}
+
+template <bool BAGS, int U>
+__global__ void __launch_bounds__(256, 5)
+fwd_vec_kernel(FwdArgs a, uint32_t ids_per_batch, uint32_t cmagic) {
+    __shared__ StageSmem sm;
+    const MapParams& mp = a.mp;
+    const uint32_t lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const int64_t warp = (int64_t)blockIdx.x * 8 + w;
+
+    stage_init(sm, mp);
+    if (a.status != nullptr && *a.status != 0) return;
+
+    int64_t lo, hi;
+    uint64_t tterm = 0;
+    if (BAGS) {
+        if (warp >= a.nbags) return;
+        bag_range(a.offsets, a.nnz, warp, lo, hi);
+        tterm = table_term(mp.h, table_of_bag((uint64_t)warp, mp));
+    } else {
+        lo = warp * (int64_t)ids_per_batch;
+        if (lo >= a.nbags) return;
+        hi = lo + ids_per_batch < a.nbags ? lo + ids_per_batch : a.nbags;
+    }
+    if (BAGS && a.keep_keys != nullptr) {  // (as in the staged kernel)
+        const int64_t C = (int64_t)mp.C;
+        if (warp == 0)
+            for (int64_t q = lane; q < lo * C; q += 32) a.keep_keys[q] = a.keep_vals[q] = 0;
+        if (warp == a.nbags - 1)
+            for (int64_t q = hi * C + lane; q < a.nnz * C; q += 32) a.keep_keys[q] = a.keep_vals[q] = 0;
+    }
+
+    const uint32_t lpi = mp.d >> 2;   // lanes per id = output vectors per row
+    const uint32_t ipi = 32u / lpi;   // ids per load instruction
+    const uint32_t grp = lane / lpi;  // which of them this lane reads
+    const uint32_t k = lane - grp * lpi;
+    const bool lane_on = grp < ipi;
+    uint32_t chk, o;
+    chunk_of(mp, 4u * k, chk, o);
+    const uint32_t* col = sm.start[w] + chk * ids_per_batch;
+
+    float4 acc = make_float4(-0.0f, -0.0f, -0.0f, -0.0f);  // -0 + v == v: the first term initialises
+    for (int64_t p0 = lo; p0 < hi; p0 += ids_per_batch) {
+        const uint32_t cnt = (uint32_t)((hi - p0) < (int64_t)ids_per_batch ? (hi - p0)
+                                                                            : (int64_t)ids_per_batch);
+        const bool wraps = stage_batch<false, BAGS>(sm, mp, a.indices, p0, cnt, ids_per_batch, tterm, 0,
+                                                    cmagic, w, lane,
+                                                    KeepBlocks{a.keep_keys, a.keep_vals, (uint64_t)warp});
+        if (wraps)
+            vec_gather_batch<BAGS, true, U>(a, col, o, cnt, p0, lpi, ipi, grp, k, lane_on, acc);
+        else
+            vec_gather_batch<BAGS, false, U>(a, col, o, cnt, p0, lpi, ipi, grp, k, lane_on, acc);
+        __syncwarp();
+    }
+    if (BAGS && grp == 0) {
+        const bool empty = hi <= lo;
+        if (empty) acc = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+        __stcs(reinterpret_cast<float4*>(a.out + warp * (int64_t)mp.d) + k, acc);
+    }
+}
+
+// what the vector kernel asks of a call
+static bool vec_kernel_ok(const Problem& pb, const float* out) {
+    const MapParams& mp = pb.mp;
+    return pb.dtype == 0 && pb.sign == 0 && mp.d <= 128 && mp.d % 4 == 0 && mp.Z % 4 == 0 && mp.m % 4 == 0 &&
+           ((uintptr_t)out & 15u) == 0 && ((uintptr_t)pb.array & 15u) == 0;
+}
+
+static void launch_vec(const FwdArgs& a, bool bags, cudaStream_t st) {
+    const uint32_t ipb = staged_ids_per_batch(a.mp, bags, false);
+    const uint32_t cmagic = chunk_magic(a.mp);
+    const int64_t warps = bags ? a.nbags : (a.nbags + ipb - 1) / ipb;
+    const unsigned blocks = (unsigned)((warps + 7) / 8);
+    if (bags) fwd_vec_kernel<true, 4><<<blocks, 256, 0, st>>>(a, ipb, cmagic);
+    else fwd_vec_kernel<false, 4><<<blocks, 256, 0, st>>>(a, ipb, cmagic);
+}
+
 // Ids whose loads are in flight together (U) and resident CTAs per SM the register budget is set
 // for (MINB).  Measured on B200: the time of the HBM-resident gather does not move between 4 and 16
 // ids in flight or between 4 and 8 CTAs per SM - the random 64-byte requests themselves are the
@@ -269,6 +426,12 @@ cudaError_t launch_forward(const Problem& pb, float* out, int variant, cudaStrea
     const bool bags = pb.offsets != nullptr;
     const bool warp_ok = pb.mp.d <= 128;
     if (variant == 2 && !warp_ok) return cudaErrorInvalidValue;
+    if (variant == 3) {  // the kernel with 16-byte loads
+        if (!vec_kernel_ok(pb, out)) return cudaErrorInvalidValue;
+        if (kept != nullptr) *kept = keep_keys != nullptr;
+        launch_vec(a, bags, st);
+        return cudaGetLastError();
+    }
     const bool use_warp = variant == 2 || (variant == 0 && warp_ok);
     if (use_warp) {
         if (kept != nullptr) *kept = keep_keys != nullptr;  // (the direct kernel keeps nothing)

@@ -61,6 +61,11 @@ void block_key_buffers(const Problem& pb, void* workspace, uint32_t** keys, uint
 cudaError_t launch_block_keys(const Problem& pb, void* workspace, size_t workspace_bytes,
                               cudaStream_t st);
 
+// dense SGD apply of the data-parallel step: array[j] = fma(-lr, grad[j], array[j]) for j < m,
+// grad zeroed afterwards when zero_grad
+cudaError_t launch_dense_sgd_apply(float* array, float* grad, uint64_t m, float lr, bool zero_grad,
+                                   cudaStream_t st);
+
 // id / offset range check into the status word
 cudaError_t launch_validate(const Problem& pb, cudaStream_t st);
 

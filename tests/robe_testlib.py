@@ -83,13 +83,13 @@ class Case:
         torch.cuda.synchronize()
         return grad_array
 
-    def step_sharing_keys(self, grad_out: torch.Tensor, mode, sgd=False, lr=0.0):
+    def step_sharing_keys(self, grad_out: torch.Tensor, mode, sgd=False, lr=0.0, fwd_kernel=0):
         """robe_forward_keep then robe_backward_kept on the same workspace: (out, dense gradient
         or None)."""
         robe.robe_set_option(self.h, robe.ROBE_OPT_BWD_MODE,
                              {"atomic": robe.ROBE_BWD_ATOMIC, "det": robe.ROBE_BWD_DETERMINISTIC,
                               "binned": robe.ROBE_BWD_BINNED}[mode])
-        robe.robe_set_option(self.h, robe.ROBE_OPT_FWD_KERNEL, 0)
+        robe.robe_set_option(self.h, robe.ROBE_OPT_FWD_KERNEL, fwd_kernel)
         robe.robe_set_option(self.h, robe.ROBE_OPT_BWD_KERNEL, 0)
         ws = None
         nbytes = robe.robe_backward_workspace_bytes(self.h, self.B, self.indices.numel())

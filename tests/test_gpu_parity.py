@@ -63,6 +63,43 @@ def test_forward_shapes(d, Z, M, bags):
                     c.forward(2)
 
 
+# The kernel with 16-byte loads (ROBE_OPT_FWD_KERNEL = 3): fp32 array, d, Z and M multiples of
+# four, sign off.  Shapes: every lanes-per-id count (d/4 = 1 .. 32, powers of two and not), blocks
+# of one vector and of many, arrays so short that every batch wraps, rows clubbed into one block.
+VEC_SHAPES = [(16, 4, 1000), (16, 4, 20), (16, 16, 16), (64, 16, 68), (64, 16, 250_000), (128, 32, 132),
+              (128, 128, 128), (128, 128, 100_004), (128, 4, 4096), (32, 8, 36), (96, 32, 100), (100, 20, 1000),
+              (12, 4, 64), (8, 8, 8), (4, 4, 4), (48, 12, 52), (16, 64, 1000), (64, 128, 5000), (128, 8, 262_144)]
+
+
+@pytest.mark.parametrize("bags", [None, (3, 0, 9), (20, 1, 80)])
+@pytest.mark.parametrize("d,Z,M", VEC_SHAPES)
+def test_forward_vector_kernel(d, Z, M, bags):
+    w = small(d=d, Z=Z, M=M, bag_rule=bags, batch=97)
+    with Case(w) as c:
+        want = c.oracle_forward()
+        assert_bits_equal(c.forward(3).cpu().numpy(), want, f"vector kernel d={d} Z={Z} M={M}")
+        # int32 ids and the forward that keeps its block starts go through the same kernel
+        g_h, g_d = _grad(c, 4)
+        can, _ = c.oracle.backward_canonical(g_h, c.indices_h, c.offsets_h, c.B)
+        robe.robe_set_option(c.h, robe.ROBE_OPT_FWD_KERNEL, 3)
+        out, det = c.step_sharing_keys(g_d, "det", fwd_kernel=3)
+        assert_bits_equal(out.cpu().numpy(), want, "vector kernel that keeps")
+        assert_bits_equal(det.cpu().numpy(), can, "deterministic on the vector kernel's kept starts")
+        c.indices = c.indices.to(torch.int32)
+        assert_bits_equal(c.forward(3).cpu().numpy(), want, "vector kernel, int32 ids")
+
+
+def test_forward_vector_kernel_refuses_what_it_cannot_do():
+    for kw in (dict(d=16, Z=4, M=1001), dict(d=16, Z=2, M=1000), dict(d=18, Z=6, M=1000),
+               dict(d=16, Z=4, M=1000, array_dtype="bf16"), dict(d=256, Z=4, M=1000)):
+        with Case(small(**kw)) as c:
+            with pytest.raises(robe.RobeError):
+                c.forward(3)
+    with Case(small(), sign=True) as c:
+        with pytest.raises(robe.RobeError):
+            c.forward(3)
+
+
 def test_forward_bf16_array():
     w = small(array_dtype="bf16", d=64, Z=16, M=5000, bag_rule=(4, 0, 12))
     with Case(w) as c:
@@ -437,8 +474,8 @@ def _sample_bags(nbags, n, seed):
     return np.sort(picks).astype(np.int64)
 
 
-def _check_forward_sampled(c, nsample=20000):
-    got = c.forward().reshape(c.nbags, c.w.d)
+def _check_forward_sampled(c, nsample=20000, kernel=0):
+    got = c.forward(kernel).reshape(c.nbags, c.w.d)
     bags = _sample_bags(c.nbags, nsample, 1)
     want = c.oracle_forward_bags(bags)
     assert_bits_equal(got[torch.from_numpy(bags).to(c.dev)].cpu().numpy(), want, c.w.name + " forward")
@@ -449,7 +486,9 @@ def test_cfg2_forward_full_size():
     with Case(synth.workload(2)) as c:
         got = c.forward()
         # the whole output, not a sample: the oracle needs a few seconds for 1.7M rows
-        assert_bits_equal(got.cpu().numpy(), c.oracle_forward(), "cfg2 forward (all rows)")
+        want = c.oracle_forward()
+        assert_bits_equal(got.cpu().numpy(), want, "cfg2 forward (all rows)")
+        assert_bits_equal(c.forward(3).cpu().numpy(), want, "cfg2 forward, 16-byte loads (all rows)")
 
 
 @pytest.mark.parametrize("Z", [1, 128])
@@ -499,6 +538,7 @@ def test_cfg4_forward_backward_full_size():
     w = synth.workload(4)
     with Case(w) as c:
         _check_forward_sampled(c)
+        _check_forward_sampled(c, kernel=3)
         g_h = synth.make_grad_out(w)
         g_d = torch.from_numpy(g_h).to(c.dev)
         delta64, l1 = c.oracle.backward_f64(g_h, c.indices_h, c.offsets_h, c.B)
@@ -534,22 +574,31 @@ def test_cfg4_forward_backward_full_size():
         assert_bits_equal(detk.cpu().numpy(), det, "cfg4 det on kept starts")
 
 
-@pytest.mark.parametrize("M,Z,dtype", [
-    (262_144, 1, "f32"), (262_144, 32, "f32"), (25_000_000, 2, "f32"), (25_000_000, 8, "f32"),
-    (25_000_000, 128, "f32"), (25_000_000, 32, "bf16"),
-])
+# the sweep: every cell of {1 MB, 100 MB} x Z in {1, 2, 8, 32, 128}, and the bf16 array
+@pytest.mark.parametrize("M,Z,dtype",
+                         [(M, Z, "f32") for M in (262_144, 25_000_000) for Z in (1, 2, 8, 32, 128)]
+                         + [(25_000_000, 32, "bf16")])
 def test_cfg5_forward_full_size(M, Z, dtype):
     w = synth.workload(5, M=M, Z=Z, array_dtype=dtype)
     with Case(w) as c:
         _check_forward_sampled(c)
 
 
-@pytest.mark.parametrize("Z", [1, 32])
+def _need_device_memory(gib):
+    free, _ = torch.cuda.mem_get_info()
+    if free < gib * 2**30:
+        pytest.skip("not enough free device memory")
+
+
+def _array_window(w, j0, jn):
+    """fp32 values of array slots [j0, j0+jn) from the counter-based generator (host side)."""
+    return synth.array_values_at(w, torch.arange(j0, j0 + jn, dtype=torch.int64)).numpy()
+
+
+@pytest.mark.parametrize("Z", [1, 2, 8, 32, 128])
 def test_cfg5_forward_10gb_array(Z):
     w = synth.workload(5, M=2_500_000_000, Z=Z)
-    free, _ = torch.cuda.mem_get_info()
-    if free < 16 * 2**30:
-        pytest.skip("not enough free device memory")
+    _need_device_memory(16)
     with Case(w, host_array=False) as c:
         got = c.forward().reshape(c.nbags, w.d)
         bags = _sample_bags(c.nbags, 3000, 2)
@@ -571,6 +620,130 @@ def test_cfg5_backward_full_size():
         det = c.backward(g_d, "det").cpu().numpy()
         can, _ = c.oracle.backward_canonical(g_h, c.indices_h, c.offsets_h, c.B)
         assert_bits_equal(det, can, "cfg5 det")
+
+
+@pytest.mark.parametrize("M,Z,dtype", [(262_144, 1, "f32"), (262_144, 32, "f32"), (25_000_000, 1, "f32"),
+                                       (25_000_000, 128, "f32"), (25_000_000, 32, "bf16")])
+def test_cfg5_backward_atomic_full_size(M, Z, dtype):
+    # dense fp32 gradient (the only backward a bf16 array has); fp32 arrays also take the fused step
+    w = synth.workload(5, M=M, Z=Z, array_dtype=dtype)
+    with Case(w) as c:
+        g_h = synth.make_grad_out(w)
+        g_d = torch.from_numpy(g_h).to(c.dev)
+        delta64, l1 = c.oracle.backward_f64(g_h, c.indices_h, c.offsets_h, c.B)
+        ga = c.backward(g_d, "atomic").cpu().numpy()
+        assert_within_l1(ga, delta64, l1, what=f"cfg5 M={M} Z={Z} {dtype} atomic")
+        assert abs(float(ga.astype(np.float64).sum()) - float(g_h.astype(np.float64).sum())) \
+            < 1e-6 * float(l1.sum())  # mass: every id contributes its row once
+        if dtype == "f32":
+            before = c.array_h.copy()
+            c.backward(g_d, "atomic", sgd=True, lr=0.5)
+            assert_within_l1(c.array.cpu().numpy(), before.astype(np.float64) - 0.5 * delta64,
+                             0.5 * l1 + np.abs(before), what=f"cfg5 M={M} Z={Z} atomic sgd")
+
+
+def test_cfg5_1mb_z32_deterministic_full_size():
+    # 4000 terms per slot: every window of the slot-major apply streams many chunks
+    w = synth.workload(5, M=262_144, Z=32)
+    with Case(w) as c:
+        g_h = synth.make_grad_out(w)
+        g_d = torch.from_numpy(g_h).to(c.dev)
+        can, touched = c.oracle.backward_canonical(g_h, c.indices_h, c.offsets_h, c.B)
+        det = c.backward(g_d, "det").cpu().numpy()
+        assert_bits_equal(det, can, "cfg5 1 MB Z=32 det")
+        assert_bits_equal(c.backward(g_d, "det").cpu().numpy(), det, "repeat")
+        before = c.array_h.copy()
+        c.backward(g_d, "det", sgd=True, lr=0.01)
+        want = before.copy()
+        orc.sgd_apply(want, can, touched, 0.01)
+        assert_bits_equal(c.array.cpu().numpy(), want, "cfg5 1 MB Z=32 det sgd")
+
+
+@pytest.mark.parametrize("M,Z", [(25_000_000, 2), (262_144, 1)])
+def test_cfg5_small_blocks_deterministic_reduced_batch(M, Z):
+    # more than 8 blocks per id: the one-thread-per-block key kernel, and the most sort passes
+    w = synth.workload(5, M=M, Z=Z)
+    with Case(w, batch=4096) as c:
+        g_h = synth.make_grad_out(w, 4096)
+        g_d = torch.from_numpy(g_h).to(c.dev)
+        can, _ = c.oracle.backward_canonical(g_h, c.indices_h, c.offsets_h, c.B)
+        assert_bits_equal(c.backward(g_d, "det").cpu().numpy(), can, f"cfg5 M={M} Z={Z} det")
+        _, detk = c.step_sharing_keys(g_d, "det")
+        assert_bits_equal(detk.cpu().numpy(), can, f"cfg5 M={M} Z={Z} det on kept starts")
+
+
+WINDOWS_10G = [(0, 200_000), (1_234_567_890, 300_000), (2_500_000_000 - 150_000, 150_000)]
+
+
+def test_cfg5_10gb_fused_sgd_atomic():
+    # the cell whose dense gradient would cost a 10 GB memset per step: the SGD step is fused into
+    # the scatter; slot windows at the start, in the middle and at the end of the array
+    w = synth.workload(5, M=2_500_000_000, Z=32)
+    _need_device_memory(16)
+    with Case(w, host_array=False) as c:
+        g_h = synth.make_grad_out(w)
+        g_d = torch.from_numpy(g_h).to(c.dev)
+        c.backward(g_d, "atomic", sgd=True, lr=0.5)
+        for j0, jn in WINDOWS_10G:
+            d64, l1 = c.oracle.backward_f64(g_h, c.indices_h, c.offsets_h, c.B, j0=j0, jn=jn)
+            before = _array_window(w, j0, jn)
+            after = c.array[j0:j0 + jn].cpu().numpy()
+            assert l1.max() > 0
+            assert_within_l1(after, before.astype(np.float64) - 0.5 * d64, 0.5 * l1 + np.abs(before),
+                             what=f"cfg5 10 GB fused SGD, window at {j0}")
+            assert_bits_equal(after[l1 == 0], before[l1 == 0], "untouched slots")
+
+
+@pytest.mark.parametrize("mode", ["binned", "det"])
+def test_cfg5_10gb_z128_sorted_backward(mode):
+    # binned (atomic accuracy) and deterministic (bit-exact) on the 10 GB array, fused SGD
+    w = synth.workload(5, M=2_500_000_000, Z=128)
+    _need_device_memory(20)
+    with Case(w, host_array=False) as c:
+        g_h = synth.make_grad_out(w)
+        g_d = torch.from_numpy(g_h).to(c.dev)
+        c.backward(g_d, mode, sgd=True, lr=0.5)
+        for j0, jn in WINDOWS_10G:
+            before = _array_window(w, j0, jn)
+            after = c.array[j0:j0 + jn].cpu().numpy()
+            if mode == "binned":
+                d64, l1 = c.oracle.backward_f64(g_h, c.indices_h, c.offsets_h, c.B, j0=j0, jn=jn)
+                assert_within_l1(after, before.astype(np.float64) - 0.5 * d64, 0.5 * l1 + np.abs(before),
+                                 what=f"cfg5 10 GB binned, window at {j0}")
+            else:
+                can, touched = c.oracle.backward_canonical(g_h, c.indices_h, c.offsets_h, c.B, j0=j0, jn=jn)
+                want = before.copy()
+                orc.sgd_apply(want, can, touched, 0.5)
+                assert touched.any()
+                assert_bits_equal(after, want, f"cfg5 10 GB deterministic, window at {j0}")
+
+
+def test_cfg4_deterministic_whole_array_vs_canonical():
+    # every one of the 250 M slots against the canonical-order oracle (one sort of 34 M blocks on a
+    # host core), dense gradient and fused SGD
+    w = synth.workload(4)
+    with Case(w) as c:
+        g_h = synth.make_grad_out(w)
+        g_d = torch.from_numpy(g_h).to(c.dev)
+        can, touched = c.oracle.backward_canonical(g_h, c.indices_h, c.offsets_h, c.B)
+        det = c.backward(g_d, "det").cpu().numpy()
+        assert_bits_equal(det, can, "cfg4 det, whole array")
+        del det
+        before = c.array_h.copy()
+        c.step_sharing_keys(g_d, "det", sgd=True, lr=0.5)
+        orc.sgd_apply(before, can, touched, 0.5)
+        assert_bits_equal(c.array.cpu().numpy(), before, "cfg4 det SGD on kept starts, whole array")
+
+
+def test_cfg3_z1_deterministic_full_batch_vs_canonical():
+    # Zipf ids, every element hashed on its own: 109 M blocks, the hottest id adds thousands of
+    # terms to each of its 128 slots (long walks); the whole 25 M-slot array bit for bit
+    w = synth.workload(3, Z=1)
+    with Case(w) as c:
+        g_h = synth.make_grad_out(w)
+        g_d = torch.from_numpy(g_h).to(c.dev)
+        can, _ = c.oracle.backward_canonical(g_h, c.indices_h, c.offsets_h, c.B)
+        assert_bits_equal(c.backward(g_d, "det").cpu().numpy(), can, "cfg3 Z=1 det, full batch")
 
 
 # ---------------------------------------------------------------------------------------

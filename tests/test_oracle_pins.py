@@ -193,6 +193,10 @@ def test_forward_equals_brute_force_table(m, Z, d):
             want = arr[np.array(loc[e][x])]
             np.testing.assert_array_equal(out[x, e], want)
             np.testing.assert_array_equal(o.locate(e, x), np.array(loc[e][x], dtype=np.uint64))
+            # the per-element form of the mapping (Section 3.2, idx equation), element by element:
+            # an in-chunk offset taken inside the hash argument would fail here for every Z > 1
+            if x < 64:
+                assert [o.idx(e, x, i) for i in range(d)] == loc[e][x]
 
 
 def brute_force_locations_clubbed(kk, m, Z, d, vocab):
@@ -595,6 +599,29 @@ def test_sgd_apply_and_accumulate():
     np.testing.assert_array_equal(g, np.array([1.5, 1.0, 8.0, 1.0], dtype=np.float32))
 
 
+def test_dense_sgd_apply_hand_values_and_agreement_with_the_fused_step():
+    # data-parallel step: every slot gets fma(-lr, g, M); hand values (exact in fp32)
+    arr = np.array([1.0, 2.0, 3.0, -0.0, 0.5], dtype=np.float32)
+    g = np.array([0.5, 0.0, 7.0, 0.0, -0.25], dtype=np.float32)
+    a = arr.copy()
+    orc.dense_sgd_apply(a, g, 2.0)
+    np.testing.assert_array_equal(a, np.array([0.0, 2.0, -11.0, -0.0, 1.0], dtype=np.float32))
+    # one rounding, not two: 1 + 2^-24 * (1 + 2^-23) is 1 + 2^-23 under fma, 1 under mul-then-add
+    one = np.array([1.0], np.float32)
+    tiny = np.array([-(2.0 ** -24) * (1 + 2.0 ** -23)], np.float32)
+    orc.dense_sgd_apply(one, tiny, 1.0)
+    assert one[0] == np.float32(1.0 + 2.0 ** -23)
+    # on touched slots it is the fused step; on untouched slots (gradient +0) it changes no bit
+    rng = np.random.default_rng(4)
+    arr = rng.standard_normal(500).astype(np.float32)
+    delta = rng.standard_normal(500).astype(np.float32)
+    touched = (rng.random(500) < 0.6).astype(np.uint8)
+    fused, dense = arr.copy(), arr.copy()
+    orc.sgd_apply(fused, delta, touched, 0.3)
+    orc.dense_sgd_apply(dense, np.where(touched == 1, delta, np.float32(0.0)).astype(np.float32), 0.3)
+    np.testing.assert_array_equal(fused.view(np.uint32), dense.view(np.uint32))
+
+
 # ---------------------------------------------------------------------------------------
 # 7. Theorem 1: the sketch's inner-product estimator is unbiased with the printed variance
 # ---------------------------------------------------------------------------------------
@@ -630,6 +657,32 @@ def test_adam_apply_matches_torch_adam_and_closed_form():
     for now, was in zip((arr, m1, m2), before):
         np.testing.assert_array_equal(now[touched == 0], was[touched == 0])
         assert np.all(now[touched == 1] != was[touched == 1])
+
+
+def test_adam_step_hand_computed_eps_sits_outside_the_square_root():
+    # Kingma & Ba, Algorithm 1: theta <- theta - lr * mhat / (sqrt(vhat) + eps).  With powers of two
+    # every operation is exact, so the step has one value that can be worked out by hand:
+    #   g = eps = 2^-10, beta1 = 1/2, beta2 = 3/4, step 1, moments 0
+    #   m1 = g/2, mhat = m1 / (1 - 1/2) = g;  m2 = g^2/4, vhat = m2 / (1 - 3/4) = g^2
+    #   sqrt(vhat) + eps = 2g  ->  update = 1/2  ->  theta = 1 - lr/2
+    # (eps inside the root would give g / sqrt(g^2 + eps) = 0.0312..., eps dropped would give 1)
+    g = np.float32(2.0 ** -10)
+    arr = np.array([1.0, 1.0, -3.0], np.float32)
+    m1, m2 = np.zeros(3, np.float32), np.zeros(3, np.float32)
+    delta = np.array([g, -g, 0.0], np.float32)
+    orc.adam_apply(arr, m1, m2, delta, np.ones(3, np.uint8), 0.25, 0.5, 0.75, float(g), 1)
+    np.testing.assert_array_equal(arr, np.array([0.875, 1.125, -3.0], np.float32))
+    np.testing.assert_array_equal(m1, np.array([g / 2, -g / 2, 0.0], np.float32))
+    np.testing.assert_array_equal(m2, np.array([g * g / 4, g * g / 4, 0.0], np.float32))
+    # step 2, zero gradient on slot 0 (touched), slots 1 and 2 untouched: no longer exact in fp32,
+    # but the closed form below fixes the move to rounding
+    before = arr.copy()
+    orc.adam_apply(arr, m1, m2, np.zeros(3, np.float32), np.array([1, 0, 0], np.uint8), 0.25, 0.5, 0.75,
+                   float(g), 2)
+    # mhat = g/3; vhat = (3/16 g^2)/(7/16) = 3/7 g^2; update = (1/3)/(sqrt(3/7) + 1)
+    want = 0.25 * (1.0 / 3.0) / (np.sqrt(3.0 / 7.0) + 1.0)
+    assert abs(float(before[0]) - float(arr[0]) - want) < 1e-7
+    assert arr[1] == before[1] and arr[2] == before[2]
 
 
 def test_theorem_1_mean_and_variance_monte_carlo():

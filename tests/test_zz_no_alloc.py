@@ -2,8 +2,9 @@
 the library a workspace (a process whose memory pool owns the whole device, or an operator that
 is given input and output buffers only).  Its scratch is an array inside the library image, so
 it allocates nothing; the checks here are that it gives the same bits as robe_backward with a
-caller-provided workspace, on two calls in a row that leave different stale contents behind,
-and that a call too large for the fixed array is refused.
+caller-provided workspace and as the CPU oracle's canonical-order gradient, on two calls in a
+row that leave different stale contents behind, that the device's free memory does not move
+across the calls, and that a call too large for the fixed array is refused.
 
 This file sorts last on purpose: a run that stops at the first failure has then already run
 every other test."""
@@ -38,6 +39,12 @@ def _reference_dense(c, g_d):
     return c.backward(g_d, "det").cpu().numpy()
 
 
+def _oracle_dense(c, g_d):
+    """The CPU oracle's canonical-order fp32 gradient of the same inputs."""
+    can, _ = c.oracle.backward_canonical(g_d.cpu().numpy(), c.indices_h, c.offsets_h, c.B)
+    return can
+
+
 def _static_dense(c, g_d):
     ga = torch.zeros(c.w.M, dtype=torch.float32, device=c.dev)
     robe.robe_backward_deterministic_static(c.h, g_d, c.indices, c.offsets, c.B, ga, 0.0)
@@ -53,28 +60,47 @@ def test_two_calls_in_a_row_match_the_workspace_variant():
     with Case(big) as c1, Case(small) as c2:
         g1, g2 = _grad(c1, 1), _grad(c2, 2)
         want1, want2 = _reference_dense(c1, g1), _reference_dense(c2, g2)
-        gc.collect()  # tensors of earlier tests that only the collector frees would move the figure
-        before = torch.cuda.memory_allocated()
-        got1 = _static_dense(c1, g1)
-        got2 = _static_dense(c2, g2)
-        assert torch.cuda.memory_allocated() == before  # nothing was taken from torch's pool either
+        # a first call so that the module holding the fixed array and the cached symbol address
+        # are loaded; what is measured below is the steady state
+        _static_dense(c2, g2)
+        ga1 = torch.zeros(c1.w.M, dtype=torch.float32, device=c1.dev)
+        ga2 = torch.zeros(c2.w.M, dtype=torch.float32, device=c2.dev)
+        gc.collect()  # tensors of earlier tests that only the collector frees would move the figures
+        torch.cuda.synchronize()
+        pool_before = torch.cuda.memory_allocated()
+        free_before = torch.cuda.mem_get_info()[0]  # cudaMemGetInfo: sees every allocation on the device
+        robe.robe_backward_deterministic_static(c1.h, g1, c1.indices, c1.offsets, c1.B, ga1, 0.0)
+        robe.robe_backward_deterministic_static(c2.h, g2, c2.indices, c2.offsets, c2.B, ga2, 0.0)
+        torch.cuda.synchronize()
+        assert torch.cuda.mem_get_info()[0] == free_before   # no cudaMalloc inside the library
+        assert torch.cuda.memory_allocated() == pool_before   # and nothing taken from torch's pool
+        got1, got2 = ga1.cpu().numpy(), ga2.cpu().numpy()
         assert_bits_equal(got1, want1, "static scratch, first call")
         assert_bits_equal(got2, want2, "static scratch, second call")
+        assert_bits_equal(got1, _oracle_dense(c1, g1), "static scratch, first call, against the oracle")
+        assert_bits_equal(got2, _oracle_dense(c2, g2), "static scratch, second call, against the oracle")
         # and once more in the other order, with the sign hash on
         robe.robe_set_option(c1.h, robe.ROBE_OPT_SIGN, 1)
         want1s = _reference_dense(c1, g1)
         assert_bits_equal(_static_dense(c2, g2), want2, "static scratch, third call")
         assert_bits_equal(_static_dense(c1, g1), want1s, "static scratch, fourth call (sign)")
+        c1.oracle.sign = 1
+        assert_bits_equal(want1s, _oracle_dense(c1, g1), "sign on, against the oracle")
 
 
 def test_fused_sgd_matches_the_workspace_variant():
     w = _workload()
     with Case(w) as ref, Case(w) as sta:
         g = _grad(ref, 3)
+        from oracle import robe_oracle as orc
+        can, touched = ref.oracle.backward_canonical(g.cpu().numpy(), ref.indices_h, ref.offsets_h, ref.B)
+        want = ref.array_h.copy()
+        orc.sgd_apply(want, can, touched, 0.25)
         ref.backward(g, "det", sgd=True, lr=0.25)
         robe.robe_backward_deterministic_static(sta.h, g, sta.indices, sta.offsets, sta.B, None, 0.25)
         torch.cuda.synchronize()
         assert_bits_equal(sta.array.cpu().numpy(), ref.array.cpu().numpy(), "static scratch SGD step 1")
+        assert_bits_equal(sta.array.cpu().numpy(), want, "static scratch SGD step 1, against the oracle")
         ref.backward(g, "det", sgd=True, lr=0.25)
         robe.robe_backward_deterministic_static(sta.h, g, sta.indices, sta.offsets, sta.B, None, 0.25)
         torch.cuda.synchronize()
