@@ -310,6 +310,8 @@ def run_ours(args, w):
     robe.robe_attach_array(h, array)
     if table_major:
         robe.robe_set_option(h, robe.ROBE_OPT_BAG_LAYOUT, robe.ROBE_BAGS_TABLE_MAJOR)
+    robe.robe_set_option(h, robe.ROBE_OPT_FWD_KERNEL, args.fwd_kernel)
+    robe.robe_set_option(h, robe.ROBE_OPT_BWD_KERNEL, args.bwd_kernel)
     lr = 1.0  # the paper trains its DLRM with plain SGD at learning rate 1.0 (Section 5)
     ws = None
     bwd_launches = 1
@@ -497,7 +499,7 @@ def run_ours(args, w):
     # a traffic record applies to the configuration it was captured on, and to no other
     own_batch = args.batch == 0
     rec = NCU_TRAFFIC_RECORDS.get((w.name, args.backward, bool(share_keys), args.ids, args.bag_layout)) \
-        if (own_batch and not dp_step and world == 1) else None
+        if (own_batch and not dp_step and world == 1 and args.fwd_kernel == 0 and args.bwd_kernel == 0) else None
     sm_mhz = clocks.get("sm_mhz")
 
     def roof(nbytes, ms, kernel, which):
@@ -546,7 +548,8 @@ def run_ours(args, w):
         "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": w.name, "num_tables": T, "d": d, "Z": w.Z, "M": w.M, "batch_per_gpu": B,
-                   "ids_per_step_per_gpu": nnz_per_step, "ids": args.ids, "bags": bags, "bag_layout": args.bag_layout,
+                   "ids_per_step_per_gpu": nnz_per_step, "ids": args.ids, "fwd_kernel": args.fwd_kernel,
+                   "bwd_kernel": args.bwd_kernel, "bags": bags, "bag_layout": args.bag_layout,
                    "backward": {"atomic": "atomic", "det": "deterministic", "binned": "binned atomic"}[args.backward] +
                    (", SGD fused" if dense is None else (", dense fp32 gradient, all-reduce, dense SGD apply" if dp_step
                                                          else ", dense fp32 gradient")),
@@ -599,6 +602,10 @@ def main():
     ap.add_argument("--ids", default="int64", choices=["int64", "int32"], help="element type of the id arrays")
     ap.add_argument("--bag-layout", default="sample-major", choices=["sample-major", "table-major"],
                     help="bag numbering of the inputs: n*T + e (default) or e*B + n (per-table id lists end to end)")
+    ap.add_argument("--fwd-kernel", type=int, default=0,
+                    help="ROBE_OPT_FWD_KERNEL: 0 automatic, 1 direct, 2 staged (4-byte loads), 3 vector (16-byte loads)")
+    ap.add_argument("--bwd-kernel", type=int, default=0,
+                    help="ROBE_OPT_BWD_KERNEL of the atomic backward: 0 automatic, 1 direct, 2 staged, others see robe.h")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--dp-step", default="auto", choices=["auto", "on", "off"],
                     help="data-parallel step (backward into a dense gradient, all-reduce over the ranks, dense "

@@ -63,9 +63,34 @@ typedef enum {
                                backward calls add nothing - and the host call still
                                returns ROBE_OK.  Read it with robe_last_device_status
                                and zero it yourself before going on.                      */
-#define ROBE_OPT_FWD_KERNEL 4 /* 0 = automatic (default); other values pick one forward
-                                 kernel variant, for benchmarking only                    */
-#define ROBE_OPT_BWD_KERNEL 5 /* same for the atomic backward                             */
+#define ROBE_OPT_FWD_KERNEL 4 /* forward kernel; every variant gives the same bits.
+                                 0 automatic (default): the lane-hashed kernel for Z <= 2 on arrays of
+                                   up to 192 MB, the staged kernel for rows of up to 128 elements, else
+                                   the direct kernel
+                                 1 direct: any (Z, d); every lane hashes its element's chunk per id
+                                 2 staged: d <= 128; block starts of a batch of ids through shared
+                                   memory, 4-byte loads, lanes on consecutive slots of a block
+                                 3 vector: 16-byte loads of the aligned pieces around a block, shifted
+                                   in registers; fp32 array, d, Z and M multiples of 4, d <= 128, sign
+                                   off (measured slower than 2 on every workload; kept for comparison)
+                                 4 lane-hashed: d <= 128, Z <= d, sign off; chunks hashed in registers by
+                                   the lane that owns the element, persistent warps
+                                 A variant asked for a call it cannot take returns
+                                 ROBE_ERR_UNSUPPORTED and launches nothing.                          */
+#define ROBE_OPT_BWD_KERNEL 5 /* kernel of the ATOMIC backward (all within the atomic bound):
+                                 0 automatic (default): lane-hashed for Z <= 2 on arrays of up to
+                                   192 MB, staged for d <= 128, else direct
+                                 1 direct   2 staged (scalar red.global.add.f32, lanes on consecutive slots)
+                                 3 vector: red.global.add.v4.f32 on the aligned middle of a block,
+                                   scalar head and tail; d, Z, M multiples of 4, d <= 128, sign off
+                                   (measured slower than 2; kept for comparison)
+                                 4 vector, repeats of an id inside a staged batch merged first
+                                 5 merged rows: one-hot input, sign off, d <= 128; a warp takes up to 64
+                                   rows of ONE table, sums the gradient rows of repeated ids in
+                                   registers and issues one reduction per element for all of them -
+                                   pays for skewed (Zipf) ids with long blocks (Z = 128: 1.34 x), costs
+                                   10-40 % on uniform ids, so it is the caller's choice
+                                 6 lane-hashed: d <= 128, Z <= d, sign off                            */
 
 #define ROBE_OPT_INDEX_TYPE 6 /* ROBE_I64 (default) | ROBE_I32: element type of `indices` in the
                                  calls that follow (offsets stay int64)                   */
@@ -320,6 +345,28 @@ int robe_backward_deterministic_static(robe_handle_t h, const float* grad_out,
  */
 int robe_set_status_word(robe_handle_t h, int32_t* dev_word);
 int robe_last_device_status(robe_handle_t h, void* stream);
+
+/*
+ * robe_debug_status / robe_debug_selftest - the index-check build (librobe_debug.so: the same
+ * sources compiled with -DROBE_DEBUG; it stands in for a memory checker on machines where none can
+ * be run).  In that build every computed index of every kernel - array slots, sorted positions,
+ * shared-memory offsets, positions in grad_out, window and hand-over record numbers - is compared
+ * with its bound before use; a violation records a ROBE_DBG_* code (the first one sticks) and the
+ * access is skipped: nothing traps, the context stays usable.  robe_debug_status synchronises
+ * `stream`, returns the recorded code (0 = none; see the ROBE_DBG_* values below) and clears it.
+ * robe_debug_selftest launches one kernel that fails a check on purpose WITHOUT touching memory
+ * (code 99), to show that the reporting path works.  The release library performs no check and
+ * returns ROBE_ERR_UNSUPPORTED from both.
+ */
+#define ROBE_DBG_ARRAY_SLOT 1
+#define ROBE_DBG_SORT_POS 2
+#define ROBE_DBG_SHARED 3
+#define ROBE_DBG_GRAD_POS 4
+#define ROBE_DBG_WINDOW 5
+#define ROBE_DBG_LONG_WALK 6
+#define ROBE_DBG_SELFTEST 99
+int robe_debug_status(void* stream);
+int robe_debug_selftest(void* stream);
 
 /* robe_status_string - static host string for a robe_status value. */
 const char* robe_status_string(int status);

@@ -13,7 +13,9 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "librobe.so")
+# ROBE_LIBRARY names another build of the same library to load instead (the index-check build
+# librobe_debug.so); it is not a fallback: a name that does not exist fails below like the default.
+LIB_PATH = os.environ.get("ROBE_LIBRARY") or os.path.join(_HERE, "librobe.so")
 
 ROBE_OK = 0
 ROBE_ERR_INVALID_ARG = -1
@@ -44,12 +46,15 @@ ROBE_BWD_BINNED = 2
 
 ROBE_STATIC_SCRATCH_BYTES = 32 << 20
 
+ROBE_DBG_SELFTEST = 99
+
 EXPORTS = [
     "robe_create", "robe_destroy", "robe_set_option", "robe_attach_array",
     "robe_get_hash_constants", "robe_forward", "robe_backward_workspace_bytes", "robe_backward",
     "robe_set_status_word", "robe_last_device_status", "robe_status_string",
     "robe_backward_deterministic_static", "robe_backward_adam",
     "robe_forward_keep", "robe_backward_kept", "robe_apply_sgd",
+    "robe_debug_status", "robe_debug_selftest",
 ]
 
 if not os.path.exists(LIB_PATH):
@@ -75,6 +80,8 @@ _lib.robe_backward_deterministic_static.argtypes = [_vp, _vp, _vp, _vp, _i64, _i
 _lib.robe_backward_adam.argtypes = [_vp, _vp, _vp, _vp, _i64, _i64, _vp, _vp, C.c_float, C.c_float,
                                     C.c_float, C.c_float, _i64, _vp, C.c_size_t, _vp]
 _lib.robe_apply_sgd.argtypes = [_vp, _vp, C.c_float, C.c_int, _vp]
+_lib.robe_debug_status.argtypes = [_vp]
+_lib.robe_debug_selftest.argtypes = [_vp]
 _lib.robe_set_status_word.argtypes = [_vp, _vp]
 _lib.robe_last_device_status.argtypes = [_vp, _vp]
 _lib.robe_status_string.argtypes = [C.c_int]
@@ -231,6 +238,16 @@ def robe_apply_sgd(h, grad_array, lr: float, zero_grad: bool = True, stream=None
     """Dense SGD apply of the data-parallel step: array <- fma(-lr, grad_array, array)."""
     _check(_lib.robe_apply_sgd(h, _dev_ptr(grad_array, torch.float32), lr, 1 if zero_grad else 0,
                                _stream_ptr(stream)), "robe_apply_sgd")
+
+
+def robe_debug_status(stream=None) -> int:
+    """Index-check build only: the first recorded ROBE_DBG_* code (0 = none), cleared by the call;
+    ROBE_ERR_UNSUPPORTED (-5) from the release library."""
+    return int(_lib.robe_debug_status(_stream_ptr(stream)))
+
+
+def robe_debug_selftest(stream=None) -> int:
+    return int(_lib.robe_debug_selftest(_stream_ptr(stream)))
 
 
 def robe_set_status_word(h, word) -> None:

@@ -37,6 +37,31 @@ def build(force: bool = False, verbose: bool = False) -> str:
     return LIB
 
 
+DEBUG_LIB = os.path.join(_HERE, "librobe_debug.so")
+
+
+def build_debug(force: bool = False) -> str:
+    """The index-check build: the same sources with -DROBE_DEBUG, compiled as ONE translation unit
+    (a generated file that includes every .cu) so that the device word the checks report into
+    exists once."""
+    stale = not os.path.exists(DEBUG_LIB) or (os.path.exists(LIB) and os.path.getmtime(DEBUG_LIB) < os.path.getmtime(LIB))
+    if force or stale or _stale():
+        nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+        unity = os.path.join(CSRC, "_unity_debug.cu")
+        try:
+            with open(unity, "w") as f:
+                for src in sources():
+                    if os.path.basename(src) != "_unity_debug.cu":
+                        f.write(f'#include "{os.path.basename(src)}"\n')
+            subprocess.run([nvcc] + NVCC_FLAGS + ["-DROBE_DEBUG", "-o", DEBUG_LIB, unity], check=True)
+        finally:
+            if os.path.exists(unity):
+                os.unlink(unity)
+    return DEBUG_LIB
+
+
 if __name__ == "__main__":
     build(force=True, verbose="-v" in sys.argv)
     print(LIB)
+    if "--debug" in sys.argv:
+        print(build_debug(force=True))

@@ -36,7 +36,7 @@ struct robe_ctx {
     cudaEvent_t fork_event, join_event;
 };
 
-namespace {
+namespace robe_api_detail {  // (named: the debug build compiles all sources as one translation unit)
 
 // SplitMix64 (Steele, Lea, Flood): the stream the hash constants are drawn from.
 uint64_t splitmix_next(uint64_t& s) {
@@ -73,6 +73,14 @@ __global__ void validate_kernel(IdList indices, const int64_t* offsets, int64_t 
         if (t < nbags && offsets[t + 1] < o) bad = true;
         if (bad) atomicCAS(status, ROBE_DEV_OK, ROBE_DEV_BAD_OFFSETS);
     }
+}
+
+// status of a launch helper: a kernel variant that cannot take the call reports an invalid value
+int launch_status(cudaError_t e) {
+    if (e == cudaSuccess) return ROBE_OK;
+    if (e == cudaErrorInvalidValue) return ROBE_ERR_UNSUPPORTED;
+    (void)cudaGetLastError();
+    return ROBE_ERR_CUDA;
 }
 
 bool check_sizes(robe_ctx* h, const void* indices, const int64_t* offsets, int64_t batch,
@@ -154,7 +162,8 @@ bool sorted_path_fits(const robe_ctx* h, const Problem& pb) {
     return (uint64_t)pb.nbags * h->mp.d <= (1ull << 32);
 }
 
-}  // namespace
+}  // namespace robe_api_detail
+using namespace robe_api_detail;
 
 namespace robe {
 cudaError_t launch_validate(const Problem& pb, cudaStream_t st) {
@@ -252,7 +261,7 @@ int robe_set_option(robe_handle_t h, int key, int64_t value) {
             h->validate = (int)value;
             return ROBE_OK;
         case ROBE_OPT_FWD_KERNEL:
-            if (value < 0 || value > 3) return ROBE_ERR_INVALID_ARG;
+            if (value < 0 || value > 4) return ROBE_ERR_INVALID_ARG;
             h->fwd_variant = (int)value;
             return ROBE_OK;
         case ROBE_OPT_INDEX_TYPE:
@@ -264,7 +273,7 @@ int robe_set_option(robe_handle_t h, int key, int64_t value) {
             h->bag_layout = (int)value;
             return ROBE_OK;
         case ROBE_OPT_BWD_KERNEL:
-            if (value < 0 || value > 2) return ROBE_ERR_INVALID_ARG;
+            if (value < 0 || value > 6) return ROBE_ERR_INVALID_ARG;
             h->bwd_variant = (int)value;
             return ROBE_OK;
         default:
@@ -312,8 +321,7 @@ int robe_forward(robe_handle_t h, const void* indices, const int64_t* offsets, i
     const Problem pb = make_problem(h, indices, offsets, batch, nnz);
     cudaStream_t st = (cudaStream_t)stream;
     if (launch_validate(pb, st) != cudaSuccess) return ROBE_ERR_CUDA;
-    if (launch_forward(pb, out, h->fwd_variant, st) != cudaSuccess) return ROBE_ERR_CUDA;
-    return ROBE_OK;
+    return launch_status(launch_forward(pb, out, h->fwd_variant, st));
 }
 
 int robe_forward_keep(robe_handle_t h, const void* indices, const int64_t* offsets, int64_t batch,
@@ -334,7 +342,8 @@ int robe_forward_keep(robe_handle_t h, const void* indices, const int64_t* offse
     uint32_t *keys = nullptr, *vals = nullptr;
     if (nnz > 0 && batch > 0) block_key_buffers(pb, workspace, &keys, &vals);
     bool kept = false;
-    if (launch_forward(pb, out, h->fwd_variant, st, keys, vals, &kept) != cudaSuccess) return ROBE_ERR_CUDA;
+    const int frc = launch_status(launch_forward(pb, out, h->fwd_variant, st, keys, vals, &kept));
+    if (frc != ROBE_OK) return frc;
     // a forward kernel that keeps nothing (rows longer than 128): the backward's own key kernels
     if (!kept && launch_block_keys(pb, workspace, workspace_bytes, st) != cudaSuccess) return ROBE_ERR_CUDA;
     return ROBE_OK;
@@ -363,10 +372,7 @@ static int backward_any(robe_handle_t h, const float* grad_out, const void* indi
     cudaStream_t st = (cudaStream_t)stream;
     if (h->bwd_mode == ROBE_BWD_ATOMIC) {
         if (launch_validate(pb, st) != cudaSuccess) return ROBE_ERR_CUDA;
-        if (launch_backward_atomic(pb, grad_out, target, sgd ? -lr : 1.0f, h->bwd_variant, st) !=
-            cudaSuccess)
-            return ROBE_ERR_CUDA;
-        return ROBE_OK;
+        return launch_status(launch_backward_atomic(pb, grad_out, target, sgd ? -lr : 1.0f, h->bwd_variant, st));
     }
     // the sort-based variants (binned, deterministic)
     if (!sorted_path_fits(h, pb)) return ROBE_ERR_UNSUPPORTED;
@@ -493,6 +499,37 @@ int robe_apply_sgd(robe_handle_t h, float* grad_array, float lr, int zero_grad, 
                                (cudaStream_t)stream) != cudaSuccess)
         return ROBE_ERR_CUDA;
     return ROBE_OK;
+}
+
+#ifdef ROBE_DEBUG
+namespace robe_api_detail {
+__global__ void debug_selftest_kernel() { (void)ROBE_CHK(threadIdx.x > 31u, ROBE_DBG_SELFTEST); }
+}  // namespace robe_api_detail
+#endif
+
+int robe_debug_status(void* stream) {
+#ifdef ROBE_DEBUG
+    cudaStream_t st = (cudaStream_t)stream;
+    int32_t code = 0;
+    const int32_t zero = 0;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return ROBE_ERR_CUDA;
+    if (cudaMemcpyFromSymbol(&code, g_robe_debug_code, sizeof code) != cudaSuccess) return ROBE_ERR_CUDA;
+    if (cudaMemcpyToSymbol(g_robe_debug_code, &zero, sizeof zero) != cudaSuccess) return ROBE_ERR_CUDA;
+    return (int)code;
+#else
+    (void)stream;
+    return ROBE_ERR_UNSUPPORTED;
+#endif
+}
+
+int robe_debug_selftest(void* stream) {
+#ifdef ROBE_DEBUG
+    debug_selftest_kernel<<<1, 32, 0, (cudaStream_t)stream>>>();
+    return cudaGetLastError() == cudaSuccess ? ROBE_OK : ROBE_ERR_CUDA;
+#else
+    (void)stream;
+    return ROBE_ERR_UNSUPPORTED;
+#endif
 }
 
 const char* robe_status_string(int status) {

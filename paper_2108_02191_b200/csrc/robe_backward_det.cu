@@ -94,6 +94,7 @@ det_keys_kernel(KeyArgs a, const uint32_t* bag_of, uint32_t* keys, uint32_t* val
     }
     const uint64_t base = hash_base(mp.h, e, x);
     for (uint32_t c = 0; c < mp.C; ++c) {
+        if (!ROBE_CHK(q0 + c < (uint64_t)a.nnz * mp.C, ROBE_DBG_SORT_POS)) break;
         keys[q0 + c] = block_start(mp, base, c);
         vals[q0 + c] = SIGN ? (uint32_t)(q0 + c) : (uint32_t)(bag * mp.d + c * mp.Z);
     }
@@ -264,6 +265,7 @@ sort_scatter_kernel(const uint32_t* __restrict__ kin, const uint32_t* __restrict
             if (idx < nb) {
                 const uint32_t dg = (key[r] >> shift) & mask;
                 const uint32_t lp = dstart[dg] + wcnt[w][dg] + rank[r];
+                if (!ROBE_CHK(lp < (uint32_t)kSortTile, ROBE_DBG_SHARED)) continue;
                 skey[lp] = key[r];
                 sval[lp] = vin[idx];  // payloads are only passed through: read them this late
             }
@@ -274,6 +276,7 @@ sort_scatter_kernel(const uint32_t* __restrict__ kin, const uint32_t* __restrict
         for (uint32_t lp = threadIdx.x; lp < in_tile; lp += kSortThreads) {
             const uint32_t k = skey[lp];
             const uint32_t dst = base[(k >> shift) & mask] + lp;
+            if (!ROBE_CHK((uint64_t)dst < nb, ROBE_DBG_SORT_POS)) continue;
             kout[dst] = k;
             vout[dst] = sval[lp];
         }
@@ -312,6 +315,7 @@ struct ApplyArgs {
     const uint8_t* win_left;
     const uint32_t* any_left;  // number of windows left over (0: the tile kernel has nothing to do)
     uint32_t win_log2;         // log2 of the window length
+    uint64_t grad_elems;       // elements of grad_out (read by the debug build's index checks only)
 };
 
 // The term that the sorted block with payload v contributes to the slot at in-block offset o
@@ -326,6 +330,7 @@ __device__ __forceinline__ bool block_term(const ApplyArgs& a, const uint32_t* b
             const uint32_t cz = v - (v / mp.d) * mp.d;
             if (cz + o >= mp.d) return false;
         }
+        if (!ROBE_CHK((uint64_t)v + o < a.grad_elems, ROBE_DBG_GRAD_POS)) return false;
         term = __ldg(a.grad_out + (uint64_t)v + o);
         return true;
     }
@@ -336,6 +341,7 @@ __device__ __forceinline__ bool block_term(const ApplyArgs& a, const uint32_t* b
     const uint64_t bag = bag_of ? (uint64_t)__ldg(bag_of + p) : (uint64_t)p;
     const uint32_t e = table_of_bag(bag, mp);
     const uint64_t x = (uint64_t)a.indices.load(p);
+    if (!ROBE_CHK(bag * mp.d + i < a.grad_elems, ROBE_DBG_GRAD_POS)) return false;
     term = sign_of(mp, hash_base(mp.g, e, x), i) * __ldg(a.grad_out + bag * mp.d + i);
     return true;
 }
@@ -346,6 +352,7 @@ __device__ __forceinline__ bool block_term(const ApplyArgs& a, const uint32_t* b
 // operation a separate correctly rounded fp32 one.  `old` is target[j].
 template <int MODE>
 __device__ __forceinline__ void commit_slot(const ApplyArgs& a, uint32_t j, float delta, float old) {
+    if (!ROBE_CHK(j < a.mp.m, ROBE_DBG_ARRAY_SLOT)) return;
     if (MODE == 0) {
         a.target[j] = __fadd_rn(old, delta);
     } else if (MODE == 1) {
@@ -501,7 +508,8 @@ __device__ __forceinline__ bool walk_deep(const ApplyArgs& a, ApplyTile& tl, App
         for (int t = 0; t < UN; ++t) {
             term[t] = 0.0f;
             if ((uint32_t)t < n_max) {
-                if ((uint32_t)t < n_in) term[t] = __ldg(a.grad_out + at[t]);
+                if ((uint32_t)t < n_in && ROBE_CHK((uint64_t)at[t] < a.grad_elems, ROBE_DBG_GRAD_POS))
+                    term[t] = __ldg(a.grad_out + at[t]);
             }
         }
 #pragma unroll
@@ -590,7 +598,7 @@ det_apply_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint32_t* __
         if (__ballot_sync(0xFFFFFFFFu, active) == 0) continue;
         const uint32_t j = (uint32_t)j64;
         float old = 0.0f;
-        if (active) old = a.target[j];
+        if (active && ROBE_CHK(j < mp.m, ROBE_DBG_ARRAY_SLOT)) old = a.target[j];
 
         if (tl.loaded_end > kRing) {  // an earlier long walk moved the ring past the tile's start
             __syncwarp();
@@ -665,7 +673,8 @@ det_bounds_kernel(const uint32_t* __restrict__ K, uint64_t nb, uint32_t* lo_of, 
         // windows b with b*W in (k[t], k[t+1]] get hi_of[b] = i (and b = 0 at i = 0)
         uint64_t from = i > 0 ? (k[t] >> win_log2) + 1 : 0;
         uint64_t to = i < nb ? (k[t + 1] >> win_log2) : nwin;
-        for (uint64_t b = from; b <= to && b <= nwin; ++b) hi_of[b] = (uint32_t)i;
+        for (uint64_t b = from; b <= to && b <= nwin; ++b)
+            if (ROBE_CHK(b <= (uint64_t)nwin, ROBE_DBG_WINDOW)) hi_of[b] = (uint32_t)i;
         from = i > 0 ? ((k[t] + (Z - 1)) >> win_log2) + 1 : 0;
         to = i < nb ? ((k[t + 1] + (Z - 1)) >> win_log2) : nwin;
         for (uint64_t b = from; b <= to && b <= nwin; ++b) lo_of[b] = (uint32_t)i;
@@ -729,9 +738,10 @@ det_apply_window_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint3
         if (e < n) {
             const uint32_t k = __ldg(K + lo + e);
             to = k - bias;
-            if (one_chunk) ent[e] = make_uint2(e * Z - k, __ldg(V + lo + e));
+            if (one_chunk && ROBE_CHK(e < kWinEnt, ROBE_DBG_SHARED)) ent[e] = make_uint2(e * Z - k, __ldg(V + lo + e));
         }
-        for (uint32_t t = from; t <= to; ++t) pre[t] = e;
+        for (uint32_t t = from; t <= to; ++t)
+            if (ROBE_CHK(t < W + kWinMaxZ + 8, ROBE_DBG_SHARED)) pre[t] = e;
     }
     __syncthreads();
     // a window in the middle of the array: every slot exists and none is a low slot
@@ -746,7 +756,8 @@ det_apply_window_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint3
         if (!one_chunk) {
             if (c0 != 0) __syncthreads();  // the chunk before has been used
             for (uint32_t e = tid; e < ne; e += kWinThreads)
-                ent[e] = make_uint2(e * Z - __ldg(K + lo + c0 + e), __ldg(V + lo + c0 + e));
+                if (ROBE_CHK(e < kWinEnt && (uint64_t)lo + c0 + e < a.nb, ROBE_DBG_SHARED))
+                    ent[e] = make_uint2(e * Z - __ldg(K + lo + c0 + e), __ldg(V + lo + c0 + e));
             __syncthreads();
         }
         if (vec4) {
@@ -754,14 +765,17 @@ det_apply_window_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint3
             const bool pow2 = mp.log2Z != 0xFFFFFFFFu;
             for (uint32_t t = tid; t < tot; t += kWinThreads) {
                 const uint32_t e = pow2 ? t >> (mp.log2Z - 2) : t / zq, o = t - e * zq;
-                reinterpret_cast<float4*>(stage)[t] =
-                    __ldg(reinterpret_cast<const float4*>(a.grad_out + ent[e].y) + o);
+                if (ROBE_CHK(4u * t + 3u < kWinStage && (uint64_t)ent[e].y + 4u * o + 3u < a.grad_elems,
+                             ROBE_DBG_GRAD_POS))
+                    reinterpret_cast<float4*>(stage)[t] =
+                        __ldg(reinterpret_cast<const float4*>(a.grad_out + ent[e].y) + o);
             }
         } else {
             const uint32_t tot = ne * Z;
             for (uint32_t t = tid; t < tot; t += kWinThreads) {
                 const uint32_t e = t / Z, o = t - e * Z;
-                stage[t] = __ldg(a.grad_out + ((uint64_t)ent[e].y + o));
+                if (ROBE_CHK(t < kWinStage && (uint64_t)ent[e].y + o < a.grad_elems, ROBE_DBG_GRAD_POS))
+                    stage[t] = __ldg(a.grad_out + ((uint64_t)ent[e].y + o));
             }
         }
         __syncthreads();
@@ -774,7 +788,9 @@ det_apply_window_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint3
             if (first < c1 && last > c0) {
                 const uint32_t j = j0 + q * kWinThreads;  // (a slot past the array is dropped at the commit)
                 float s = acc[q];
-                for (uint32_t e = f; e < l; ++e) s = __fadd_rn(s, stage[ent[e].x + j]);
+                for (uint32_t e = f; e < l; ++e)
+                    if (ROBE_CHK(e < kWinEnt && ent[e].x + j < kWinStage, ROBE_DBG_SHARED))
+                        s = __fadd_rn(s, stage[ent[e].x + j]);
                 acc[q] = s;
             }
         }
@@ -841,6 +857,7 @@ det_apply_long_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint32_
         __syncthreads();  // (the barriers inside a round order this store after all reads of the last one)
         const uint32_t rec = rec_s;
         if (rec >= n_rec) break;
+        if (!ROBE_CHK(rec < a.long_cap, ROBE_DBG_LONG_WALK)) break;
         const LongWalk* lw = a.long_walks + rec;
         const uint64_t i0 = lw->i0;
         const uint32_t j = lw->j[lane];
@@ -866,7 +883,8 @@ det_apply_long_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint32_
 #pragma unroll
             for (int q = 0; q < kPerCopier; ++q) {
                 const uint32_t t = (w - 1) + q * kLongCopiers;
-                if (t < (uint32_t)kLongStep && mine && kv[q].x <= j) {
+                if (t < (uint32_t)kLongStep && mine && kv[q].x <= j &&
+                    ROBE_CHK((uint64_t)kv[q].y + (j - kv[q].x) < a.grad_elems, ROBE_DBG_GRAD_POS)) {
                     const float* src = a.grad_out + (kv[q].y + (j - kv[q].x));
                     asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst + t * 128u), "l"(src));
                 }
@@ -1031,7 +1049,7 @@ binned_apply_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint32_t*
         if (ok[t]) {
             uint64_t j = (uint64_t)k[t] + u;
             if (j >= mp.m) j -= mp.m;
-            atomicAdd(a.target + j, a.lr * term[t]);
+            if (ROBE_CHK(j < mp.m, ROBE_DBG_ARRAY_SLOT)) atomicAdd(a.target + j, a.lr * term[t]);
         }
     }
 }
@@ -1251,7 +1269,7 @@ cudaError_t launch_backward_det(const Problem& pb, const float* grad_out, float*
         sort_scatter_kernel<false><<<sp.grid, kSortThreads, 0, st>>>(kA, vA, kB, vB, counts, totals, nb,
                                                                     sp.tiles, shift, mask);
         ApplyArgs ab{mp, grad_out, pb.indices, target, lr, nb, pb.status, AdamState{}, nullptr, nullptr, 0,
-                     nullptr, nullptr, 0};
+                     nullptr, nullptr, 0, (uint64_t)pb.nbags * mp.d};
         uint32_t log2Zp = 0;
         while ((1u << log2Zp) < mp.Z) ++log2Zp;
         const uint64_t groups = (nb + kBinnedPer - 1) / kBinnedPer;
@@ -1283,7 +1301,8 @@ cudaError_t launch_backward_det(const Problem& pb, const float* grad_out, float*
     uint32_t* long_count = (uint32_t*)(ws + L.long_count);
     cudaMemsetAsync(long_count, 0, 2 * sizeof(uint32_t), st);  // [0] rounds handed over, [1] rounds taken
     ApplyArgs aa{mp, grad_out, pb.indices, target, lr, nb, pb.status, adam ? *adam : AdamState{},
-                 long_count, (LongWalk*)(ws + L.long_walks), L.long_cap, nullptr, nullptr, 0};
+                 long_count, (LongWalk*)(ws + L.long_walks), L.long_cap, nullptr, nullptr, 0,
+                 (uint64_t)pb.nbags * mp.d};
     const WindowBuffers wb{(uint32_t*)(ws + L.bounds),
                            (uint32_t*)(ws + L.bounds + align256(((size_t)L.nwin + 1) * sizeof(uint32_t))),
                            (uint8_t*)(ws + L.win_left), L.nwin, L.win_log2,

@@ -16,6 +16,31 @@ namespace robe {
 
 constexpr uint64_t kP61 = (1ull << 61) - 1ull;
 
+// Index checks of the debug build (compiled with -DROBE_DEBUG as ONE translation unit, so that
+// the word below exists once).  ROBE_CHK(cond, code) guards a computed index: in the debug build a
+// false condition records `code` (the first one sticks) and the guarded access is skipped - no
+// trap, no assert, the context stays usable; in the release build it is the constant `true` and
+// costs nothing.  robe_debug_status() reads and clears the word.
+// codes (the values the C header documents):
+//   ROBE_DBG_ARRAY_SLOT  array / gradient slot >= m
+//   ROBE_DBG_SORT_POS    sorted position or block number >= number of blocks
+//   ROBE_DBG_SHARED      shared-memory index beyond its buffer
+//   ROBE_DBG_GRAD_POS    position in grad_out beyond bags * d
+//   ROBE_DBG_WINDOW      window number beyond the window tables
+//   ROBE_DBG_LONG_WALK   hand-over record beyond the list
+//   ROBE_DBG_SELFTEST    planted by robe_debug_selftest
+#include "../../include/robe.h"
+#ifdef ROBE_DEBUG
+__device__ int32_t g_robe_debug_code;
+__device__ __forceinline__ bool robe_dbg_ok(bool cond, int32_t code) {
+    if (!cond) atomicCAS(&g_robe_debug_code, 0, code);
+    return cond;
+}
+#define ROBE_CHK(cond, code) (::robe::robe_dbg_ok((cond), (code)))
+#else
+#define ROBE_CHK(cond, code) true
+#endif
+
 struct HashConsts {  // all < P
     uint64_t A, B, C, D;
 };

@@ -44,7 +44,8 @@ __global__ void __launch_bounds__(256) fwd_direct_kernel(FwdArgs a) {
             const uint64_t x = (uint64_t)a.indices.load(p);
             uint32_t j = id_block_start(mp, e, x, c) + o;  // < m + d <= 2^32
             if (j >= mp.m) j -= mp.m;
-            float v = load_elem<DT>(a.array, j);
+            float v = 0.0f;
+            if (ROBE_CHK(j < mp.m, ROBE_DBG_ARRAY_SLOT)) v = load_elem<DT>(a.array, j);
             if (SIGN) v = sign_of(mp, hash_base(mp.g, e, x), i) * v;
             acc = (p == lo) ? v : acc + v;
         }
@@ -81,7 +82,7 @@ __device__ __forceinline__ void gather_group(const FwdArgs& a, const uint32_t* c
             if (on && live[u]) {
                 uint32_t j = col[u][g0 + gg] + off[u];  // < m + d <= 2^32
                 if (WRAP && j >= mp.m) j -= mp.m;
-                val = gather_elem<DT>(a.array, j);
+                if (ROBE_CHK(j < mp.m, ROBE_DBG_ARRAY_SLOT)) val = gather_elem<DT>(a.array, j);
                 if (SIGN) val = sign_of(mp, gbase_s[g0 + gg], lane + 32u * u) * val;
             }
             v[gg][u] = val;
@@ -202,7 +203,7 @@ fwd_staged_kernel(FwdArgs a, uint32_t ids_per_batch, uint32_t cmagic) {
                                                                             : (int64_t)ids_per_batch);
         const bool wraps = stage_batch<SIGN, BAGS>(sm, mp, a.indices, p0, cnt, ids_per_batch, tterm,
                                                    gterm, cmagic, w, lane,
-                                                   KeepBlocks{a.keep_keys, a.keep_vals, (uint64_t)warp});
+                                                   KeepBlocks{a.keep_keys, a.keep_vals, (uint64_t)warp, (uint64_t)a.nnz * mp.C});
         if (wraps)
             gather_batch<EPL, DT, SIGN, BAGS, U, true>(a, col, off, live, gbase_s, cnt, p0, lane, acc);
         else
@@ -260,6 +261,7 @@ __device__ __forceinline__ void vec_gather_batch(const FwdArgs& a, const uint32_
                 const uint32_t r = pos & 3u;
                 uint32_t a0 = pos & ~3u;
                 if (WRAP && a0 >= mp.m) a0 -= mp.m;
+                if (!ROBE_CHK(a0 < mp.m && (r == 0 || WRAP || a0 + 4u < mp.m), ROBE_DBG_ARRAY_SLOT)) continue;
                 const float4 lo = ldg_f4_64B(array + a0);
                 float4 hi = lo;
                 if (r != 0) {
@@ -345,7 +347,7 @@ fwd_vec_kernel(FwdArgs a, uint32_t ids_per_batch, uint32_t cmagic) {
                                                                             : (int64_t)ids_per_batch);
         const bool wraps = stage_batch<false, BAGS>(sm, mp, a.indices, p0, cnt, ids_per_batch, tterm, 0,
                                                     cmagic, w, lane,
-                                                    KeepBlocks{a.keep_keys, a.keep_vals, (uint64_t)warp});
+                                                    KeepBlocks{a.keep_keys, a.keep_vals, (uint64_t)warp, (uint64_t)a.nnz * mp.C});
         if (wraps)
             vec_gather_batch<BAGS, true, U>(a, col, o, cnt, p0, lpi, ipi, grp, k, lane_on, acc);
         else
@@ -417,6 +419,126 @@ static void launch_staged_epl(const FwdArgs& a, bool bags, bool sign, cudaStream
         launch_staged_flags<4, DT>(a, bags, sign, st);
 }
 
+// Lane-hashed kernel for short blocks (Z <= 2 by default; any Z <= d whose lanes can afford to hash
+// their own chunks).  With d/Z chunks per id as numerous as the elements themselves, staging the
+// block starts in shared memory buys nothing: every lane owns elements lane, lane+32, .. of every
+// row and hashes exactly the chunks of those elements, in registers (LaneChunks).  Per id the shared
+// part of the hash is evaluated once, by one lane, 32 ids at a time, and handed round by shuffle.
+// Warps are persistent: the per-lane chunk constants are set up once and serve every row the
+// warp takes (rows in groups of 32, or one bag after another).
+template <int EPL, int DT, bool BAGS, bool M30, int U>
+__global__ void __launch_bounds__(256, 4)
+fwd_lanehash_kernel(FwdArgs a, uint32_t padj) {
+    __shared__ uint64_t tt_s[kRowTables];
+    const MapParams& mp = a.mp;
+    const uint32_t lane = threadIdx.x & 31;
+    for (uint32_t e = threadIdx.x; e < mp.T && e < (uint32_t)kRowTables; e += 256) tt_s[e] = table_term(mp.h, e);
+    __syncthreads();
+    if (a.status != nullptr && *a.status != 0) return;
+
+    LaneChunks<EPL> lc;
+    lc.init(mp, lane, padj);
+    const uint32_t m = mp.m;
+
+    // the loads of U ids (the owned elements of each) are issued together
+    auto gather_ids = [&](uint32_t bm, uint64_t thr, uint32_t g0, uint32_t n, float (&v)[U][EPL]) {
+#pragma unroll
+        for (int gg = 0; gg < U; ++gg) {
+            const int src = (int)(g0 + gg < n ? g0 + gg : n - 1);
+            const uint32_t bm_g = __shfl_sync(0xFFFFFFFFu, bm, src);
+            const uint64_t thr_g = __shfl_sync(0xFFFFFFFFu, thr, src);
+#pragma unroll
+            for (int u = 0; u < EPL; ++u) {
+                v[gg][u] = 0.0f;
+                if (lc.live[u]) {
+                    const uint32_t j = lc.template slot<M30>(u, bm_g, thr_g);
+                    if (ROBE_CHK(j < m, ROBE_DBG_ARRAY_SLOT)) v[gg][u] = gather_elem<DT>(a.array, j);
+                }
+            }
+        }
+    };
+
+    const int64_t nwarps = (int64_t)gridDim.x * 8;
+    const int64_t gw = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (!BAGS) {
+        for (int64_t r0 = gw * 32; r0 < a.nbags; r0 += nwarps * 32) {
+            const int64_t row = r0 + lane;
+            uint32_t bm = 0;
+            uint64_t thr = kP61;
+            if (row < a.nbags)
+                lane_id_base(mp, lane_table_term(tt_s, mp, (uint64_t)row), (uint64_t)a.indices.load(row), bm, thr);
+            const uint32_t n = (uint32_t)(a.nbags - r0 < 32 ? a.nbags - r0 : 32);
+            for (uint32_t g0 = 0; g0 < n; g0 += U) {
+                float v[U][EPL];
+                gather_ids(bm, thr, g0, n, v);
+#pragma unroll
+                for (int gg = 0; gg < U; ++gg) {
+                    if (g0 + gg < n) {
+                        float* orow = a.out + (r0 + g0 + gg) * (int64_t)mp.d;
+#pragma unroll
+                        for (int u = 0; u < EPL; ++u)
+                            if (lc.live[u]) __stcs(orow + lane + 32u * u, v[gg][u]);
+                    }
+                }
+            }
+        }
+    } else {
+        for (int64_t bag = gw; bag < a.nbags; bag += nwarps) {
+            int64_t lo, hi;
+            bag_range(a.offsets, a.nnz, bag, lo, hi);
+            const uint64_t tterm = lane_table_term(tt_s, mp, (uint64_t)bag);
+            float acc[EPL];
+#pragma unroll
+            for (int u = 0; u < EPL; ++u) acc[u] = -0.0f;  // -0 + v == v: the first term initialises
+            for (int64_t p0 = lo; p0 < hi; p0 += 32) {
+                uint32_t bm = 0;
+                uint64_t thr = kP61;
+                if (p0 + lane < hi) lane_id_base(mp, tterm, (uint64_t)a.indices.load(p0 + lane), bm, thr);
+                const uint32_t n = (uint32_t)(hi - p0 < 32 ? hi - p0 : 32);
+                for (uint32_t g0 = 0; g0 < n; g0 += U) {
+                    float v[U][EPL];
+                    gather_ids(bm, thr, g0, n, v);
+#pragma unroll
+                    for (int gg = 0; gg < U; ++gg)
+                        if (g0 + gg < n) {
+#pragma unroll
+                            for (int u = 0; u < EPL; ++u) acc[u] = acc[u] + v[gg][u];
+                        }
+                }
+            }
+            float* orow = a.out + bag * (int64_t)mp.d;
+#pragma unroll
+            for (int u = 0; u < EPL; ++u)
+                if (lc.live[u]) __stcs(orow + lane + 32u * u, hi <= lo ? 0.0f : acc[u]);
+        }
+    }
+}
+
+// what the lane-hashed kernel asks of a call: plain blocks (no rows clubbed into one), sign off
+static bool lanehash_ok(const Problem& pb) { return pb.sign == 0 && pb.mp.R == 1 && pb.mp.d <= 128; }
+
+template <int EPL, int DT>
+static void launch_lanehash_m(const FwdArgs& a, bool bags, cudaStream_t st) {
+    const unsigned blocks = lane_grid(bags ? a.nbags : (a.nbags + 31) / 32);
+    const uint32_t padj = lane_padj(a.mp);
+    const bool m30 = a.mp.m < (1u << 30);
+    constexpr int U = EPL == 4 ? 2 : 4;
+    if (bags) {
+        if (m30) fwd_lanehash_kernel<EPL, DT, true, true, U><<<blocks, 256, 0, st>>>(a, padj);
+        else fwd_lanehash_kernel<EPL, DT, true, false, U><<<blocks, 256, 0, st>>>(a, padj);
+    } else {
+        if (m30) fwd_lanehash_kernel<EPL, DT, false, true, U><<<blocks, 256, 0, st>>>(a, padj);
+        else fwd_lanehash_kernel<EPL, DT, false, false, U><<<blocks, 256, 0, st>>>(a, padj);
+    }
+}
+
+template <int DT>
+static void launch_lanehash(const FwdArgs& a, bool bags, cudaStream_t st) {
+    if (a.mp.d <= 32) launch_lanehash_m<1, DT>(a, bags, st);
+    else if (a.mp.d <= 64) launch_lanehash_m<2, DT>(a, bags, st);
+    else launch_lanehash_m<4, DT>(a, bags, st);
+}
+
 cudaError_t launch_forward(const Problem& pb, float* out, int variant, cudaStream_t st,
                            uint32_t* keep_keys, uint32_t* keep_vals, bool* kept) {
     if (kept != nullptr) *kept = false;
@@ -430,6 +552,18 @@ cudaError_t launch_forward(const Problem& pb, float* out, int variant, cudaStrea
         if (!vec_kernel_ok(pb, out)) return cudaErrorInvalidValue;
         if (kept != nullptr) *kept = keep_keys != nullptr;
         launch_vec(a, bags, st);
+        return cudaGetLastError();
+    }
+    // Short blocks: every lane hashes its own chunks (keeps nothing for a sort-based backward).
+    // Automatic for arrays of L2 size, where the staged kernel is bound by its instruction count
+    // (measured on B200, Z = 1 / 2: 1 MB array 2.27 -> 1.72 ms / 1.72 -> 1.00 ms, 100 MB 3.59 -> 3.40 /
+    // 2.14 -> 2.09); on a 10 GB array the staged kernel's higher occupancy keeps more DRAM requests
+    // in flight and stays ahead (9.5 vs 10.2 ms), so it keeps those.
+    const bool l2_sized = (uint64_t)pb.mp.m * (pb.dtype == 0 ? 4u : 2u) <= (192ull << 20);
+    if (variant == 4 || (variant == 0 && pb.mp.Z <= 2 && l2_sized && lanehash_ok(pb) && keep_keys == nullptr)) {
+        if (!lanehash_ok(pb)) return cudaErrorInvalidValue;
+        if (pb.dtype == 0) launch_lanehash<0>(a, bags, st);
+        else launch_lanehash<1>(a, bags, st);
         return cudaGetLastError();
     }
     const bool use_warp = variant == 2 || (variant == 0 && warp_ok);

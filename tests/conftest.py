@@ -24,3 +24,14 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(autouse=True)
+def _index_checks_stay_clean(request):
+    """When the suite runs on the index-check build of the library (ROBE_LIBRARY names it), every GPU
+    test must leave the library's debug word at zero: no kernel computed an index beyond its bound."""
+    yield
+    if "gpu" in request.keywords and os.environ.get("ROBE_LIBRARY"):
+        import paper_2108_02191_b200 as robe
+        code = robe.robe_debug_status()
+        assert code == 0, f"a kernel of the index-check build failed check {code} (ROBE_DBG_* in include/robe.h)"

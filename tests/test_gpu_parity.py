@@ -56,11 +56,15 @@ def test_forward_shapes(d, Z, M, bags):
         with Case(w, sign=sign) as c:
             want = c.oracle_forward()
             warp_ok = d <= 128
-            for kernel in ([0, 1, 2] if warp_ok else [0, 1]):
+            lane_hashed_ok = warp_ok and Z <= d and not sign  # kernel 4: every lane hashes its own chunks
+            for kernel in ([0, 1, 2] if warp_ok else [0, 1]) + ([4] if lane_hashed_ok else []):
                 assert_bits_equal(c.forward(kernel).cpu().numpy(), want, f"d={d} Z={Z} M={M} k={kernel}")
             if not warp_ok:
                 with pytest.raises(robe.RobeError):
                     c.forward(2)
+            if not lane_hashed_ok:
+                with pytest.raises(robe.RobeError):
+                    c.forward(4)
 
 
 # The kernel with 16-byte loads (ROBE_OPT_FWD_KERNEL = 3): fp32 array, d, Z and M multiples of
@@ -104,8 +108,11 @@ def test_forward_bf16_array():
     w = small(array_dtype="bf16", d=64, Z=16, M=5000, bag_rule=(4, 0, 12))
     with Case(w) as c:
         want = c.oracle_forward()
-        for kernel in FWD_KERNELS:
+        for kernel in FWD_KERNELS + [4]:
             assert_bits_equal(c.forward(kernel).cpu().numpy(), want, "bf16")
+    for Z in (1, 2):  # short blocks take the lane-hashed kernel by themselves
+        with Case(small(array_dtype="bf16", d=96, Z=Z, M=5003, bag_rule=(4, 0, 12))) as c:
+            assert_bits_equal(c.forward().cpu().numpy(), c.oracle_forward(), "bf16, short blocks")
 
 
 @pytest.mark.parametrize("bags", [None, (3, 0, 9)])
@@ -126,6 +133,17 @@ def test_int32_indices(bags):
                     assert_within_l1(c.backward(g_d, "atomic", kernel=kernel).cpu().numpy(), delta64, l1,
                                      what="int32 ids atomic")
                 assert_bits_equal(c.backward(g_d, "det").cpu().numpy(), can, "int32 ids deterministic")
+
+
+def test_forward_lane_hashed_kernel_many_tables_and_large_ids():
+    # more tables than the kernel keeps table terms for in shared memory; ids beyond 2^32
+    T = 700
+    w = small(num_tables=T, vocab_arg=tuple([2**40 + 12345] * T), d=40, Z=1, M=3001, batch=9)
+    with Case(w) as c:
+        assert_bits_equal(c.forward(4).cpu().numpy(), c.oracle_forward(), "lane-hashed, 700 tables")
+    w = small(num_tables=T, vocab_arg=tuple([2**40 + 12345] * T), d=40, Z=2, M=3001, batch=9, bag_rule=(3, 0, 70))
+    with Case(w) as c:
+        assert_bits_equal(c.forward(4).cpu().numpy(), c.oracle_forward(), "lane-hashed, 700 tables, bags")
 
 
 def test_forward_empty_and_degenerate_inputs():
@@ -227,9 +245,13 @@ def test_backward_shapes(d, Z, M, bags):
             delta64, l1 = c.oracle.backward_f64(g_h, c.indices_h, c.offsets_h, c.B)
             can, touched = c.oracle.backward_canonical(g_h, c.indices_h, c.offsets_h, c.B)
             warp_ok = d <= 128
-            for kernel in ([0, 1, 2] if warp_ok else [0, 1]):
+            lane_hashed_ok = warp_ok and Z <= d and not sign  # kernel 6: every lane hashes its own chunks
+            for kernel in ([0, 1, 2] if warp_ok else [0, 1]) + ([6] if lane_hashed_ok else []):
                 ga = c.backward(g_d, "atomic", kernel=kernel).cpu().numpy()
                 assert_within_l1(ga, delta64, l1, what=f"atomic d={d} Z={Z} M={M} k={kernel}")
+            if not lane_hashed_ok:
+                with pytest.raises(robe.RobeError):
+                    c.backward(g_d, "atomic", kernel=6)
             gb = c.backward(g_d, "binned").cpu().numpy()
             assert_within_l1(gb, delta64, l1, what=f"binned d={d} Z={Z} M={M}")
             det = c.backward(g_d, "det").cpu().numpy()
@@ -239,6 +261,57 @@ def test_backward_shapes(d, Z, M, bags):
             di, _ = c.oracle.backward_f64(gi_h, c.indices_h, c.offsets_h, c.B)
             assert_bits_equal(c.backward(gi_d, "atomic").cpu().numpy(), di.astype(np.float32), "int atomic")
             assert_bits_equal(c.backward(gi_d, "det").cpu().numpy(), di.astype(np.float32), "int det")
+
+
+# Atomic backward with 16-byte reductions (ROBE_OPT_BWD_KERNEL = 3) and with the duplicates of an
+# id merged in the warp first (4): the forward vector kernel's shapes, uniform ids and ids so
+# skewed that most rows of a batch repeat one id.
+@pytest.mark.parametrize("bags", [None, (3, 0, 9), (20, 1, 80)])
+@pytest.mark.parametrize("d,Z,M", VEC_SHAPES)
+def test_backward_vector_kernels(d, Z, M, bags):
+    for vocab, dist_ in (((50, 7, 1000), "uniform"), ((3, 2, 40), "zipf1.05")):
+        w = small(d=d, Z=Z, M=M, bag_rule=bags, batch=131, vocab_arg=vocab, id_dist=dist_)
+        with Case(w) as c:
+            g_h, g_d = _grad(c, 6)
+            delta64, l1 = c.oracle.backward_f64(g_h, c.indices_h, c.offsets_h, c.B)
+            gi_h, gi_d = _grad(c, 2, integer=True)
+            di, _ = c.oracle.backward_f64(gi_h, c.indices_h, c.offsets_h, c.B)
+            for kernel in (3, 4) + ((5,) if bags is None else ()):
+                ga = c.backward(g_d, "atomic", kernel=kernel).cpu().numpy()
+                assert_within_l1(ga, delta64, l1, what=f"vector atomic k={kernel} d={d} Z={Z} M={M} {dist_}")
+                # integer gradients: exact whatever the order and the grouping
+                assert_bits_equal(c.backward(gi_d, "atomic", kernel=kernel).cpu().numpy(),
+                                  di.astype(np.float32), f"vector atomic k={kernel}, integer gradient")
+            before = c.array_h.copy()
+            c.backward(g_d, "atomic", sgd=True, lr=0.5, kernel=4)
+            assert_within_l1(c.array.cpu().numpy(), before.astype(np.float64) - 0.5 * delta64,
+                             0.5 * l1 + np.abs(before), what="vector atomic sgd")
+
+
+# Kernel 5: one-hot rows taken table by table and the repeats of an id merged in the warp before
+# the reduction; any (d, Z, M) the staged kernel takes, both bag numberings, batches that do not
+# fill the last warp, ids so skewed that most rows of a batch repeat one id.
+@pytest.mark.parametrize("table_major", [False, True])
+@pytest.mark.parametrize("d,Z,M", [(16, 4, 4096), (128, 128, 1280), (128, 32, 129), (128, 1, 4099), (64, 16, 70),
+                                   (100, 32, 1013), (12, 5, 64), (33, 1, 64), (16, 64, 1000), (1, 1, 1)])
+def test_backward_merged_rows_kernel(d, Z, M, table_major):
+    for vocab, dist_, batch in (((50, 7, 1000), "uniform", 131), ((3, 2, 40), "zipf1.05", 200), ((1, 1, 1), "uniform", 65)):
+        w = small(d=d, Z=Z, M=M, batch=batch, vocab_arg=vocab, id_dist=dist_)
+        with Case(w, table_major=table_major) as c:
+            rng = np.random.default_rng(8)
+            shape = (c.T, c.B, d) if table_major else (c.B, c.T, d)
+            g_h = rng.standard_normal(shape).astype(np.float32)
+            gi_h = rng.integers(-4, 5, size=shape).astype(np.float32)
+            delta64, l1 = c.oracle.backward_f64(g_h, c.indices_h, c.offsets_h, c.B)
+            di, _ = c.oracle.backward_f64(gi_h, c.indices_h, c.offsets_h, c.B)
+            ga = c.backward(torch.from_numpy(g_h).to(c.dev), "atomic", kernel=5).cpu().numpy()
+            assert_within_l1(ga, delta64, l1, what=f"merged rows d={d} Z={Z} M={M} {dist_} tm={table_major}")
+            assert_bits_equal(c.backward(torch.from_numpy(gi_h).to(c.dev), "atomic", kernel=5).cpu().numpy(),
+                              di.astype(np.float32), "merged rows, integer gradient")
+    with Case(small(d=d, Z=Z, M=M, bag_rule=(3, 0, 9))) as c:  # pooled input is refused
+        _, g_d = _grad(c, 1)
+        with pytest.raises(robe.RobeError):
+            c.backward(g_d, "atomic", kernel=5)
 
 
 @pytest.mark.parametrize("mode", ["atomic", "det"])
@@ -501,6 +574,9 @@ def test_cfg3_forward_backward_full_size(Z):
         delta64, l1 = c.oracle.backward_f64(g_h, c.indices_h, c.offsets_h, c.B)
         ga = c.backward(g_d, "atomic").cpu().numpy()
         assert_within_l1(ga, delta64, l1, what=f"cfg3 Z={Z} atomic")
+        for kernel in ((3, 4, 5) if Z == 128 else (5,)):
+            gv = c.backward(g_d, "atomic", kernel=kernel).cpu().numpy()
+            assert_within_l1(gv, delta64, l1, what=f"cfg3 Z={Z} atomic, kernel {kernel}")
         det = c.backward(g_d, "det").cpu().numpy()
         assert_within_l1(det, delta64, l1, what=f"cfg3 Z={Z} det vs fp64")
         assert_bits_equal(c.backward(g_d, "det").cpu().numpy(), det, "cfg3 det repeat")
@@ -544,6 +620,9 @@ def test_cfg4_forward_backward_full_size():
         delta64, l1 = c.oracle.backward_f64(g_h, c.indices_h, c.offsets_h, c.B)
         ga = c.backward(g_d, "atomic").cpu().numpy()
         assert_within_l1(ga, delta64, l1, what="cfg4 atomic")
+        gv = c.backward(g_d, "atomic", kernel=3).cpu().numpy()
+        assert_within_l1(gv, delta64, l1, what="cfg4 atomic, 16-byte reductions")
+        del gv
         gb = c.backward(g_d, "binned").cpu().numpy()
         assert_within_l1(gb, delta64, l1, what="cfg4 binned")
         before = c.array_h.copy()
