@@ -311,7 +311,13 @@ def run_ours(args, w):
     if table_major:
         robe.robe_set_option(h, robe.ROBE_OPT_BAG_LAYOUT, robe.ROBE_BAGS_TABLE_MAJOR)
     robe.robe_set_option(h, robe.ROBE_OPT_FWD_KERNEL, args.fwd_kernel)
+    if (args.bwd_kernel == 0 and not bags and w.id_dist.startswith("zipf") and min(w.Z, w.d) >= 64 and d <= 128):
+        # skewed ids, long blocks: the repeats of an id are merged in the warp (the caller knows its
+        # ids; the library cannot tell from the shapes)
+        args.bwd_kernel = 5
     robe.robe_set_option(h, robe.ROBE_OPT_BWD_KERNEL, args.bwd_kernel)
+    l2_keep = args.l2_keep
+    robe.robe_set_option(h, robe.ROBE_OPT_ARRAY_L2_KEEP, l2_keep)
     lr = 1.0  # the paper trains its DLRM with plain SGD at learning rate 1.0 (Section 5)
     ws = None
     bwd_launches = 1
@@ -418,12 +424,15 @@ def run_ours(args, w):
     # from pinned host memory and the output of step i-1 goes back - what a caller that feeds the
     # library from the host would do.  Every byte of every step still crosses the bus inside
     # the timed region.
-    h_ids = [torch.from_numpy(b[0]).to(id_dtype).pin_memory() for b in batches]
+    # ids cross the bus as int32 when they fit (ROBE_OPT_INDEX_TYPE = ROBE_I32: half the id bytes)
+    e2e_id_dtype = torch.int32 if max(int(b[0].max()) if len(b[0]) else 0 for b in batches) < 2**31 else id_dtype
+    e2e_id_bytes = 4 if e2e_id_dtype == torch.int32 else 8
+    h_ids = [torch.from_numpy(b[0]).to(e2e_id_dtype).pin_memory() for b in batches]
     h_offs = [None if b[1] is None else torch.from_numpy(b[1]).pin_memory() for b in batches]
     h_grad = grad_out.cpu().pin_memory()
     h_out = [torch.empty(B, T, d, dtype=torch.float32).pin_memory() for _ in range(2)]
     max_nnz = max(len(b[0]) for b in batches)
-    e_ids = [torch.empty(max_nnz, dtype=id_dtype, device=dev) for _ in range(2)]
+    e_ids = [torch.empty(max_nnz, dtype=e2e_id_dtype, device=dev) for _ in range(2)]
     e_offs = [torch.empty(nbags + 1, dtype=torch.int64, device=dev) if bags else None for _ in range(2)]
     e_grad = [torch.empty_like(grad_out) for _ in range(2)]
     e_out = [torch.empty_like(out) for _ in range(2)]
@@ -474,7 +483,7 @@ def run_ours(args, w):
     barrier()
     e2e_ms = s0.elapsed_time(s1)
     e2e_nnz = float(np.mean([len(batches[i % NB][0]) for i in range(e2e_steps)]))
-    h2d = int(id_bytes * e2e_nnz + (8 * (nbags + 1) if bags else 0) + 4 * nbags * d)
+    h2d = int(e2e_id_bytes * e2e_nnz + (8 * (nbags + 1) if bags else 0) + 4 * nbags * d)
     d2h = int(4 * nbags * d)
 
     # ---- max over ranks --------------------------------------------------------------------
@@ -548,7 +557,7 @@ def run_ours(args, w):
         "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": w.name, "num_tables": T, "d": d, "Z": w.Z, "M": w.M, "batch_per_gpu": B,
-                   "ids_per_step_per_gpu": nnz_per_step, "ids": args.ids, "fwd_kernel": args.fwd_kernel,
+                   "ids_per_step_per_gpu": nnz_per_step, "ids": args.ids, "fwd_kernel": args.fwd_kernel, "l2_keep": l2_keep,
                    "bwd_kernel": args.bwd_kernel, "bags": bags, "bag_layout": args.bag_layout,
                    "backward": {"atomic": "atomic", "det": "deterministic", "binned": "binned atomic"}[args.backward] +
                    (", SGD fused" if dense is None else (", dense fp32 gradient, all-reduce, dense SGD apply" if dp_step
@@ -560,6 +569,7 @@ def run_ours(args, w):
         "clocks": clocks,
         "e2e": {"value": job_e2e_ids / (e2e_ms * 1e-3), "unit": UNIT,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
+                "ids": "int32" if e2e_id_bytes == 4 else "int64",
                 "ms_per_step": e2e_ms / e2e_steps},
         "gpu_launches": (1 + bwd_launches + (1 if dp_step else 0)) * args.steps,
         # ONE kernel: the forward gather (the largest single kernel of the step by the ncu launch
@@ -606,6 +616,9 @@ def main():
                     help="ROBE_OPT_FWD_KERNEL: 0 automatic, 1 direct, 2 staged (4-byte loads), 3 vector (16-byte loads)")
     ap.add_argument("--bwd-kernel", type=int, default=0,
                     help="ROBE_OPT_BWD_KERNEL of the atomic backward: 0 automatic, 1 direct, 2 staged, others see robe.h")
+    ap.add_argument("--l2-keep", type=int, default=0, choices=[0, 1, 2],
+                    help="ROBE_OPT_ARRAY_L2_KEEP: 0 automatic (the backward's reductions carry the L2 evict-last "
+                         "policy), 1 off, 2 on for the forward's loads too")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--dp-step", default="auto", choices=["auto", "on", "off"],
                     help="data-parallel step (backward into a dense gradient, all-reduce over the ranks, dense "

@@ -78,8 +78,7 @@ typedef enum {
                                  A variant asked for a call it cannot take returns
                                  ROBE_ERR_UNSUPPORTED and launches nothing.                          */
 #define ROBE_OPT_BWD_KERNEL 5 /* kernel of the ATOMIC backward (all within the atomic bound):
-                                 0 automatic (default): lane-hashed for Z <= 2 on arrays of up to
-                                   192 MB, staged for d <= 128, else direct
+                                 0 automatic (default): staged for d <= 128, else direct
                                  1 direct   2 staged (scalar red.global.add.f32, lanes on consecutive slots)
                                  3 vector: red.global.add.v4.f32 on the aligned middle of a block,
                                    scalar head and tail; d, Z, M multiples of 4, d <= 128, sign off
@@ -90,7 +89,8 @@ typedef enum {
                                    registers and issues one reduction per element for all of them -
                                    pays for skewed (Zipf) ids with long blocks (Z = 128: 1.34 x), costs
                                    10-40 % on uniform ids, so it is the caller's choice
-                                 6 lane-hashed: d <= 128, Z <= d, sign off                            */
+                                 6 lane-hashed: d <= 128, Z <= d, sign off (the reductions, not the
+                                   hashing, bound this pass: measured no faster than 2)              */
 
 #define ROBE_OPT_INDEX_TYPE 6 /* ROBE_I64 (default) | ROBE_I32: element type of `indices` in the
                                  calls that follow (offsets stay int64)                   */
@@ -102,6 +102,16 @@ typedef enum {
                                  that follow; offsets index bags in the chosen order.              */
 #define ROBE_BAGS_SAMPLE_MAJOR 0
 #define ROBE_BAGS_TABLE_MAJOR 1
+
+#define ROBE_OPT_ARRAY_L2_KEEP 8 /* L2 cache policy "evict these lines last" (createpolicy ...
+                                    L2::evict_last) on the accesses to the array or gradient array;
+                                    results are unchanged.
+                                    0 automatic (default): on the reductions of the atomic and the
+                                      binned backward (a target about the size of the L2 then stays
+                                      there next to the streamed ids and gradient rows: 19-35 % faster
+                                      on a 100 MB array, no slower elsewhere), not on the forward's loads
+                                      (measured: no effect)
+                                    1 off everywhere      2 on for both                              */
 
 /* index element types */
 #define ROBE_I64 0

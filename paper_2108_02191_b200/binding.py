@@ -33,6 +33,7 @@ ROBE_OPT_VALIDATE = 3
 ROBE_OPT_FWD_KERNEL = 4
 ROBE_OPT_BWD_KERNEL = 5
 ROBE_OPT_INDEX_TYPE = 6
+ROBE_OPT_ARRAY_L2_KEEP = 8
 
 ROBE_I64 = 0
 ROBE_I32 = 1

@@ -29,6 +29,7 @@ struct robe_ctx {
     int32_t* status_word;
     int index_type;
     int bag_layout;
+    int l2_keep;
     // second stream of the deterministic backward, made at the first call that can use it
     bool side_tried;
     int side_device;  // the device the stream and events below belong to
@@ -110,6 +111,7 @@ Problem make_problem(robe_ctx* h, const void* indices, const int64_t* offsets, i
     pb.nbags = batch * (int64_t)h->T;
     pb.nnz = nnz;
     pb.status = (h->validate && h->status_word) ? h->status_word : nullptr;
+    pb.l2_keep = h->l2_keep == 2 ? 1 : 0;  // (forward loads; the backward calls decide below)
     return pb;
 }
 
@@ -224,6 +226,7 @@ int robe_create(robe_handle_t* out, uint64_t M, uint32_t Z, uint32_t d, uint32_t
     h->status_word = nullptr;
     h->index_type = ROBE_I64;
     h->bag_layout = ROBE_BAGS_SAMPLE_MAJOR;
+    h->l2_keep = 0;
     h->side_tried = false;
     h->side_device = -1;
     h->side = nullptr;
@@ -261,7 +264,7 @@ int robe_set_option(robe_handle_t h, int key, int64_t value) {
             h->validate = (int)value;
             return ROBE_OK;
         case ROBE_OPT_FWD_KERNEL:
-            if (value < 0 || value > 4) return ROBE_ERR_INVALID_ARG;
+            if (value < 0 || value > 5) return ROBE_ERR_INVALID_ARG;
             h->fwd_variant = (int)value;
             return ROBE_OK;
         case ROBE_OPT_INDEX_TYPE:
@@ -271,6 +274,10 @@ int robe_set_option(robe_handle_t h, int key, int64_t value) {
         case ROBE_OPT_BAG_LAYOUT:
             if (value != ROBE_BAGS_SAMPLE_MAJOR && value != ROBE_BAGS_TABLE_MAJOR) return ROBE_ERR_INVALID_ARG;
             h->bag_layout = (int)value;
+            return ROBE_OK;
+        case ROBE_OPT_ARRAY_L2_KEEP:
+            if (value < 0 || value > 2) return ROBE_ERR_INVALID_ARG;
+            h->l2_keep = (int)value;
             return ROBE_OK;
         case ROBE_OPT_BWD_KERNEL:
             if (value < 0 || value > 6) return ROBE_ERR_INVALID_ARG;
@@ -339,10 +346,10 @@ int robe_forward_keep(robe_handle_t h, const void* indices, const int64_t* offse
     if (((uintptr_t)workspace & 255u) != 0) return ROBE_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
     if (launch_validate(pb, st) != cudaSuccess) return ROBE_ERR_CUDA;
-    uint32_t *keys = nullptr, *vals = nullptr;
-    if (nnz > 0 && batch > 0) block_key_buffers(pb, workspace, &keys, &vals);
+    uint32_t *keys = nullptr, *bag_of = nullptr;
+    if (nnz > 0 && batch > 0) block_key_buffers(pb, workspace, &keys, &bag_of);
     bool kept = false;
-    const int frc = launch_status(launch_forward(pb, out, h->fwd_variant, st, keys, vals, &kept));
+    const int frc = launch_status(launch_forward(pb, out, h->fwd_variant, st, keys, bag_of, &kept));
     if (frc != ROBE_OK) return frc;
     // a forward kernel that keeps nothing (rows longer than 128): the backward's own key kernels
     if (!kept && launch_block_keys(pb, workspace, workspace_bytes, st) != cudaSuccess) return ROBE_ERR_CUDA;
@@ -369,6 +376,7 @@ static int backward_any(robe_handle_t h, const float* grad_out, const void* indi
     }
     float* target = sgd ? (float*)h->array : grad_array;
     Problem pb = make_problem(h, indices, offsets, batch, nnz);
+    pb.l2_keep = h->l2_keep != 1 ? 1 : 0;  // the reductions of the atomic and the binned backward
     cudaStream_t st = (cudaStream_t)stream;
     if (h->bwd_mode == ROBE_BWD_ATOMIC) {
         if (launch_validate(pb, st) != cudaSuccess) return ROBE_ERR_CUDA;

@@ -22,7 +22,9 @@ struct BwdArgs {
     int64_t nbags;
     int64_t nnz;
     const int32_t* status;
+    int l2_keep;  // the reductions carry the L2 "keep" policy
 };
+
 
 template <bool SIGN>
 __global__ void __launch_bounds__(256) bwd_atomic_direct_kernel(BwdArgs a) {
@@ -34,6 +36,7 @@ __global__ void __launch_bounds__(256) bwd_atomic_direct_kernel(BwdArgs a) {
     int64_t lo, hi;
     bag_range(a.offsets, a.nnz, k, lo, hi);
     const uint32_t e = table_of_bag((uint64_t)k, mp);
+    const uint64_t pol = l2_keep_policy(a.l2_keep != 0);
     for (uint32_t i = lane; i < mp.d; i += 32) {
         uint32_t c, o;
         chunk_of(mp, i, c, o);
@@ -44,7 +47,7 @@ __global__ void __launch_bounds__(256) bwd_atomic_direct_kernel(BwdArgs a) {
             if (j >= mp.m) j -= mp.m;
             float t = gv;
             if (SIGN) t = sign_of(mp, hash_base(mp.g, e, x), i) * t;
-            if (ROBE_CHK(j < mp.m, ROBE_DBG_ARRAY_SLOT)) atomicAdd(a.target + j, t);
+            if (ROBE_CHK(j < mp.m, ROBE_DBG_ARRAY_SLOT)) red_add(a.target + j, t, pol);
         }
     }
 }
@@ -119,6 +122,7 @@ bwd_atomic_staged_kernel(BwdArgs a, uint32_t ids_per_batch, uint32_t cmagic) {
     }
     const uint32_t* start_s = sm.start[w];
     const uint64_t* gbase_s = sm.base[w] + kStageIds / 2;
+    const uint64_t pol = l2_keep_policy(a.l2_keep != 0);
 
     for (int64_t p0 = lo; p0 < hi; p0 += (int64_t)ids_per_batch * pstride) {
         const int64_t left = (hi - p0 + pstride - 1) / pstride;
@@ -164,7 +168,7 @@ bwd_atomic_staged_kernel(BwdArgs a, uint32_t ids_per_batch, uint32_t cmagic) {
                 if (live[u] && ROBE_CHK(j < mp.m, ROBE_DBG_ARRAY_SLOT)) {
                     float t = gv[u];
                     if (SIGN) t = sign_of(mp, gbase_s[g], lane + 32u * u) * t;
-                    atomicAdd(a.target + j, t);
+                    red_add(a.target + j, t, pol);
                 }
             }
         }
@@ -370,6 +374,7 @@ bwd_atomic_lanehash_kernel(BwdArgs a, uint32_t padj) {
     LaneChunks<EPL> lc;
     lc.init(mp, lane, padj);
     const uint32_t m = mp.m;
+    const uint64_t pol = l2_keep_policy(a.l2_keep != 0);
     const int64_t nwarps = (int64_t)gridDim.x * 8;
     const int64_t gw = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
 
@@ -380,7 +385,7 @@ bwd_atomic_lanehash_kernel(BwdArgs a, uint32_t padj) {
         for (int u = 0; u < EPL; ++u)
             if (lc.live[u]) {
                 const uint32_t j = lc.template slot<M30>(u, bm_g, thr_g);
-                if (ROBE_CHK(j < m, ROBE_DBG_ARRAY_SLOT)) atomicAdd(a.target + j, gv[u]);
+                if (ROBE_CHK(j < m, ROBE_DBG_ARRAY_SLOT)) red_add(a.target + j, gv[u], pol);
             }
     };
 
@@ -486,15 +491,16 @@ static void launch_bwd_staged_epl(const BwdArgs& a, bool bags, bool sign, cudaSt
 cudaError_t launch_backward_atomic(const Problem& pb, const float* grad_out, float* target,
                                    float scale, int variant, cudaStream_t st) {
     if (pb.nbags == 0) return cudaSuccess;
-    BwdArgs a{pb.mp, grad_out, pb.indices, pb.offsets, target, scale, pb.nbags, pb.nnz, pb.status};
+    BwdArgs a{pb.mp, grad_out, pb.indices, pb.offsets, target, scale, pb.nbags, pb.nnz, pb.status, pb.l2_keep};
     const bool bags = pb.offsets != nullptr;
     const bool warp_ok = pb.mp.d <= 128;
     if (variant == 2 && !warp_ok) return cudaErrorInvalidValue;
-    // short blocks: every lane hashes its own chunks (6; automatic for Z <= 2 on arrays of L2 size,
-    // where the staged kernel is bound by its instruction count)
+    // Short blocks: every lane hashes its own chunks.  Never the automatic choice: unlike the forward,
+    // the backward at Z <= 2 is bound by the reductions themselves, not by instruction issue (measured
+    // on B200 against the staged kernel: 1 MB array Z=1 2.28 -> 2.45 ms, Z=2 1.61 -> 1.43 ms, 100 MB
+    // 5.03 -> 5.66 / 3.24 -> 3.42 ms, Zipf ids Z=1 0.91 -> 0.97 ms).
     const bool lane_ok = pb.sign == 0 && pb.mp.R == 1 && warp_ok;
-    const bool l2_sized = (uint64_t)pb.mp.m * 4u <= (192ull << 20);
-    if (variant == 6 || (variant == 0 && pb.mp.Z <= 2 && l2_sized && lane_ok)) {
+    if (variant == 6) {
         if (!lane_ok) return cudaErrorInvalidValue;
         launch_bwd_lanehash(a, bags, st);
         return cudaGetLastError();

@@ -1,8 +1,9 @@
 // Deterministic backward (Section 3.1 backward equation, evaluated in a fixed order).
 //
 // Blocks are numbered q = p*C + c in input order (p = position in indices, c = chunk).
-//   1. key kernel      key[q] = h(e, x_p, c); val[q] = where the block's gradient elements
-//                      start in grad_out (sign off) or q itself (sign on)
+//   1. key kernel      key[q] = h(e, x_p, c) (or left by the forward of the same step).  The payload
+//                      val[q] - where the block's gradient elements start in grad_out (sign off) or q
+//                      itself (sign on) - is not stored: the first sort pass derives it from q
 //   2. radix sort      stable LSD sort of (key, val) by key - our own passes: digit count per
 //                      CTA range, per-digit exclusive scan, ranked scatter through shared
 //                      memory (so that every digit's run leaves the CTA as one coalesced piece)
@@ -74,12 +75,10 @@ __global__ void __launch_bounds__(256) det_bag_of_kernel(KeyArgs a, uint32_t* ba
     for (int64_t p = lo + lane; p < hi; p += 32) bag_of[p] = (uint32_t)k;
 }
 
-// key[q] = h(e, x_p, c) for q = p*C + c.  val[q] = q when the sign hash is on (the apply kernel
-// then needs the id again), else the position bag*d + c*Z of the block's first gradient element.
+// key[q] = h(e, x_p, c) for q = p*C + c.
 // One thread per id: the part of the hash that all chunks of the id share is evaluated once.
-template <bool SIGN>
 __global__ void __launch_bounds__(256)
-det_keys_kernel(KeyArgs a, const uint32_t* bag_of, uint32_t* keys, uint32_t* vals) {
+det_keys_kernel(KeyArgs a, const uint32_t* bag_of, uint32_t* keys) {
     const uint64_t p = (uint64_t)blockIdx.x * 256 + threadIdx.x;
     if (p >= (uint64_t)a.nnz) return;
     const MapParams& mp = a.mp;
@@ -89,23 +88,19 @@ det_keys_kernel(KeyArgs a, const uint32_t* bag_of, uint32_t* keys, uint32_t* val
     const uint64_t q0 = p * mp.C;
     if (mp.R > 1) {  // rows clubbed into one block: a single key
         keys[q0] = id_block_start(mp, e, x, 0);
-        vals[q0] = SIGN ? (uint32_t)q0 : (uint32_t)(bag * mp.d);
         return;
     }
     const uint64_t base = hash_base(mp.h, e, x);
     for (uint32_t c = 0; c < mp.C; ++c) {
         if (!ROBE_CHK(q0 + c < (uint64_t)a.nnz * mp.C, ROBE_DBG_SORT_POS)) break;
         keys[q0 + c] = block_start(mp, base, c);
-        vals[q0 + c] = SIGN ? (uint32_t)(q0 + c) : (uint32_t)(bag * mp.d + c * mp.Z);
     }
 }
 
 // The same, one thread per block: for many blocks per id (small Z) the writes of one thread per
 // id would be far apart, and re-evaluating the shared part of the hash per block costs less.
-template <bool SIGN>
 __global__ void __launch_bounds__(256)
-det_keys_by_block_kernel(KeyArgs a, const uint32_t* bag_of, uint32_t* keys, uint32_t* vals,
-                         uint64_t nb) {
+det_keys_by_block_kernel(KeyArgs a, const uint32_t* bag_of, uint32_t* keys, uint64_t nb) {
     const uint64_t q = (uint64_t)blockIdx.x * 256 + threadIdx.x;
     if (q >= nb) return;
     const MapParams& mp = a.mp;
@@ -115,8 +110,21 @@ det_keys_by_block_kernel(KeyArgs a, const uint32_t* bag_of, uint32_t* keys, uint
     const uint32_t e = table_of_bag(bag, mp);
     const uint64_t x = (uint64_t)a.indices.load(p);
     keys[q] = id_block_start(mp, e, x, c);
-    vals[q] = SIGN ? (uint32_t)q : (uint32_t)(bag * mp.d + c * mp.Z);
 }
+
+// The payload of block q = p*C + c, as the first sort pass derives it: q itself when the sign hash
+// is on (the apply kernel then needs the id again), else the position bag*d + c*Z of the block's
+// first gradient element, bag = bag_of[p] (pooled input) or p (one-hot).
+struct PayloadGen {
+    const uint32_t* bag_of;
+    uint32_t C, d, Z, sign;
+    __device__ __forceinline__ uint32_t operator()(uint32_t q) const {
+        if (sign) return q;
+        const uint32_t p = q / C, c = q - p * C;
+        const uint32_t bag = bag_of != nullptr ? __ldg(bag_of + p) : p;
+        return bag * d + c * Z;
+    }
+};
 
 // ---- radix sort pass, kernel 1: digit histogram of each CTA's contiguous key range
 __global__ void __launch_bounds__(kSortThreads)
@@ -189,7 +197,9 @@ __global__ void __launch_bounds__(kSortThreads, 4)
 sort_scatter_kernel(const uint32_t* __restrict__ kin, const uint32_t* __restrict__ vin,
                     uint32_t* __restrict__ kout, uint32_t* __restrict__ vout,
                     const uint32_t* __restrict__ cta_offsets, const uint32_t* __restrict__ totals,
-                    uint64_t nb, uint64_t tiles, uint32_t shift, uint32_t mask) {
+                    uint64_t nb, uint64_t tiles, uint32_t shift, uint32_t mask, PayloadGen gen) {
+    // vin == nullptr: first pass of a sort, the pairs are still in block order and the payload of
+    // the pair at position q is gen(q)
     __shared__ uint32_t skey[kSortTile];
     __shared__ uint32_t sval[kSortTile];
     __shared__ uint32_t wcnt[kSortWarps][kRadix];
@@ -267,7 +277,8 @@ sort_scatter_kernel(const uint32_t* __restrict__ kin, const uint32_t* __restrict
                 const uint32_t lp = dstart[dg] + wcnt[w][dg] + rank[r];
                 if (!ROBE_CHK(lp < (uint32_t)kSortTile, ROBE_DBG_SHARED)) continue;
                 skey[lp] = key[r];
-                sval[lp] = vin[idx];  // payloads are only passed through: read them this late
+                // payloads are only passed through: read them this late
+                sval[lp] = vin != nullptr ? vin[idx] : gen((uint32_t)idx);
             }
         }
         __syncthreads();
@@ -316,6 +327,7 @@ struct ApplyArgs {
     const uint32_t* any_left;  // number of windows left over (0: the tile kernel has nothing to do)
     uint32_t win_log2;         // log2 of the window length
     uint64_t grad_elems;       // elements of grad_out (read by the debug build's index checks only)
+    int l2_keep;               // binned adds: the reductions carry the L2 "keep" policy
 };
 
 // The term that the sorted block with payload v contributes to the slot at in-block offset o
@@ -1039,6 +1051,7 @@ binned_apply_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint32_t*
         k[t] = __ldg(K + i);
         v[t] = __ldg(V + i);
     }
+    const uint64_t pol = l2_keep_policy(a.l2_keep != 0);
     float term[kBinnedPer];
     bool ok[kBinnedPer];
 #pragma unroll
@@ -1049,7 +1062,7 @@ binned_apply_kernel(ApplyArgs a, const uint32_t* __restrict__ K, const uint32_t*
         if (ok[t]) {
             uint64_t j = (uint64_t)k[t] + u;
             if (j >= mp.m) j -= mp.m;
-            if (ROBE_CHK(j < mp.m, ROBE_DBG_ARRAY_SLOT)) atomicAdd(a.target + j, a.lr * term[t]);
+            if (ROBE_CHK(j < mp.m, ROBE_DBG_ARRAY_SLOT)) red_add(a.target + j, a.lr * term[t], pol);
         }
     }
 }
@@ -1186,11 +1199,12 @@ size_t det_workspace_bytes(const MapParams& mp, int64_t nbags, int64_t nnz, bool
     return make_layout(nb, nnz, bags, mp.m).total;
 }
 
-void block_key_buffers(const Problem& pb, void* workspace, uint32_t** keys, uint32_t** vals) {
+void block_key_buffers(const Problem& pb, void* workspace, uint32_t** keys, uint32_t** bag_of) {
     const uint64_t nb = (uint64_t)pb.nnz * pb.mp.C;
-    const Layout L = make_layout(nb, pb.nnz, pb.offsets != nullptr, pb.mp.m);
+    const bool bags = pb.offsets != nullptr;
+    const Layout L = make_layout(nb, pb.nnz, bags, pb.mp.m);
     *keys = (uint32_t*)((char*)workspace + L.keysA);
-    *vals = (uint32_t*)((char*)workspace + L.valsA);
+    *bag_of = bags ? (uint32_t*)((char*)workspace + L.bag_of) : nullptr;
 }
 
 // bag_of (pooled input) into the workspace
@@ -1212,18 +1226,13 @@ cudaError_t launch_block_keys(const Problem& pb, void* workspace, size_t workspa
     if (workspace == nullptr || workspace_bytes < L.total) return cudaErrorInvalidValue;
     char* ws = (char*)workspace;
     uint32_t* kA = (uint32_t*)(ws + L.keysA);
-    uint32_t* vA = (uint32_t*)(ws + L.valsA);
     uint32_t* bag_of = bags ? (uint32_t*)(ws + L.bag_of) : nullptr;
     KeyArgs ka{mp, pb.indices, pb.offsets, pb.nbags, pb.nnz, pb.status};
     if (bags) launch_bag_of(pb, L, ws, st);
     if (mp.C <= 8) {
-        const unsigned kb = (unsigned)((pb.nnz + 255) / 256);
-        if (pb.sign) det_keys_kernel<true><<<kb, 256, 0, st>>>(ka, bag_of, kA, vA);
-        else det_keys_kernel<false><<<kb, 256, 0, st>>>(ka, bag_of, kA, vA);
+        det_keys_kernel<<<(unsigned)((pb.nnz + 255) / 256), 256, 0, st>>>(ka, bag_of, kA);
     } else {
-        const unsigned kb = (unsigned)((nb + 255) / 256);
-        if (pb.sign) det_keys_by_block_kernel<true><<<kb, 256, 0, st>>>(ka, bag_of, kA, vA, nb);
-        else det_keys_by_block_kernel<false><<<kb, 256, 0, st>>>(ka, bag_of, kA, vA, nb);
+        det_keys_by_block_kernel<<<(unsigned)((nb + 255) / 256), 256, 0, st>>>(ka, bag_of, kA, nb);
     }
     return cudaGetLastError();
 }
@@ -1248,12 +1257,11 @@ cudaError_t launch_backward_det(const Problem& pb, const float* grad_out, float*
     uint32_t* counts = (uint32_t*)(ws + L.counts);
     uint32_t* totals = (uint32_t*)(ws + L.totals);
 
-    if (!keys_kept) {
+    if (!keys_kept) {  // (else the forward of the step left the block starts and the bags of the ids)
         const cudaError_t err = launch_block_keys(pb, workspace, workspace_bytes, st);
         if (err != cudaSuccess) return err;
-    } else if (bags && pb.sign) {
-        launch_bag_of(pb, L, ws, st);  // the signed terms look the id's bag up again
     }
+    const PayloadGen gen{bag_of, mp.C, mp.d, mp.Z, pb.sign ? 1u : 0u};
 
     const SortPlan sp = make_plan(nb);
     const uint32_t bits = bits_for(mp.m);
@@ -1266,10 +1274,10 @@ cudaError_t launch_backward_det(const Problem& pb, const float* grad_out, float*
         const uint32_t mask = (1u << (bits - shift)) - 1u;
         sort_count_kernel<<<sp.grid, kSortThreads, 0, st>>>(kA, counts, nb, sp.tiles, shift, mask);
         sort_scan_kernel<<<kRadix, kSortThreads, 0, st>>>(counts, totals, sp.grid);
-        sort_scatter_kernel<false><<<sp.grid, kSortThreads, 0, st>>>(kA, vA, kB, vB, counts, totals, nb,
-                                                                    sp.tiles, shift, mask);
+        sort_scatter_kernel<false><<<sp.grid, kSortThreads, 0, st>>>(kA, nullptr, kB, vB, counts, totals, nb,
+                                                                    sp.tiles, shift, mask, gen);
         ApplyArgs ab{mp, grad_out, pb.indices, target, lr, nb, pb.status, AdamState{}, nullptr, nullptr, 0,
-                     nullptr, nullptr, 0, (uint64_t)pb.nbags * mp.d};
+                     nullptr, nullptr, 0, (uint64_t)pb.nbags * mp.d, pb.l2_keep};
         uint32_t log2Zp = 0;
         while ((1u << log2Zp) < mp.Z) ++log2Zp;
         const uint64_t groups = (nb + kBinnedPer - 1) / kBinnedPer;
@@ -1292,8 +1300,8 @@ cudaError_t launch_backward_det(const Problem& pb, const float* grad_out, float*
         const uint32_t mask = (1u << width) - 1u;
         sort_count_kernel<<<sp.grid, kSortThreads, 0, st>>>(kA, counts, nb, sp.tiles, shift, mask);
         sort_scan_kernel<<<kRadix, kSortThreads, 0, st>>>(counts, totals, sp.grid);
-        sort_scatter_kernel<true><<<sp.grid, kSortThreads, 0, st>>>(kA, vA, kB, vB, counts, totals, nb,
-                                                             sp.tiles, shift, mask);
+        sort_scatter_kernel<true><<<sp.grid, kSortThreads, 0, st>>>(kA, pass == 0 ? nullptr : vA, kB, vB, counts,
+                                                                   totals, nb, sp.tiles, shift, mask, gen);
         uint32_t* t = kA; kA = kB; kB = t;
         t = vA; vA = vB; vB = t;
     }
@@ -1302,7 +1310,7 @@ cudaError_t launch_backward_det(const Problem& pb, const float* grad_out, float*
     cudaMemsetAsync(long_count, 0, 2 * sizeof(uint32_t), st);  // [0] rounds handed over, [1] rounds taken
     ApplyArgs aa{mp, grad_out, pb.indices, target, lr, nb, pb.status, adam ? *adam : AdamState{},
                  long_count, (LongWalk*)(ws + L.long_walks), L.long_cap, nullptr, nullptr, 0,
-                 (uint64_t)pb.nbags * mp.d};
+                 (uint64_t)pb.nbags * mp.d, 0};
     const WindowBuffers wb{(uint32_t*)(ws + L.bounds),
                            (uint32_t*)(ws + L.bounds + align256(((size_t)L.nwin + 1) * sizeof(uint32_t))),
                            (uint8_t*)(ws + L.win_left), L.nwin, L.win_log2,

@@ -191,8 +191,39 @@ __device__ __forceinline__ float load_elem(const void* array, uint32_t j) {
 // Array read of the gather kernels: read-only path, with the 64-byte L2 fetch hint.  Random
 // Z-blocks gain nothing from the wider default fetch; measured on B200 this hint shortens a
 // random 64-byte-block gather from a 1 GB array by about 13 %.
+// L2 cache policy "keep": lines fetched under it are the last to be evicted.  For an array about
+// the size of the L2 that shares it with gigabytes of streamed ids, output rows and gradients.
+// 0 stands for "no policy" (createpolicy never returns 0 for evict_last).
+__device__ __forceinline__ uint64_t l2_keep_policy(bool on) {
+    uint64_t pol = 0;
+    if (on) asm("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+
+// fp32 reduction into global memory, with the L2 "keep" policy when pol != 0 (warp-uniform)
+__device__ __forceinline__ void red_add(float* p, float v, uint64_t pol) {
+    if (pol != 0)
+        asm volatile("red.global.add.L2::cache_hint.f32 [%0], %1, %2;" ::"l"(p), "f"(v), "l"(pol) : "memory");
+    else
+        atomicAdd(p, v);
+}
+
 template <int DT>
-__device__ __forceinline__ float gather_elem(const void* array, uint32_t j) {
+__device__ __forceinline__ float gather_elem(const void* array, uint32_t j, uint64_t pol = 0) {
+    if (pol != 0) {  // (warp-uniform)
+        if (DT == 0) {
+            float v;
+            asm("ld.global.nc.L2::cache_hint.L2::64B.f32 %0, [%1], %2;"
+                : "=f"(v)
+                : "l"((const float*)array + j), "l"(pol));
+            return v;
+        }
+        unsigned short b;
+        asm("ld.global.nc.L2::cache_hint.L2::64B.u16 %0, [%1], %2;"
+            : "=h"(b)
+            : "l"((const unsigned short*)array + j), "l"(pol));
+        return bf16_bits_to_float(b);
+    }
     if (DT == 0) {
         float v;
         asm("ld.global.nc.L2::64B.f32 %0, [%1];" : "=f"(v) : "l"((const float*)array + j));
