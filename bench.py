@@ -429,20 +429,21 @@ def run_ours(args, w):
     e2e_id_bytes = 4 if e2e_id_dtype == torch.int32 else 8
     h_ids = [torch.from_numpy(b[0]).to(e2e_id_dtype).pin_memory() for b in batches]
     h_offs = [None if b[1] is None else torch.from_numpy(b[1]).pin_memory() for b in batches]
+    NBUF = args.e2e_buffers  # sets of device and pinned buffers the steps rotate through
     h_grad = grad_out.cpu().pin_memory()
-    h_out = [torch.empty(B, T, d, dtype=torch.float32).pin_memory() for _ in range(2)]
+    h_out = [torch.empty(B, T, d, dtype=torch.float32).pin_memory() for _ in range(NBUF)]
     max_nnz = max(len(b[0]) for b in batches)
-    e_ids = [torch.empty(max_nnz, dtype=e2e_id_dtype, device=dev) for _ in range(2)]
-    e_offs = [torch.empty(nbags + 1, dtype=torch.int64, device=dev) if bags else None for _ in range(2)]
-    e_grad = [torch.empty_like(grad_out) for _ in range(2)]
-    e_out = [torch.empty_like(out) for _ in range(2)]
+    e_ids = [torch.empty(max_nnz, dtype=e2e_id_dtype, device=dev) for _ in range(NBUF)]
+    e_offs = [torch.empty(nbags + 1, dtype=torch.int64, device=dev) if bags else None for _ in range(NBUF)]
+    e_grad = [torch.empty_like(grad_out) for _ in range(NBUF)]
+    e_out = [torch.empty_like(out) for _ in range(NBUF)]
     s_in, s_comp, s_out = torch.cuda.Stream(dev), torch.cuda.Stream(dev), torch.cuda.Stream(dev)
-    ev_in = [torch.cuda.Event() for _ in range(2)]
-    ev_comp = [torch.cuda.Event() for _ in range(2)]
-    ev_out = [torch.cuda.Event() for _ in range(2)]
+    ev_in = [torch.cuda.Event() for _ in range(NBUF)]
+    ev_comp = [torch.cuda.Event() for _ in range(NBUF)]
+    ev_out = [torch.cuda.Event() for _ in range(NBUF)]
 
     def e2e_step(i):
-        b, k = i % 2, i % NB
+        b, k = i % NBUF, i % NB
         n = h_ids[k].numel()
         ids_d = e_ids[b][:n]
         with torch.cuda.stream(s_in):
@@ -616,9 +617,11 @@ def main():
                     help="ROBE_OPT_FWD_KERNEL: 0 automatic, 1 direct, 2 staged (4-byte loads), 3 vector (16-byte loads)")
     ap.add_argument("--bwd-kernel", type=int, default=0,
                     help="ROBE_OPT_BWD_KERNEL of the atomic backward: 0 automatic, 1 direct, 2 staged, others see robe.h")
-    ap.add_argument("--l2-keep", type=int, default=0, choices=[0, 1, 2],
-                    help="ROBE_OPT_ARRAY_L2_KEEP: 0 automatic (the backward's reductions carry the L2 evict-last "
-                         "policy), 1 off, 2 on for the forward's loads too")
+    ap.add_argument("--l2-keep", type=int, default=0, choices=[0, 1],
+                    help="ROBE_OPT_ARRAY_L2_KEEP: 0 the backward's reductions carry the L2 evict-last policy "
+                         "(default), 1 off")
+    ap.add_argument("--e2e-buffers", type=int, default=2, choices=[2, 3, 4],
+                    help="buffer sets of the end-to-end leg (copies of neighbouring steps overlap the compute)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--dp-step", default="auto", choices=["auto", "on", "off"],
                     help="data-parallel step (backward into a dense gradient, all-reduce over the ranks, dense "

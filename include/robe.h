@@ -103,15 +103,13 @@ typedef enum {
 #define ROBE_BAGS_SAMPLE_MAJOR 0
 #define ROBE_BAGS_TABLE_MAJOR 1
 
-#define ROBE_OPT_ARRAY_L2_KEEP 8 /* L2 cache policy "evict these lines last" (createpolicy ...
-                                    L2::evict_last) on the accesses to the array or gradient array;
-                                    results are unchanged.
-                                    0 automatic (default): on the reductions of the atomic and the
-                                      binned backward (a target about the size of the L2 then stays
-                                      there next to the streamed ids and gradient rows: 19-35 % faster
-                                      on a 100 MB array, no slower elsewhere), not on the forward's loads
-                                      (measured: no effect)
-                                    1 off everywhere      2 on for both                              */
+#define ROBE_OPT_ARRAY_L2_KEEP 8 /* 0 (default) on | 1 off: the reductions of the atomic and the binned
+                                    backward carry the L2 cache policy "evict these lines last"
+                                    (createpolicy ... L2::evict_last), so that a gradient target about
+                                    the size of the L2 stays there next to the streamed ids and gradient
+                                    rows: 19-35 % faster on a 100 MB array, no slower elsewhere.  Results
+                                    are unchanged.  (The same policy on the forward's loads measured no
+                                    effect and is not offered.)                                      */
 
 /* index element types */
 #define ROBE_I64 0

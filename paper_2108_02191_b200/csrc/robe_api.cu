@@ -111,7 +111,7 @@ Problem make_problem(robe_ctx* h, const void* indices, const int64_t* offsets, i
     pb.nbags = batch * (int64_t)h->T;
     pb.nnz = nnz;
     pb.status = (h->validate && h->status_word) ? h->status_word : nullptr;
-    pb.l2_keep = h->l2_keep == 2 ? 1 : 0;  // (forward loads; the backward calls decide below)
+    pb.l2_keep = 0;  // (the backward calls set it)
     return pb;
 }
 
@@ -264,7 +264,7 @@ int robe_set_option(robe_handle_t h, int key, int64_t value) {
             h->validate = (int)value;
             return ROBE_OK;
         case ROBE_OPT_FWD_KERNEL:
-            if (value < 0 || value > 5) return ROBE_ERR_INVALID_ARG;
+            if (value < 0 || value > 4) return ROBE_ERR_INVALID_ARG;
             h->fwd_variant = (int)value;
             return ROBE_OK;
         case ROBE_OPT_INDEX_TYPE:
@@ -276,7 +276,7 @@ int robe_set_option(robe_handle_t h, int key, int64_t value) {
             h->bag_layout = (int)value;
             return ROBE_OK;
         case ROBE_OPT_ARRAY_L2_KEEP:
-            if (value < 0 || value > 2) return ROBE_ERR_INVALID_ARG;
+            if (value != 0 && value != 1) return ROBE_ERR_INVALID_ARG;
             h->l2_keep = (int)value;
             return ROBE_OK;
         case ROBE_OPT_BWD_KERNEL:
@@ -376,7 +376,7 @@ static int backward_any(robe_handle_t h, const float* grad_out, const void* indi
     }
     float* target = sgd ? (float*)h->array : grad_array;
     Problem pb = make_problem(h, indices, offsets, batch, nnz);
-    pb.l2_keep = h->l2_keep != 1 ? 1 : 0;  // the reductions of the atomic and the binned backward
+    pb.l2_keep = h->l2_keep == 0 ? 1 : 0;  // the reductions of the atomic and the binned backward
     cudaStream_t st = (cudaStream_t)stream;
     if (h->bwd_mode == ROBE_BWD_ATOMIC) {
         if (launch_validate(pb, st) != cudaSuccess) return ROBE_ERR_CUDA;

@@ -461,9 +461,8 @@ static bool bwd_vec_ok(const Problem& pb, const float* grad_out, const float* ta
            ((uintptr_t)grad_out & 15u) == 0 && ((uintptr_t)target & 15u) == 0;
 }
 
-template <int EPL, bool SIGN, bool FULLD>
-static void launch_bwd_staged(const BwdArgs& a, bool bags, cudaStream_t st) {
-    constexpr int MINB = (EPL == 4) ? 6 : 8;
+template <int EPL, bool SIGN, bool FULLD, int MINB>
+static void launch_bwd_staged_minb(const BwdArgs& a, bool bags, cudaStream_t st) {
     const uint32_t ipb = staged_ids_per_batch(a.mp, bags, SIGN);
     const uint32_t cmagic = chunk_magic(a.mp);
     const int64_t warps = bags ? a.nbags : (a.nbags + ipb - 1) / ipb;
@@ -472,6 +471,15 @@ static void launch_bwd_staged(const BwdArgs& a, bool bags, cudaStream_t st) {
         bwd_atomic_staged_kernel<EPL, SIGN, true, FULLD, MINB><<<blocks, 256, 0, st>>>(a, ipb, cmagic);
     else
         bwd_atomic_staged_kernel<EPL, SIGN, false, FULLD, MINB><<<blocks, 256, 0, st>>>(a, ipb, cmagic);
+}
+
+template <int EPL, bool SIGN, bool FULLD>
+static void launch_bwd_staged(const BwdArgs& a, bool bags, cudaStream_t st) {
+    const bool l2_sized = (uint64_t)a.mp.m * 4u <= kL2SizedBytes;  // (see kStagedCtas*)
+    if constexpr (SIGN) launch_bwd_staged_minb<EPL, SIGN, FULLD, kStagedCtasSign>(a, bags, st);
+    else if constexpr (EPL == 4) launch_bwd_staged_minb<EPL, SIGN, FULLD, kStagedCtasWide>(a, bags, st);
+    else if (l2_sized) launch_bwd_staged_minb<EPL, SIGN, FULLD, kStagedCtasL2>(a, bags, st);
+    else launch_bwd_staged_minb<EPL, SIGN, FULLD, kStagedCtasHbm>(a, bags, st);
 }
 
 template <int EPL>

@@ -24,8 +24,24 @@ struct FwdArgs {
     const int32_t* status;
     uint32_t* keep_keys;    // block starts kept for the backward, or nullptr
     uint32_t* keep_bag_of;  // with them, pooled input: the bag of every id position
-    int l2_keep;          // array loads carry the L2 "keep" policy
 };
+
+// Kept block starts, pooled input: id positions before the first bag or after the last one (offsets
+// that break the contract offsets[0] = 0, offsets[nbags] = nnz) belong to no warp of the forward
+// kernel; they get block start 0 and bag 0 here, so that the backward reads nothing stale.  With
+// well-formed offsets there is nothing to do.  (A kernel of its own: inside the gather kernel these
+// two loops cost registers that its occupancy has no room for.)
+__global__ void __launch_bounds__(256) keep_gaps_kernel(FwdArgs a) {
+    int64_t lo, hi, lo_last, hi_last;
+    bag_range(a.offsets, a.nnz, 0, lo, hi);
+    bag_range(a.offsets, a.nnz, a.nbags - 1, lo_last, hi_last);
+    const int64_t C = (int64_t)a.mp.C;
+    const int64_t step = (int64_t)gridDim.x * 256, t0 = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    for (int64_t q = t0; q < lo * C; q += step) a.keep_keys[q] = 0;
+    for (int64_t p = t0; p < lo; p += step) a.keep_bag_of[p] = 0;
+    for (int64_t q = hi_last * C + t0; q < a.nnz * C; q += step) a.keep_keys[q] = 0;
+    for (int64_t p = hi_last + t0; p < a.nnz; p += step) a.keep_bag_of[p] = 0;
+}
 
 template <int DT, bool SIGN>
 __global__ void __launch_bounds__(256) fwd_direct_kernel(FwdArgs a) {
@@ -72,7 +88,7 @@ template <int EPL, int DT, bool SIGN, int U, bool WRAP, bool TAIL>
 __device__ __forceinline__ void gather_group(const FwdArgs& a, const uint32_t* const (&col)[EPL],
                                              const uint32_t (&off)[EPL], const bool (&live)[EPL],
                                              const uint64_t* gbase_s, uint32_t g0, uint32_t n,
-                                             uint32_t lane, uint64_t pol, float (&v)[U][EPL]) {
+                                             uint32_t lane, float (&v)[U][EPL]) {
     const MapParams& mp = a.mp;
 #pragma unroll
     for (int gg = 0; gg < U; ++gg) {
@@ -83,7 +99,7 @@ __device__ __forceinline__ void gather_group(const FwdArgs& a, const uint32_t* c
             if (on && live[u]) {
                 uint32_t j = col[u][g0 + gg] + off[u];  // < m + d <= 2^32
                 if (WRAP && j >= mp.m) j -= mp.m;
-                if (ROBE_CHK(j < mp.m, ROBE_DBG_ARRAY_SLOT)) val = gather_elem<DT>(a.array, j, pol);
+                if (ROBE_CHK(j < mp.m, ROBE_DBG_ARRAY_SLOT)) val = gather_elem<DT>(a.array, j);
                 if (SIGN) val = sign_of(mp, gbase_s[g0 + gg], lane + 32u * u) * val;
             }
             v[gg][u] = val;
@@ -97,13 +113,12 @@ template <int EPL, int DT, bool SIGN, bool BAGS, int U, bool WRAP>
 __device__ __forceinline__ void gather_batch(const FwdArgs& a, const uint32_t* const (&col)[EPL],
                                              const uint32_t (&off)[EPL], const bool (&live)[EPL],
                                              const uint64_t* gbase_s, uint32_t cnt, int64_t p0,
-                                             int64_t pstride, uint32_t lane, uint64_t pol,
-                                             float (&acc)[EPL]) {
+                                             uint32_t lane, float (&acc)[EPL]) {
     const MapParams& mp = a.mp;
     uint32_t g0 = 0;
     for (; g0 + U <= cnt; g0 += U) {
         float v[U][EPL];
-        gather_group<EPL, DT, SIGN, U, WRAP, false>(a, col, off, live, gbase_s, g0, U, lane, pol, v);
+        gather_group<EPL, DT, SIGN, U, WRAP, false>(a, col, off, live, gbase_s, g0, U, lane, v);
         if (BAGS) {
 #pragma unroll
             for (int gg = 0; gg < U; ++gg)
@@ -112,7 +127,7 @@ __device__ __forceinline__ void gather_batch(const FwdArgs& a, const uint32_t* c
         } else {
 #pragma unroll
             for (int gg = 0; gg < U; ++gg) {
-                float* orow = a.out + (p0 + (int64_t)(g0 + gg) * pstride) * (int64_t)mp.d;
+                float* orow = a.out + (p0 + g0 + gg) * (int64_t)mp.d;
 #pragma unroll
                 for (int u = 0; u < EPL; ++u)
                     if (live[u]) __stcs(orow + lane + 32u * u, v[gg][u]);
@@ -122,7 +137,7 @@ __device__ __forceinline__ void gather_batch(const FwdArgs& a, const uint32_t* c
     if (g0 < cnt) {
         const uint32_t n = cnt - g0;
         float v[U][EPL];
-        gather_group<EPL, DT, SIGN, U, WRAP, true>(a, col, off, live, gbase_s, g0, n, lane, pol, v);
+        gather_group<EPL, DT, SIGN, U, WRAP, true>(a, col, off, live, gbase_s, g0, n, lane, v);
         if (BAGS) {
 #pragma unroll
             for (int gg = 0; gg < U; ++gg)
@@ -134,7 +149,7 @@ __device__ __forceinline__ void gather_batch(const FwdArgs& a, const uint32_t* c
 #pragma unroll
             for (int gg = 0; gg < U; ++gg)
                 if ((uint32_t)gg < n) {
-                    float* orow = a.out + (p0 + (int64_t)(g0 + gg) * pstride) * (int64_t)mp.d;
+                    float* orow = a.out + (p0 + g0 + gg) * (int64_t)mp.d;
 #pragma unroll
                     for (int u = 0; u < EPL; ++u)
                         if (live[u]) __stcs(orow + lane + 32u * u, v[gg][u]);
@@ -143,12 +158,9 @@ __device__ __forceinline__ void gather_batch(const FwdArgs& a, const uint32_t* c
     }
 }
 
-// by_table (one-hot, sample-major input, nothing kept): a warp takes ids_per_batch rows of ONE table -
-// every T-th row - instead of consecutive rows, neighbouring warps different tables.  The repeats of
-// a table's hot ids then meet in one warp's batch and in one SM's L1.
 template <int EPL, int DT, bool SIGN, bool BAGS, bool FULLD, int MINB, int U>
 __global__ void __launch_bounds__(256, MINB)
-fwd_staged_kernel(FwdArgs a, uint32_t ids_per_batch, uint32_t cmagic, int by_table) {
+fwd_staged_kernel(FwdArgs a, uint32_t ids_per_batch, uint32_t cmagic) {
     __shared__ StageSmem sm;
     const MapParams& mp = a.mp;
     const uint32_t lane = threadIdx.x & 31, w = threadIdx.x >> 5;
@@ -165,34 +177,10 @@ fwd_staged_kernel(FwdArgs a, uint32_t ids_per_batch, uint32_t cmagic, int by_tab
         const uint32_t e_bag = table_of_bag((uint64_t)warp, mp);
         tterm = table_term(mp.h, e_bag);
         if (SIGN) gterm = table_term(mp.g, e_bag);
-    } else if (!by_table) {
+    } else {
         lo = warp * (int64_t)ids_per_batch;  // this warp serves rows [lo, lo + ids_per_batch)
         if (lo >= a.nbags) return;
         hi = lo + ids_per_batch < a.nbags ? lo + ids_per_batch : a.nbags;
-    }
-    int64_t pstride = 1;
-    if (!BAGS && by_table) {  // rows (n0 + t) T + e, t < cnt
-        const int64_t batch = a.nbags / mp.T;
-        const int64_t n0 = (warp / mp.T) * (int64_t)ids_per_batch;
-        if (n0 >= batch) return;
-        const int64_t cnt = n0 + ids_per_batch < batch ? ids_per_batch : batch - n0;
-        pstride = mp.T;
-        lo = n0 * mp.T + warp % mp.T;
-        hi = lo + cnt * pstride;  // (one batch: the loop below runs once)
-    }
-
-    if (BAGS && a.keep_keys != nullptr) {
-        // id positions before the first bag or after the last one (offsets that break the
-        // contract) get block start 0 and bag 0, so that the backward reads nothing stale
-        const int64_t C = (int64_t)mp.C;
-        if (warp == 0) {
-            for (int64_t q = lane; q < lo * C; q += 32) a.keep_keys[q] = 0;
-            for (int64_t p = lane; p < lo; p += 32) a.keep_bag_of[p] = 0;
-        }
-        if (warp == a.nbags - 1) {
-            for (int64_t q = hi * C + lane; q < a.nnz * C; q += 32) a.keep_keys[q] = 0;
-            for (int64_t p = hi + lane; p < a.nnz; p += 32) a.keep_bag_of[p] = 0;
-        }
     }
 
     // per-lane constants of the gather: element i = lane + 32u, its in-block offset, and the
@@ -210,7 +198,6 @@ fwd_staged_kernel(FwdArgs a, uint32_t ids_per_batch, uint32_t cmagic, int by_tab
         col[u] = sm.start[w] + chk * ids_per_batch;
     }
     const uint64_t* gbase_s = sm.base[w] + kStageIds / 2;  // sign-hash bases (sign on only)
-    const uint64_t pol = l2_keep_policy(a.l2_keep != 0);
 
     // -0 + v == v for every v (also v = -0): starting from -0 makes the first term initialise
     // the sum exactly as the definition says
@@ -218,17 +205,16 @@ fwd_staged_kernel(FwdArgs a, uint32_t ids_per_batch, uint32_t cmagic, int by_tab
 #pragma unroll
     for (int u = 0; u < EPL; ++u) acc[u] = -0.0f;
 
-    for (int64_t p0 = lo; p0 < hi; p0 += (int64_t)ids_per_batch * pstride) {
-        const int64_t left = (hi - p0 + pstride - 1) / pstride;
-        const uint32_t cnt = (uint32_t)(left < (int64_t)ids_per_batch ? left : (int64_t)ids_per_batch);
+    for (int64_t p0 = lo; p0 < hi; p0 += ids_per_batch) {
+        const uint32_t cnt = (uint32_t)((hi - p0) < (int64_t)ids_per_batch ? (hi - p0)
+                                                                            : (int64_t)ids_per_batch);
         const bool wraps = stage_batch<SIGN, BAGS>(sm, mp, a.indices, p0, cnt, ids_per_batch, tterm,
                                                    gterm, cmagic, w, lane,
-                                                   KeepBlocks{a.keep_keys, a.keep_bag_of, (uint64_t)warp, (uint64_t)a.nnz * mp.C},
-                                                   pstride);
+                                                   KeepBlocks{a.keep_keys, a.keep_bag_of, (uint64_t)warp, (uint64_t)a.nnz * mp.C});
         if (wraps)
-            gather_batch<EPL, DT, SIGN, BAGS, U, true>(a, col, off, live, gbase_s, cnt, p0, pstride, lane, pol, acc);
+            gather_batch<EPL, DT, SIGN, BAGS, U, true>(a, col, off, live, gbase_s, cnt, p0, lane, acc);
         else
-            gather_batch<EPL, DT, SIGN, BAGS, U, false>(a, col, off, live, gbase_s, cnt, p0, pstride, lane, pol, acc);
+            gather_batch<EPL, DT, SIGN, BAGS, U, false>(a, col, off, live, gbase_s, cnt, p0, lane, acc);
         __syncwarp();  // the staging area is rewritten by the next batch
     }
     if (BAGS) {
@@ -345,17 +331,6 @@ fwd_vec_kernel(FwdArgs a, uint32_t ids_per_batch, uint32_t cmagic) {
         if (lo >= a.nbags) return;
         hi = lo + ids_per_batch < a.nbags ? lo + ids_per_batch : a.nbags;
     }
-    if (BAGS && a.keep_keys != nullptr) {  // (as in the staged kernel)
-        const int64_t C = (int64_t)mp.C;
-        if (warp == 0) {
-            for (int64_t q = lane; q < lo * C; q += 32) a.keep_keys[q] = 0;
-            for (int64_t p = lane; p < lo; p += 32) a.keep_bag_of[p] = 0;
-        }
-        if (warp == a.nbags - 1) {
-            for (int64_t q = hi * C + lane; q < a.nnz * C; q += 32) a.keep_keys[q] = 0;
-            for (int64_t p = hi + lane; p < a.nnz; p += 32) a.keep_bag_of[p] = 0;
-        }
-    }
 
     const uint32_t lpi = mp.d >> 2;   // lanes per id = output vectors per row
     const uint32_t ipi = 32u / lpi;   // ids per load instruction
@@ -403,47 +378,52 @@ static void launch_vec(const FwdArgs& a, bool bags, cudaStream_t st) {
 }
 
 // Ids whose loads are in flight together (U) and resident CTAs per SM the register budget is set
-// for (MINB).  Measured on B200: the time of the HBM-resident gather does not move between 4 and 16
-// ids in flight or between 4 and 8 CTAs per SM - the random 64-byte requests themselves are the
-// limit - so the smallest register footprint is kept.
+// for (MINB, see kStagedCtas*).  Measured on B200: the time of the HBM-resident gather does not move
+// between 4 and 16 ids in flight - the random 64-byte requests themselves are the limit.
 
-template <int EPL, int DT, bool SIGN, bool FULLD>
-static void launch_staged(const FwdArgs& a, bool bags, bool by_table, cudaStream_t st) {
-    constexpr int MINB = (EPL == 4) ? 6 : 8;
+template <int EPL, int DT, bool SIGN, bool FULLD, int MINB>
+static void launch_staged_minb(const FwdArgs& a, bool bags, cudaStream_t st) {
     constexpr int UB = (EPL == 4) ? 2 : 4;
     constexpr int UO = (EPL == 4) ? 2 : 4;
     const uint32_t ipb = staged_ids_per_batch(a.mp, bags, SIGN);
     const uint32_t cmagic = chunk_magic(a.mp);
-    int64_t warps = bags ? a.nbags : (a.nbags + ipb - 1) / ipb;
-    if (by_table) warps = ((a.nbags / a.mp.T + ipb - 1) / ipb) * a.mp.T;
+    const int64_t warps = bags ? a.nbags : (a.nbags + ipb - 1) / ipb;
     const unsigned blocks = (unsigned)((warps + 7) / 8);
     if (bags)
-        fwd_staged_kernel<EPL, DT, SIGN, true, FULLD, MINB, UB><<<blocks, 256, 0, st>>>(a, ipb, cmagic, 0);
+        fwd_staged_kernel<EPL, DT, SIGN, true, FULLD, MINB, UB><<<blocks, 256, 0, st>>>(a, ipb, cmagic);
     else
-        fwd_staged_kernel<EPL, DT, SIGN, false, FULLD, MINB, UO><<<blocks, 256, 0, st>>>(a, ipb, cmagic,
-                                                                                       by_table ? 1 : 0);
+        fwd_staged_kernel<EPL, DT, SIGN, false, FULLD, MINB, UO><<<blocks, 256, 0, st>>>(a, ipb, cmagic);
+}
+
+template <int EPL, int DT, bool SIGN, bool FULLD>
+static void launch_staged(const FwdArgs& a, bool bags, cudaStream_t st) {
+    const bool l2_sized = (uint64_t)a.mp.m * (DT == 0 ? 4u : 2u) <= kL2SizedBytes;
+    if constexpr (SIGN) launch_staged_minb<EPL, DT, SIGN, FULLD, kStagedCtasSign>(a, bags, st);
+    else if constexpr (EPL == 4) launch_staged_minb<EPL, DT, SIGN, FULLD, kStagedCtasWide>(a, bags, st);
+    else if (l2_sized) launch_staged_minb<EPL, DT, SIGN, FULLD, kStagedCtasL2>(a, bags, st);
+    else launch_staged_minb<EPL, DT, SIGN, FULLD, kStagedCtasHbm>(a, bags, st);
 }
 
 template <int EPL, int DT>
-static void launch_staged_flags(const FwdArgs& a, bool bags, bool sign, bool by_table, cudaStream_t st) {
+static void launch_staged_flags(const FwdArgs& a, bool bags, bool sign, cudaStream_t st) {
     const bool fulld = a.mp.d == 32u * EPL;
     if (sign) {  // the sign hash is off in every timed configuration: one generic variant
-        launch_staged<EPL, DT, true, false>(a, bags, by_table, st);
+        launch_staged<EPL, DT, true, false>(a, bags, st);
     } else if (fulld) {
-        launch_staged<EPL, DT, false, true>(a, bags, by_table, st);
+        launch_staged<EPL, DT, false, true>(a, bags, st);
     } else {
-        launch_staged<EPL, DT, false, false>(a, bags, by_table, st);
+        launch_staged<EPL, DT, false, false>(a, bags, st);
     }
 }
 
 template <int DT>
-static void launch_staged_epl(const FwdArgs& a, bool bags, bool sign, bool by_table, cudaStream_t st) {
+static void launch_staged_epl(const FwdArgs& a, bool bags, bool sign, cudaStream_t st) {
     if (a.mp.d <= 32)
-        launch_staged_flags<1, DT>(a, bags, sign, by_table, st);
+        launch_staged_flags<1, DT>(a, bags, sign, st);
     else if (a.mp.d <= 64)
-        launch_staged_flags<2, DT>(a, bags, sign, by_table, st);
+        launch_staged_flags<2, DT>(a, bags, sign, st);
     else
-        launch_staged_flags<4, DT>(a, bags, sign, by_table, st);
+        launch_staged_flags<4, DT>(a, bags, sign, st);
 }
 
 // Lane-hashed kernel for short blocks (Z <= 2 by default; any Z <= d whose lanes can afford to hash
@@ -466,7 +446,6 @@ fwd_lanehash_kernel(FwdArgs a, uint32_t padj) {
     LaneChunks<EPL> lc;
     lc.init(mp, lane, padj);
     const uint32_t m = mp.m;
-    const uint64_t pol = l2_keep_policy(a.l2_keep != 0);
 
     // the loads of U ids (the owned elements of each) are issued together
     auto gather_ids = [&](uint32_t bm, uint64_t thr, uint32_t g0, uint32_t n, float (&v)[U][EPL]) {
@@ -480,7 +459,7 @@ fwd_lanehash_kernel(FwdArgs a, uint32_t padj) {
                 v[gg][u] = 0.0f;
                 if (lc.live[u]) {
                     const uint32_t j = lc.template slot<M30>(u, bm_g, thr_g);
-                    if (ROBE_CHK(j < m, ROBE_DBG_ARRAY_SLOT)) v[gg][u] = gather_elem<DT>(a.array, j, pol);
+                    if (ROBE_CHK(j < m, ROBE_DBG_ARRAY_SLOT)) v[gg][u] = gather_elem<DT>(a.array, j);
                 }
             }
         }
@@ -572,13 +551,14 @@ cudaError_t launch_forward(const Problem& pb, float* out, int variant, cudaStrea
     if (kept != nullptr) *kept = false;
     if (pb.nbags == 0) return cudaSuccess;
     FwdArgs a{pb.mp, pb.array, pb.indices, pb.offsets, out, pb.nbags, pb.nnz, pb.status, keep_keys,
-              keep_bag_of, pb.l2_keep};
+              keep_bag_of};
     const bool bags = pb.offsets != nullptr;
     const bool warp_ok = pb.mp.d <= 128;
     if (variant == 2 && !warp_ok) return cudaErrorInvalidValue;
     if (variant == 3) {  // the kernel with 16-byte loads
         if (!vec_kernel_ok(pb, out)) return cudaErrorInvalidValue;
         if (kept != nullptr) *kept = keep_keys != nullptr;
+        if (bags && keep_keys != nullptr) keep_gaps_kernel<<<8, 256, 0, st>>>(a);
         launch_vec(a, bags, st);
         return cudaGetLastError();
     }
@@ -587,20 +567,19 @@ cudaError_t launch_forward(const Problem& pb, float* out, int variant, cudaStrea
     // (measured on B200, Z = 1 / 2: 1 MB array 2.27 -> 1.72 ms / 1.72 -> 1.00 ms, 100 MB 3.59 -> 3.40 /
     // 2.14 -> 2.09); on a 10 GB array the staged kernel's higher occupancy keeps more DRAM requests
     // in flight and stays ahead (9.5 vs 10.2 ms), so it keeps those.
-    const bool l2_sized = (uint64_t)pb.mp.m * (pb.dtype == 0 ? 4u : 2u) <= (192ull << 20);
+    const bool l2_sized = (uint64_t)pb.mp.m * (pb.dtype == 0 ? 4u : 2u) <= kL2SizedBytes;
     if (variant == 4 || (variant == 0 && pb.mp.Z <= 2 && l2_sized && lanehash_ok(pb) && keep_keys == nullptr)) {
         if (!lanehash_ok(pb)) return cudaErrorInvalidValue;
         if (pb.dtype == 0) launch_lanehash<0>(a, bags, st);
         else launch_lanehash<1>(a, bags, st);
         return cudaGetLastError();
     }
-    if (variant == 5 && (!warp_ok || bags || pb.mp.B != 0 || keep_keys != nullptr)) return cudaErrorInvalidValue;
-    const bool use_warp = variant == 2 || variant == 5 || (variant == 0 && warp_ok);
+    const bool use_warp = variant == 2 || (variant == 0 && warp_ok);
     if (use_warp) {
         if (kept != nullptr) *kept = keep_keys != nullptr;  // (the direct kernel keeps nothing)
-        const bool by_table = variant == 5;
-        if (pb.dtype == 0) launch_staged_epl<0>(a, bags, pb.sign != 0, by_table, st);
-        else launch_staged_epl<1>(a, bags, pb.sign != 0, by_table, st);
+        if (bags && keep_keys != nullptr) keep_gaps_kernel<<<8, 256, 0, st>>>(a);
+        if (pb.dtype == 0) launch_staged_epl<0>(a, bags, pb.sign != 0, st);
+        else launch_staged_epl<1>(a, bags, pb.sign != 0, st);
     } else {
         const unsigned blocks = (unsigned)((pb.nbags + 7) / 8);
         if (pb.dtype == 0) {

@@ -21,6 +21,15 @@ __device__ __forceinline__ void bag_range(const int64_t* offsets, int64_t nnz, i
     }
 }
 
+// Resident CTAs of 256 threads per SM that the staged kernels' register budget is set for.  Rows of up
+// to 64 elements come in two builds: 8 CTAs (32 registers; the kernels then spill 8-24 bytes per
+// thread) for arrays of L2 size, where the gather is bound by L2 latency and the extra warps pay
+// (2-8 % measured on B200), and 6 CTAs (40 registers, no spill) for arrays in HBM, where occupancy buys
+// nothing and the spill traffic costs DRAM bandwidth (cfg 4 forward 0.895 -> 0.864 ms).  Rows of up to
+// 128 elements: 6 CTAs (42 registers).  With the sign hash on: 4 CTAs (it needs the registers).
+constexpr int kStagedCtasL2 = 8, kStagedCtasHbm = 6, kStagedCtasWide = 6, kStagedCtasSign = 4;
+constexpr uint64_t kL2SizedBytes = 192ull << 20;  // arrays up to this size count as "of L2 size"
+
 constexpr int kStageEntries = 256;  // block starts per warp
 constexpr int kStageIds = 64;       // ids per warp batch
 

@@ -59,7 +59,7 @@ def test_create_accepts_limits_and_constants_match_oracle():
 def test_options_and_errors_without_device():
     h = robe.robe_create(4096, 4, 16, 4, 7)
     for key, val in [(robe.ROBE_OPT_SIGN, 2), (robe.ROBE_OPT_BWD_MODE, 5), (99, 0),
-                     (robe.ROBE_OPT_VALIDATE, -1), (robe.ROBE_OPT_FWD_KERNEL, 6), (robe.ROBE_OPT_BWD_KERNEL, 7),
+                     (robe.ROBE_OPT_VALIDATE, -1), (robe.ROBE_OPT_FWD_KERNEL, 5), (robe.ROBE_OPT_BWD_KERNEL, 7),
                      (robe.ROBE_OPT_INDEX_TYPE, 2), (robe.ROBE_OPT_BAG_LAYOUT, 2)]:
         with pytest.raises(robe.RobeError):
             robe.robe_set_option(h, key, val)

@@ -57,12 +57,8 @@ def test_forward_shapes(d, Z, M, bags):
             want = c.oracle_forward()
             warp_ok = d <= 128
             lane_hashed_ok = warp_ok and Z <= d and not sign  # kernel 4: every lane hashes its own chunks
-            by_table_ok = warp_ok and bags is None  # kernel 5: a warp takes the rows of one table
-            for kernel in ([0, 1, 2] if warp_ok else [0, 1]) + ([4] if lane_hashed_ok else []) + ([5] if by_table_ok else []):
+            for kernel in ([0, 1, 2] if warp_ok else [0, 1]) + ([4] if lane_hashed_ok else []):
                 assert_bits_equal(c.forward(kernel).cpu().numpy(), want, f"d={d} Z={Z} M={M} k={kernel}")
-            if not by_table_ok:
-                with pytest.raises(robe.RobeError):
-                    c.forward(5)
             if not warp_ok:
                 with pytest.raises(robe.RobeError):
                     c.forward(2)
