@@ -346,10 +346,10 @@ int robe_forward_keep(robe_handle_t h, const void* indices, const int64_t* offse
     if (((uintptr_t)workspace & 255u) != 0) return ROBE_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
     if (launch_validate(pb, st) != cudaSuccess) return ROBE_ERR_CUDA;
-    uint32_t *keys = nullptr, *bag_of = nullptr;
-    if (nnz > 0 && batch > 0) block_key_buffers(pb, workspace, &keys, &bag_of);
+    uint32_t *keys = nullptr, *vals = nullptr;
+    if (nnz > 0 && batch > 0) block_key_buffers(pb, workspace, &keys, &vals);
     bool kept = false;
-    const int frc = launch_status(launch_forward(pb, out, h->fwd_variant, st, keys, bag_of, &kept));
+    const int frc = launch_status(launch_forward(pb, out, h->fwd_variant, st, keys, vals, &kept));
     if (frc != ROBE_OK) return frc;
     // a forward kernel that keeps nothing (rows longer than 128): the backward's own key kernels
     if (!kept && launch_block_keys(pb, workspace, workspace_bytes, st) != cudaSuccess) return ROBE_ERR_CUDA;

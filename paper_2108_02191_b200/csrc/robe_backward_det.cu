@@ -1,9 +1,9 @@
 // Deterministic backward (Section 3.1 backward equation, evaluated in a fixed order).
 //
 // Blocks are numbered q = p*C + c in input order (p = position in indices, c = chunk).
-//   1. key kernel      key[q] = h(e, x_p, c) (or left by the forward of the same step).  The payload
-//                      val[q] - where the block's gradient elements start in grad_out (sign off) or q
-//                      itself (sign on) - is not stored: the first sort pass derives it from q
+//   1. key kernel      key[q] = h(e, x_p, c); val[q] = where the block's gradient elements
+//                      start in grad_out (sign off) or q itself (sign on); or both left by the
+//                      forward of the same step
 //   2. radix sort      stable LSD sort of (key, val) by key - our own passes: digit count per
 //                      CTA range, per-digit exclusive scan, ranked scatter through shared
 //                      memory (so that every digit's run leaves the CTA as one coalesced piece)
@@ -75,10 +75,12 @@ __global__ void __launch_bounds__(256) det_bag_of_kernel(KeyArgs a, uint32_t* ba
     for (int64_t p = lo + lane; p < hi; p += 32) bag_of[p] = (uint32_t)k;
 }
 
-// key[q] = h(e, x_p, c) for q = p*C + c.
+// key[q] = h(e, x_p, c) for q = p*C + c.  val[q] = q when the sign hash is on (the apply kernel
+// then needs the id again), else the position bag*d + c*Z of the block's first gradient element.
 // One thread per id: the part of the hash that all chunks of the id share is evaluated once.
+template <bool SIGN>
 __global__ void __launch_bounds__(256)
-det_keys_kernel(KeyArgs a, const uint32_t* bag_of, uint32_t* keys) {
+det_keys_kernel(KeyArgs a, const uint32_t* bag_of, uint32_t* keys, uint32_t* vals) {
     const uint64_t p = (uint64_t)blockIdx.x * 256 + threadIdx.x;
     if (p >= (uint64_t)a.nnz) return;
     const MapParams& mp = a.mp;
@@ -88,19 +90,23 @@ det_keys_kernel(KeyArgs a, const uint32_t* bag_of, uint32_t* keys) {
     const uint64_t q0 = p * mp.C;
     if (mp.R > 1) {  // rows clubbed into one block: a single key
         keys[q0] = id_block_start(mp, e, x, 0);
+        vals[q0] = SIGN ? (uint32_t)q0 : (uint32_t)(bag * mp.d);
         return;
     }
     const uint64_t base = hash_base(mp.h, e, x);
     for (uint32_t c = 0; c < mp.C; ++c) {
         if (!ROBE_CHK(q0 + c < (uint64_t)a.nnz * mp.C, ROBE_DBG_SORT_POS)) break;
         keys[q0 + c] = block_start(mp, base, c);
+        vals[q0 + c] = SIGN ? (uint32_t)(q0 + c) : (uint32_t)(bag * mp.d + c * mp.Z);
     }
 }
 
 // The same, one thread per block: for many blocks per id (small Z) the writes of one thread per
 // id would be far apart, and re-evaluating the shared part of the hash per block costs less.
+template <bool SIGN>
 __global__ void __launch_bounds__(256)
-det_keys_by_block_kernel(KeyArgs a, const uint32_t* bag_of, uint32_t* keys, uint64_t nb) {
+det_keys_by_block_kernel(KeyArgs a, const uint32_t* bag_of, uint32_t* keys, uint32_t* vals,
+                         uint64_t nb) {
     const uint64_t q = (uint64_t)blockIdx.x * 256 + threadIdx.x;
     if (q >= nb) return;
     const MapParams& mp = a.mp;
@@ -110,21 +116,9 @@ det_keys_by_block_kernel(KeyArgs a, const uint32_t* bag_of, uint32_t* keys, uint
     const uint32_t e = table_of_bag(bag, mp);
     const uint64_t x = (uint64_t)a.indices.load(p);
     keys[q] = id_block_start(mp, e, x, c);
+    vals[q] = SIGN ? (uint32_t)q : (uint32_t)(bag * mp.d + c * mp.Z);
 }
 
-// The payload of block q = p*C + c, as the first sort pass derives it: q itself when the sign hash
-// is on (the apply kernel then needs the id again), else the position bag*d + c*Z of the block's
-// first gradient element, bag = bag_of[p] (pooled input) or p (one-hot).
-struct PayloadGen {
-    const uint32_t* bag_of;
-    uint32_t C, d, Z, sign;
-    __device__ __forceinline__ uint32_t operator()(uint32_t q) const {
-        if (sign) return q;
-        const uint32_t p = q / C, c = q - p * C;
-        const uint32_t bag = bag_of != nullptr ? __ldg(bag_of + p) : p;
-        return bag * d + c * Z;
-    }
-};
 
 // ---- radix sort pass, kernel 1: digit histogram of each CTA's contiguous key range
 __global__ void __launch_bounds__(kSortThreads)
@@ -197,9 +191,7 @@ __global__ void __launch_bounds__(kSortThreads, 4)
 sort_scatter_kernel(const uint32_t* __restrict__ kin, const uint32_t* __restrict__ vin,
                     uint32_t* __restrict__ kout, uint32_t* __restrict__ vout,
                     const uint32_t* __restrict__ cta_offsets, const uint32_t* __restrict__ totals,
-                    uint64_t nb, uint64_t tiles, uint32_t shift, uint32_t mask, PayloadGen gen) {
-    // vin == nullptr: first pass of a sort, the pairs are still in block order and the payload of
-    // the pair at position q is gen(q)
+                    uint64_t nb, uint64_t tiles, uint32_t shift, uint32_t mask) {
     __shared__ uint32_t skey[kSortTile];
     __shared__ uint32_t sval[kSortTile];
     __shared__ uint32_t wcnt[kSortWarps][kRadix];
@@ -277,8 +269,7 @@ sort_scatter_kernel(const uint32_t* __restrict__ kin, const uint32_t* __restrict
                 const uint32_t lp = dstart[dg] + wcnt[w][dg] + rank[r];
                 if (!ROBE_CHK(lp < (uint32_t)kSortTile, ROBE_DBG_SHARED)) continue;
                 skey[lp] = key[r];
-                // payloads are only passed through: read them this late
-                sval[lp] = vin != nullptr ? vin[idx] : gen((uint32_t)idx);
+                sval[lp] = vin[idx];  // payloads are only passed through: read them this late
             }
         }
         __syncthreads();
@@ -351,9 +342,9 @@ __device__ __forceinline__ bool block_term(const ApplyArgs& a, const uint32_t* b
     const uint32_t i = c * mp.Z + o;
     if (i >= mp.d) return false;
     const uint64_t bag = bag_of ? (uint64_t)__ldg(bag_of + p) : (uint64_t)p;
+    if (!ROBE_CHK(bag * mp.d + i < a.grad_elems, ROBE_DBG_GRAD_POS)) return false;
     const uint32_t e = table_of_bag(bag, mp);
     const uint64_t x = (uint64_t)a.indices.load(p);
-    if (!ROBE_CHK(bag * mp.d + i < a.grad_elems, ROBE_DBG_GRAD_POS)) return false;
     term = sign_of(mp, hash_base(mp.g, e, x), i) * __ldg(a.grad_out + bag * mp.d + i);
     return true;
 }
@@ -1199,12 +1190,11 @@ size_t det_workspace_bytes(const MapParams& mp, int64_t nbags, int64_t nnz, bool
     return make_layout(nb, nnz, bags, mp.m).total;
 }
 
-void block_key_buffers(const Problem& pb, void* workspace, uint32_t** keys, uint32_t** bag_of) {
+void block_key_buffers(const Problem& pb, void* workspace, uint32_t** keys, uint32_t** vals) {
     const uint64_t nb = (uint64_t)pb.nnz * pb.mp.C;
-    const bool bags = pb.offsets != nullptr;
-    const Layout L = make_layout(nb, pb.nnz, bags, pb.mp.m);
+    const Layout L = make_layout(nb, pb.nnz, pb.offsets != nullptr, pb.mp.m);
     *keys = (uint32_t*)((char*)workspace + L.keysA);
-    *bag_of = bags ? (uint32_t*)((char*)workspace + L.bag_of) : nullptr;
+    *vals = (uint32_t*)((char*)workspace + L.valsA);
 }
 
 // bag_of (pooled input) into the workspace
@@ -1226,13 +1216,18 @@ cudaError_t launch_block_keys(const Problem& pb, void* workspace, size_t workspa
     if (workspace == nullptr || workspace_bytes < L.total) return cudaErrorInvalidValue;
     char* ws = (char*)workspace;
     uint32_t* kA = (uint32_t*)(ws + L.keysA);
+    uint32_t* vA = (uint32_t*)(ws + L.valsA);
     uint32_t* bag_of = bags ? (uint32_t*)(ws + L.bag_of) : nullptr;
     KeyArgs ka{mp, pb.indices, pb.offsets, pb.nbags, pb.nnz, pb.status};
     if (bags) launch_bag_of(pb, L, ws, st);
     if (mp.C <= 8) {
-        det_keys_kernel<<<(unsigned)((pb.nnz + 255) / 256), 256, 0, st>>>(ka, bag_of, kA);
+        const unsigned kb = (unsigned)((pb.nnz + 255) / 256);
+        if (pb.sign) det_keys_kernel<true><<<kb, 256, 0, st>>>(ka, bag_of, kA, vA);
+        else det_keys_kernel<false><<<kb, 256, 0, st>>>(ka, bag_of, kA, vA);
     } else {
-        det_keys_by_block_kernel<<<(unsigned)((nb + 255) / 256), 256, 0, st>>>(ka, bag_of, kA, nb);
+        const unsigned kb = (unsigned)((nb + 255) / 256);
+        if (pb.sign) det_keys_by_block_kernel<true><<<kb, 256, 0, st>>>(ka, bag_of, kA, vA, nb);
+        else det_keys_by_block_kernel<false><<<kb, 256, 0, st>>>(ka, bag_of, kA, vA, nb);
     }
     return cudaGetLastError();
 }
@@ -1257,11 +1252,12 @@ cudaError_t launch_backward_det(const Problem& pb, const float* grad_out, float*
     uint32_t* counts = (uint32_t*)(ws + L.counts);
     uint32_t* totals = (uint32_t*)(ws + L.totals);
 
-    if (!keys_kept) {  // (else the forward of the step left the block starts and the bags of the ids)
+    if (!keys_kept) {
         const cudaError_t err = launch_block_keys(pb, workspace, workspace_bytes, st);
         if (err != cudaSuccess) return err;
+    } else if (bags && pb.sign) {
+        launch_bag_of(pb, L, ws, st);  // the signed terms look the id's bag up again
     }
-    const PayloadGen gen{bag_of, mp.C, mp.d, mp.Z, pb.sign ? 1u : 0u};
 
     const SortPlan sp = make_plan(nb);
     const uint32_t bits = bits_for(mp.m);
@@ -1274,8 +1270,8 @@ cudaError_t launch_backward_det(const Problem& pb, const float* grad_out, float*
         const uint32_t mask = (1u << (bits - shift)) - 1u;
         sort_count_kernel<<<sp.grid, kSortThreads, 0, st>>>(kA, counts, nb, sp.tiles, shift, mask);
         sort_scan_kernel<<<kRadix, kSortThreads, 0, st>>>(counts, totals, sp.grid);
-        sort_scatter_kernel<false><<<sp.grid, kSortThreads, 0, st>>>(kA, nullptr, kB, vB, counts, totals, nb,
-                                                                    sp.tiles, shift, mask, gen);
+        sort_scatter_kernel<false><<<sp.grid, kSortThreads, 0, st>>>(kA, vA, kB, vB, counts, totals, nb,
+                                                                    sp.tiles, shift, mask);
         ApplyArgs ab{mp, grad_out, pb.indices, target, lr, nb, pb.status, AdamState{}, nullptr, nullptr, 0,
                      nullptr, nullptr, 0, (uint64_t)pb.nbags * mp.d, pb.l2_keep};
         uint32_t log2Zp = 0;
@@ -1300,8 +1296,8 @@ cudaError_t launch_backward_det(const Problem& pb, const float* grad_out, float*
         const uint32_t mask = (1u << width) - 1u;
         sort_count_kernel<<<sp.grid, kSortThreads, 0, st>>>(kA, counts, nb, sp.tiles, shift, mask);
         sort_scan_kernel<<<kRadix, kSortThreads, 0, st>>>(counts, totals, sp.grid);
-        sort_scatter_kernel<true><<<sp.grid, kSortThreads, 0, st>>>(kA, pass == 0 ? nullptr : vA, kB, vB, counts,
-                                                                   totals, nb, sp.tiles, shift, mask, gen);
+        sort_scatter_kernel<true><<<sp.grid, kSortThreads, 0, st>>>(kA, vA, kB, vB, counts, totals, nb,
+                                                                   sp.tiles, shift, mask);
         uint32_t* t = kA; kA = kB; kB = t;
         t = vA; vA = vB; vB = t;
     }

@@ -22,8 +22,8 @@ struct FwdArgs {
     int64_t nbags;
     int64_t nnz;
     const int32_t* status;
-    uint32_t* keep_keys;    // block starts kept for the backward, or nullptr
-    uint32_t* keep_bag_of;  // with them, pooled input: the bag of every id position
+    uint32_t* keep_keys;  // block starts and payloads kept for the backward, or nullptr
+    uint32_t* keep_vals;
 };
 
 // Kept block starts, pooled input: id positions before the first bag or after the last one (offsets
@@ -37,10 +37,8 @@ __global__ void __launch_bounds__(256) keep_gaps_kernel(FwdArgs a) {
     bag_range(a.offsets, a.nnz, a.nbags - 1, lo_last, hi_last);
     const int64_t C = (int64_t)a.mp.C;
     const int64_t step = (int64_t)gridDim.x * 256, t0 = (int64_t)blockIdx.x * 256 + threadIdx.x;
-    for (int64_t q = t0; q < lo * C; q += step) a.keep_keys[q] = 0;
-    for (int64_t p = t0; p < lo; p += step) a.keep_bag_of[p] = 0;
-    for (int64_t q = hi_last * C + t0; q < a.nnz * C; q += step) a.keep_keys[q] = 0;
-    for (int64_t p = hi_last + t0; p < a.nnz; p += step) a.keep_bag_of[p] = 0;
+    for (int64_t q = t0; q < lo * C; q += step) a.keep_keys[q] = a.keep_vals[q] = 0;
+    for (int64_t q = hi_last * C + t0; q < a.nnz * C; q += step) a.keep_keys[q] = a.keep_vals[q] = 0;
 }
 
 template <int DT, bool SIGN>
@@ -210,7 +208,7 @@ fwd_staged_kernel(FwdArgs a, uint32_t ids_per_batch, uint32_t cmagic) {
                                                                             : (int64_t)ids_per_batch);
         const bool wraps = stage_batch<SIGN, BAGS>(sm, mp, a.indices, p0, cnt, ids_per_batch, tterm,
                                                    gterm, cmagic, w, lane,
-                                                   KeepBlocks{a.keep_keys, a.keep_bag_of, (uint64_t)warp, (uint64_t)a.nnz * mp.C});
+                                                   KeepBlocks{a.keep_keys, a.keep_vals, (uint64_t)warp, (uint64_t)a.nnz * mp.C});
         if (wraps)
             gather_batch<EPL, DT, SIGN, BAGS, U, true>(a, col, off, live, gbase_s, cnt, p0, lane, acc);
         else
@@ -347,7 +345,7 @@ fwd_vec_kernel(FwdArgs a, uint32_t ids_per_batch, uint32_t cmagic) {
                                                                             : (int64_t)ids_per_batch);
         const bool wraps = stage_batch<false, BAGS>(sm, mp, a.indices, p0, cnt, ids_per_batch, tterm, 0,
                                                     cmagic, w, lane,
-                                                    KeepBlocks{a.keep_keys, a.keep_bag_of, (uint64_t)warp, (uint64_t)a.nnz * mp.C});
+                                                    KeepBlocks{a.keep_keys, a.keep_vals, (uint64_t)warp, (uint64_t)a.nnz * mp.C});
         if (wraps)
             vec_gather_batch<BAGS, true, U>(a, col, o, cnt, p0, lpi, ipi, grp, k, lane_on, acc);
         else
@@ -547,11 +545,11 @@ static void launch_lanehash(const FwdArgs& a, bool bags, cudaStream_t st) {
 }
 
 cudaError_t launch_forward(const Problem& pb, float* out, int variant, cudaStream_t st,
-                           uint32_t* keep_keys, uint32_t* keep_bag_of, bool* kept) {
+                           uint32_t* keep_keys, uint32_t* keep_vals, bool* kept) {
     if (kept != nullptr) *kept = false;
     if (pb.nbags == 0) return cudaSuccess;
     FwdArgs a{pb.mp, pb.array, pb.indices, pb.offsets, out, pb.nbags, pb.nnz, pb.status, keep_keys,
-              keep_bag_of};
+              keep_vals};
     const bool bags = pb.offsets != nullptr;
     const bool warp_ok = pb.mp.d <= 128;
     if (variant == 2 && !warp_ok) return cudaErrorInvalidValue;

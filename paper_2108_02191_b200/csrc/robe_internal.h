@@ -26,11 +26,11 @@ struct Problem {
     cudaEvent_t join_event = nullptr;
 };
 
-// forward: out [nbags, d].  With keep_keys (device, one word per block) and, for pooled input,
-// keep_bag_of (one word per id) the staged kernel also stores every block's start and every id's bag
-// as the sort-based backward wants them; *kept says whether the kernel that ran did so.
+// forward: out [nbags, d].  With keep_keys/keep_vals (device, one word per block each) the staged
+// kernel also stores every block's start and payload as the sort-based backward wants them;
+// *kept says whether the kernel that ran did so.
 cudaError_t launch_forward(const Problem& pb, float* out, int variant, cudaStream_t st,
-                           uint32_t* keep_keys = nullptr, uint32_t* keep_bag_of = nullptr,
+                           uint32_t* keep_keys = nullptr, uint32_t* keep_vals = nullptr,
                            bool* kept = nullptr);
 
 // atomic backward: adds scale * g * grad_out into target (fp32 [M])
@@ -51,15 +51,14 @@ struct AdamState {
 // mode 0: target[j] += delta; 1: target = attached array, target[j] = fma(-lr, delta, target[j]);
 // 2: Adam step on the attached array with the moments in *adam; 3: binned atomic adds of
 // lr * delta terms into target (one sort pass on the top key bits, then red.global in bin order)
-// keys_kept: the workspace already holds the block starts (and, pooled input, the bags of the id
-// positions) of these ids, left by launch_forward or launch_block_keys: not computed again.
+// keys_kept: the workspace already holds the block starts and payloads of these ids (left by
+// launch_forward or launch_block_keys), so they are not computed again.
 cudaError_t launch_backward_det(const Problem& pb, const float* grad_out, float* target, int mode,
                                 float lr, const AdamState* adam, void* workspace,
                                 size_t workspace_bytes, cudaStream_t st, bool keys_kept = false);
-// where in a workspace of the sort-based backward the block starts and the bags of the id positions
-// (nullptr for one-hot input) go
-void block_key_buffers(const Problem& pb, void* workspace, uint32_t** keys, uint32_t** bag_of);
-// block starts (and bags of the id positions) of pb's ids into the workspace (what the backward does first)
+// where in a workspace of the sort-based backward the block starts and payloads go
+void block_key_buffers(const Problem& pb, void* workspace, uint32_t** keys, uint32_t** vals);
+// block starts and payloads of pb's ids into the workspace (what the backward does first)
 cudaError_t launch_block_keys(const Problem& pb, void* workspace, size_t workspace_bytes,
                               cudaStream_t st);
 

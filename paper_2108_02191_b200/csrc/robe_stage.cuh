@@ -68,12 +68,15 @@ __device__ __forceinline__ void stage_init(StageSmem& sm, const MapParams& mp) {
 }
 
 // Where the hash phase also leaves the block starts for a later sort-based backward of the same
-// ids: keys[q] = h(e, x_p, c) for block q = p*C + c and, for pooled input, bag_of[p] = the bag of
-// id position p (one word per id; the backward derives every block's payload from q and that).
-// keys == nullptr: not kept.  `bag` is the warp's bag in pooled mode (one-hot: row p is bag p).
+// ids: keys[q] = h(e, x_p, c) and vals[q] for block q = p*C + c, vals[q] = q when the sign hash is
+// on, else the position bag*d + c*Z of the block's first gradient element.  keys == nullptr: not
+// kept.  `bag` is the warp's bag in pooled mode (one-hot: row p is bag p).
+// (Storing the starts alone and deriving the payloads in the first sort pass - from q and one bag
+// word per id - was measured: it saves 0.1 GB of writes per cfg 4 step and 8 us in the forward, and
+// costs 50-60 us in the scatter pass, which is bound by latency and instruction issue, not by bytes.)
 struct KeepBlocks {
     uint32_t* keys;
-    uint32_t* bag_of;
+    uint32_t* vals;
     uint64_t bag;
     uint64_t nb;  // number of blocks of the call (read by the debug build's index check only)
 };
@@ -112,7 +115,6 @@ __device__ __forceinline__ bool stage_batch(StageSmem& sm, const MapParams& mp,
         }
         if (!ROBE_CHK(t < (uint32_t)(SIGN ? kStageIds / 2 : kStageIds), ROBE_DBG_SHARED)) continue;
         base_s[t] = addmod_p61(tt, mulmod_p61_any(mp.h.B, xh));
-        if (BAGS && keep.keys != nullptr) keep.bag_of[p0 + t] = (uint32_t)keep.bag;
         if (SIGN) gbase_s[t] = addmod_p61(gt, mulmod_p61_any(mp.g.B, x));
     }
     __syncwarp();
@@ -131,7 +133,10 @@ __device__ __forceinline__ bool stage_batch(StageSmem& sm, const MapParams& mp,
         wraps |= s > last_fit;
         if (keep.keys != nullptr &&
             ROBE_CHK((uint64_t)p0 * mp.C + t < keep.nb, ROBE_DBG_SORT_POS)) {  // consecutive lanes, consecutive words
-            keep.keys[(uint64_t)p0 * mp.C + t] = s;
+            const uint64_t q = (uint64_t)p0 * mp.C + t;
+            const uint64_t bag = BAGS ? keep.bag : (uint64_t)p0 + idl;
+            keep.keys[q] = s;
+            keep.vals[q] = SIGN ? (uint32_t)q : (uint32_t)(bag * mp.d + c * mp.Z);
         }
     }
     const bool any = __any_sync(0xFFFFFFFFu, wraps);
