@@ -43,6 +43,20 @@ UNIT = "ids/s"
 # Records go stale when a kernel changes: they are re-captured with the kernel, never edited.
 NCU_TRAFFIC_RECORDS = {
     # (workload, backward variant, block starts shared, id type, bag layout)
+    ("cfg4_multihot", "binned", True, "int64", "sample-major"): {
+        "forward": 4_412_000_000, "backward": 4_838_700_000,
+        "source": "profiles/launches_cfg4_multihot.md: full-size one-pass ncu capture of `python bench.py --steps 3 "
+                  "--warmup 3 --no-cpu-baseline`; forward = fwd_staged_kernel, backward = sort_count + sort_scan + "
+                  "sort_scatter + binned_apply"},
+    ("cfg4_multihot", "atomic", False, "int64", "sample-major"): {
+        "forward": 4_130_800_000, "backward": 7_378_600_000,
+        "source": "profiles/launches_cfg4_multihot.md: full-size one-pass ncu capture of `python bench.py --steps 3 "
+                  "--warmup 3 --no-cpu-baseline --backward atomic`"},
+    ("cfg4_multihot", "det", True, "int64", "sample-major"): {
+        "forward": 4_411_800_000, "backward": 7_246_000_000,
+        "source": "profiles/launches_cfg4_multihot.md: full-size one-pass ncu capture of `python bench.py --steps 3 "
+                  "--warmup 3 --no-cpu-baseline --backward det`; backward = 4 sort passes, window bounds and classes, "
+                  "apply kernels"},
 }
 
 
@@ -509,7 +523,8 @@ def run_ours(args, w):
     # a traffic record applies to the configuration it was captured on, and to no other
     own_batch = args.batch == 0
     rec = NCU_TRAFFIC_RECORDS.get((w.name, args.backward, bool(share_keys), args.ids, args.bag_layout)) \
-        if (own_batch and not dp_step and world == 1 and args.fwd_kernel == 0 and args.bwd_kernel == 0) else None
+        if (own_batch and not dp_step and world == 1 and args.fwd_kernel == 0 and args.bwd_kernel == 0
+            and args.l2_keep == 0) else None
     sm_mhz = clocks.get("sm_mhz")
 
     def roof(nbytes, ms, kernel, which):
@@ -572,7 +587,10 @@ def run_ours(args, w):
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
                 "ids": "int32" if e2e_id_bytes == 4 else "int64",
                 "ms_per_step": e2e_ms / e2e_steps},
-        "gpu_launches": (1 + bwd_launches + (1 if dp_step else 0)) * args.steps,
+        # forward kernel (+ the gap-fill kernel beside it when block starts of pooled input are kept),
+        # the backward's kernels, the dense apply of the data-parallel step
+        "gpu_launches": (1 + (1 if (share_keys and bags and d <= 128) else 0) + bwd_launches
+                         + (1 if dp_step else 0)) * args.steps,
         # ONE kernel: the forward gather (the largest single kernel of the step by the ncu launch
         # list under profiles/, and the kernel the >= 0.60 target is stated for)
         "roofline": roof(fwd_bytes, fwd_ms, fwd_kernel, "forward"),
