@@ -280,6 +280,25 @@ int robe_backward_adam(robe_handle_t h, const float* grad_out, const void* indic
                        size_t workspace_bytes, void* stream);
 
 /*
+ * robe_backward_adagrad - deterministic backward with the Adagrad step fused in (Duchi, Hazan, Singer,
+ * "Adaptive subgradient methods ..."; the optimizer recommendation models are commonly trained with,
+ * beside the SGD and Adam of the paper's Section 5).  Embedding tables usually keep ONE accumulator
+ * per row ("row-wise Adagrad"); the ROBE array has no rows - a slot is shared by elements of many
+ * rows of many tables - so the accumulator is per slot.  For every array slot j that receives at
+ * least one gradient term, with delta[j] summed in the deterministic order of robe_backward:
+ *     sum_sq[j] = sum_sq[j] + delta[j]^2
+ *     M[j]      = M[j] - lr * delta[j] / (sqrt(sum_sq[j]) + eps)
+ * each operation a separate round-to-nearest fp32 one; other slots keep M and sum_sq.  Bit-reproducible.
+ *   sum_sq   device pointer, fp32 [M], caller-owned, zeroed by the caller before the first step.
+ *   workspace / workspace_bytes  as for robe_backward in deterministic mode.
+ * The handle's ROBE_OPT_BWD_MODE is not consulted.  The attached array must be fp32.
+ * Errors: as robe_backward; ROBE_ERR_INVALID_ARG also for a null sum_sq or eps < 0.
+ */
+int robe_backward_adagrad(robe_handle_t h, const float* grad_out, const void* indices,
+                          const int64_t* offsets, int64_t batch, int64_t nnz, float* sum_sq, float lr,
+                          float eps, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * robe_apply_sgd - the dense SGD apply of a data-parallel training step (Section 1 of the
  * paper, implications of the compression: the whole model fits every GPU, so training is plain
  * data-parallel and the ranks exchange one gradient the size of the array; Section 5: SGD).

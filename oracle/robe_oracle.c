@@ -353,6 +353,25 @@ void robe_oracle_accumulate(float *grad_array, const float *delta, const uint8_t
         if (touched[j]) grad_array[j] = grad_array[j] + delta[j];
 }
 
+/* Adagrad step (Duchi, Hazan, Singer) on the slots that received at least one term, in fp32, one
+   operation at a time, one accumulator per slot:
+     s <- s + g^2;  M <- M - lr g / (sqrt(s) + eps)
+   Slots without a term keep M and s. */
+void robe_oracle_adagrad_apply(float *array, float *sum_sq, const float *delta, const uint8_t *touched,
+                               uint64_t n, float lr, float eps) {
+    for (uint64_t j = 0; j < n; ++j) {
+        if (!touched[j]) continue;
+        float g = delta[j];
+        float gg = g * g;
+        float s = sum_sq[j] + gg;
+        sum_sq[j] = s;
+        float den = sqrtf(s) + eps;
+        float upd = g / den;
+        float step = lr * upd;
+        array[j] = array[j] - step;
+    }
+}
+
 /* Adam step (Kingma & Ba, Algorithm 1; Section 5 trains five of the six models with Adam) on
    the slots that received at least one term, in fp32, one operation at a time:
      m1 <- beta1 m1 + (1-beta1) g;  m2 <- beta2 m2 + (1-beta2) g^2

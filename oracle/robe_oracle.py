@@ -59,6 +59,7 @@ def lib() -> C.CDLL:
         _lib.robe_oracle_accumulate.argtypes = [p, p, p, u64]
         _lib.robe_oracle_dense_sgd_apply.argtypes = [p, p, u64, C.c_float]
         _lib.robe_oracle_adam_apply.argtypes = [p, p, p, p, p, u64] + [C.c_float] * 6
+        _lib.robe_oracle_adagrad_apply.argtypes = [p, p, p, p, u64, C.c_float, C.c_float]
     return _lib
 
 
@@ -186,6 +187,14 @@ def accumulate(grad_array, delta, touched) -> None:
     """In place: grad_array[j] = grad_array[j] + delta[j] on touched slots."""
     assert grad_array.dtype == np.float32 and delta.dtype == np.float32
     lib().robe_oracle_accumulate(_ptr(grad_array), _ptr(delta), _ptr(touched), len(delta))
+
+
+def adagrad_apply(array, sum_sq, delta, touched, lr, eps) -> None:
+    """In place: one Adagrad step (one accumulator per slot) on the touched slots."""
+    for a in (array, sum_sq, delta):
+        assert a.dtype == np.float32
+    lib().robe_oracle_adagrad_apply(_ptr(array), _ptr(sum_sq), _ptr(delta), _ptr(touched), len(delta),
+                                    C.c_float(lr), C.c_float(eps))
 
 
 def adam_bias(beta: float, step: int) -> np.float32:

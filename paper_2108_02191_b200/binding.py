@@ -55,7 +55,7 @@ EXPORTS = [
     "robe_set_status_word", "robe_last_device_status", "robe_status_string",
     "robe_backward_deterministic_static", "robe_backward_adam",
     "robe_forward_keep", "robe_backward_kept", "robe_apply_sgd",
-    "robe_debug_status", "robe_debug_selftest",
+    "robe_debug_status", "robe_debug_selftest", "robe_backward_adagrad",
 ]
 
 if not os.path.exists(LIB_PATH):
@@ -81,6 +81,8 @@ _lib.robe_backward_deterministic_static.argtypes = [_vp, _vp, _vp, _vp, _i64, _i
 _lib.robe_backward_adam.argtypes = [_vp, _vp, _vp, _vp, _i64, _i64, _vp, _vp, C.c_float, C.c_float,
                                     C.c_float, C.c_float, _i64, _vp, C.c_size_t, _vp]
 _lib.robe_apply_sgd.argtypes = [_vp, _vp, C.c_float, C.c_int, _vp]
+_lib.robe_backward_adagrad.argtypes = [_vp, _vp, _vp, _vp, _i64, _i64, _vp, C.c_float, C.c_float, _vp,
+                                       C.c_size_t, _vp]
 _lib.robe_debug_status.argtypes = [_vp]
 _lib.robe_debug_selftest.argtypes = [_vp]
 _lib.robe_set_status_word.argtypes = [_vp, _vp]
@@ -233,6 +235,16 @@ def robe_backward_adam(h, grad_out, indices, offsets, batch: int, m1, m2, lr: fl
         h, _dev_ptr(grad_out, torch.float32), _ids_ptr(indices), _dev_ptr(offsets, torch.int64), batch,
         indices.numel(), _dev_ptr(m1, torch.float32), _dev_ptr(m2, torch.float32), lr, beta1, beta2, eps,
         step, _dev_ptr(workspace), ws_bytes, _stream_ptr(stream)), "robe_backward_adam")
+
+
+def robe_backward_adagrad(h, grad_out, indices, offsets, batch: int, sum_sq, lr: float, eps: float,
+                          workspace, stream=None) -> None:
+    _state_index_type(h, indices)
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(_lib.robe_backward_adagrad(
+        h, _dev_ptr(grad_out, torch.float32), _ids_ptr(indices), _dev_ptr(offsets, torch.int64), batch,
+        indices.numel(), _dev_ptr(sum_sq, torch.float32), lr, eps, _dev_ptr(workspace), ws_bytes,
+        _stream_ptr(stream)), "robe_backward_adagrad")
 
 
 def robe_apply_sgd(h, grad_array, lr: float, zero_grad: bool = True, stream=None) -> None:

@@ -497,6 +497,32 @@ int robe_backward_adam(robe_handle_t h, const float* grad_out, const void* indic
     return ROBE_OK;
 }
 
+int robe_backward_adagrad(robe_handle_t h, const float* grad_out, const void* indices,
+                          const int64_t* offsets, int64_t batch, int64_t nnz, float* sum_sq, float lr,
+                          float eps, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!check_sizes(h, indices, offsets, batch, nnz)) return ROBE_ERR_INVALID_ARG;
+    if (batch > 0 && grad_out == nullptr) return ROBE_ERR_INVALID_ARG;
+    if (sum_sq == nullptr || !(eps >= 0.0f)) return ROBE_ERR_INVALID_ARG;
+    if (h->validate && h->status_word == nullptr) return ROBE_ERR_INVALID_ARG;
+    if (h->array == nullptr) return ROBE_ERR_NO_ARRAY;
+    if (h->dtype != ROBE_F32) return ROBE_ERR_INVALID_ARG;
+    Problem pb = make_problem(h, indices, offsets, batch, nnz);
+    if (!sorted_path_fits(h, pb)) return ROBE_ERR_UNSUPPORTED;
+    const size_t need = det_workspace_bytes(h->mp, pb.nbags, nnz, offsets != nullptr);
+    if (nnz > 0 && (workspace == nullptr || workspace_bytes < need)) return ROBE_ERR_WORKSPACE;
+    if (((uintptr_t)workspace & 255u) != 0) return ROBE_ERR_WORKSPACE;
+    lend_side_stream(h, pb);
+    AdamState ad{};
+    ad.m2 = sum_sq;
+    ad.eps = eps;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (launch_validate(pb, st) != cudaSuccess) return ROBE_ERR_CUDA;
+    if (launch_backward_det(pb, grad_out, (float*)h->array, 4, lr, &ad, workspace, workspace_bytes, st) !=
+        cudaSuccess)
+        return ROBE_ERR_CUDA;
+    return ROBE_OK;
+}
+
 int robe_apply_sgd(robe_handle_t h, float* grad_array, float lr, int zero_grad, void* stream) {
     if (h == nullptr || grad_array == nullptr) return ROBE_ERR_INVALID_ARG;
     if (zero_grad != 0 && zero_grad != 1) return ROBE_ERR_INVALID_ARG;

@@ -350,7 +350,7 @@ __device__ __forceinline__ bool block_term(const ApplyArgs& a, const uint32_t* b
 }
 
 // What a served slot does with its sum delta (MODE): 0 - add it to a dense gradient; 1 - the
-// SGD step M[j] = fma(-lr, delta, M[j]); 2 - the Adam step (Kingma & Ba, Algorithm 1; the paper
+// SGD step M[j] = fma(-lr, delta, M[j]); 3 - the Adagrad step; 2 - the Adam step (Kingma & Ba, Algorithm 1; the paper
 // trains five of its six models with Adam, Section 5) on the slot and its two moment slots, every
 // operation a separate correctly rounded fp32 one.  `old` is target[j].
 template <int MODE>
@@ -360,6 +360,13 @@ __device__ __forceinline__ void commit_slot(const ApplyArgs& a, uint32_t j, floa
         a.target[j] = __fadd_rn(old, delta);
     } else if (MODE == 1) {
         a.target[j] = __fmaf_rn(-a.lr, delta, old);
+    } else if (MODE == 3) {
+        // Adagrad (Duchi, Hazan, Singer): one accumulator of squared gradients per slot
+        const AdamState& ad = a.adam;  // m2 = the accumulators, eps
+        const float s = __fadd_rn(ad.m2[j], __fmul_rn(delta, delta));
+        ad.m2[j] = s;
+        const float den = __fadd_rn(__fsqrt_rn(s), ad.eps);
+        a.target[j] = __fsub_rn(old, __fmul_rn(a.lr, __fdiv_rn(delta, den)));
     } else {
         const AdamState& ad = a.adam;
         const float m = __fadd_rn(__fmul_rn(ad.beta1, ad.m1[j]), __fmul_rn(__fsub_rn(1.0f, ad.beta1), delta));
@@ -1312,11 +1319,13 @@ cudaError_t launch_backward_det(const Problem& pb, const float* grad_out, float*
                            (uint8_t*)(ws + L.win_left), L.nwin, L.win_log2,
                            pb.side, pb.fork_event, pb.join_event};
     if (pb.sign) {
-        if (mode == 2) launch_apply<true, 2>(aa, kA, vA, bag_of, wb, st);
+        if (mode == 4) launch_apply<true, 3>(aa, kA, vA, bag_of, wb, st);
+        else if (mode == 2) launch_apply<true, 2>(aa, kA, vA, bag_of, wb, st);
         else if (mode == 1) launch_apply<true, 1>(aa, kA, vA, bag_of, wb, st);
         else launch_apply<true, 0>(aa, kA, vA, bag_of, wb, st);
     } else {
-        if (mode == 2) launch_apply<false, 2>(aa, kA, vA, bag_of, wb, st);
+        if (mode == 4) launch_apply<false, 3>(aa, kA, vA, bag_of, wb, st);
+        else if (mode == 2) launch_apply<false, 2>(aa, kA, vA, bag_of, wb, st);
         else if (mode == 1) launch_apply<false, 1>(aa, kA, vA, bag_of, wb, st);
         else launch_apply<false, 0>(aa, kA, vA, bag_of, wb, st);
     }

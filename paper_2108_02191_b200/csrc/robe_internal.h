@@ -49,7 +49,8 @@ struct AdamState {
 };
 
 // mode 0: target[j] += delta; 1: target = attached array, target[j] = fma(-lr, delta, target[j]);
-// 2: Adam step on the attached array with the moments in *adam; 3: binned atomic adds of
+// 2: Adam step on the attached array with the moments in *adam; 4: Adagrad step on the attached
+// array with the accumulators in adam->m2 and adam->eps; 3: binned atomic adds of
 // lr * delta terms into target (one sort pass on the top key bits, then red.global in bin order)
 // keys_kept: the workspace already holds the block starts and payloads of these ids (left by
 // launch_forward or launch_block_keys), so they are not computed again.

@@ -46,7 +46,7 @@ def test_shape_lists_run_clean_on_the_index_check_build():
     if os.environ.get("ROBE_LIBRARY"):
         pytest.skip("already inside the child run")
     pick = ("forward_shapes or backward_shapes or window_apply or step_sharing or vector_kernel or "
-            "lane_hashed or adam or table_major or int32 or cfg1 or hot_id or bit_reproducible")
+            "lane_hashed or adam or adagrad or merged_rows or table_major or int32 or cfg1 or hot_id or bit_reproducible")
     r = subprocess.run([sys.executable, "-m", "pytest", "tests/test_gpu_parity.py", "tests/test_zz_no_alloc.py",
                         "-m", "gpu", "-x", "-q", "-k", pick + " or two_calls or fused_sgd"],
                        env=_debug_env(), cwd=ROOT, capture_output=True, text=True, timeout=3000)

@@ -380,6 +380,34 @@ def test_backward_adam_matches_oracle_over_steps(bags):
                 robe.robe_backward_adam(c.h, g_d, c.indices, c.offsets, c.B, m1_d, m2_d, lr, b1, b2, eps, 0, ws)
 
 
+@pytest.mark.parametrize("bags", [None, (3, 0, 9)])
+def test_backward_adagrad_matches_oracle_over_steps(bags):
+    # three Adagrad steps in a row (array and accumulators carried over), bit for bit; the dense
+    # window apply, the position-tile apply and rows clubbed into one block
+    lr, eps = 0.05, 1e-8
+    for w in (synth.workload(1).with_(bag_rule=bags), small(d=64, Z=16, M=70, bag_rule=bags, batch=200),
+              small(d=16, Z=64, M=1000, bag_rule=bags, batch=97, vocab_arg=(3, 7, 1000)),
+              small(d=32, Z=8, M=300_007, bag_rule=bags, batch=40)):
+        with Case(w) as c:
+            robe.robe_set_option(c.h, robe.ROBE_OPT_BWD_MODE, robe.ROBE_BWD_DETERMINISTIC)
+            ws = torch.empty(robe.robe_backward_workspace_bytes(c.h, c.B, c.indices.numel()),
+                             dtype=torch.uint8, device=c.dev)
+            ssq_d = torch.zeros(w.M, device=c.dev)
+            arr, ssq = c.array_h.copy(), np.zeros(w.M, np.float32)
+            for step in (1, 2, 3):
+                g_h, g_d = _grad(c, 30 + step)
+                can, touched = c.oracle.backward_canonical(g_h, c.indices_h, c.offsets_h, c.B)
+                orc.adagrad_apply(arr, ssq, can, touched, lr, eps)
+                robe.robe_backward_adagrad(c.h, g_d, c.indices, c.offsets, c.B, ssq_d, lr, eps, ws)
+                torch.cuda.synchronize()
+                assert_bits_equal(c.array.cpu().numpy(), arr, f"adagrad array, step {step}")
+                assert_bits_equal(ssq_d.cpu().numpy(), ssq, f"adagrad accumulators, step {step}")
+            with pytest.raises(robe.RobeError):
+                robe.robe_backward_adagrad(c.h, g_d, c.indices, c.offsets, c.B, ssq_d, lr, -1.0, ws)
+            with pytest.raises(robe.RobeError):
+                robe.robe_backward_adagrad(c.h, g_d, c.indices, c.offsets, c.B, None, lr, eps, ws)
+
+
 def test_deterministic_is_bit_reproducible_and_order_sensitive_case():
     # a hot id: thousands of terms on the same slots; five runs must give identical bits
     w = small(d=32, Z=8, M=300, batch=2000, vocab_arg=(2, 3, 1000))

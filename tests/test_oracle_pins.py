@@ -599,6 +599,38 @@ def test_sgd_apply_and_accumulate():
     np.testing.assert_array_equal(g, np.array([1.5, 1.0, 8.0, 1.0], dtype=np.float32))
 
 
+def test_adagrad_apply_hand_computed_and_torch():
+    # Adagrad (Duchi et al.): s <- s + g^2, theta <- theta - lr g / (sqrt(s) + eps).  Powers of two make
+    # the first step exact: g = eps = 2^-3, s = 2^-6, sqrt(s) + eps = 2^-2, update 1/2, theta = 1 - lr/2;
+    # second step with the same g: s = 2^-5, no longer exact, closed form to rounding.
+    g = np.float32(0.125)
+    arr = np.array([1.0, 1.0, -3.0], np.float32)
+    ssq = np.zeros(3, np.float32)
+    delta = np.array([g, -g, 0.5], np.float32)
+    touched = np.array([1, 1, 0], np.uint8)
+    orc.adagrad_apply(arr, ssq, delta, touched, 0.25, float(g))
+    np.testing.assert_array_equal(arr, np.array([0.875, 1.125, -3.0], np.float32))
+    np.testing.assert_array_equal(ssq, np.array([g * g, g * g, 0.0], np.float32))
+    orc.adagrad_apply(arr, ssq, delta, touched, 0.25, float(g))
+    want = 0.875 - 0.25 * 0.125 / (np.sqrt(2.0 ** -5) + 0.125)
+    assert abs(float(arr[0]) - want) < 1e-7 and arr[2] == -3.0 and ssq[2] == 0.0
+    # a library routine: torch.optim.Adagrad (no decay), all slots touched, several steps
+    import torch
+    rng = np.random.default_rng(12)
+    n, lr, eps = 1000, 0.05, 1e-10
+    arr = rng.standard_normal(n).astype(np.float32)
+    ssq = np.zeros(n, np.float32)
+    p_ = torch.nn.Parameter(torch.from_numpy(arr.copy()))
+    opt = torch.optim.Adagrad([p_], lr=lr, eps=eps)
+    ones = np.ones(n, np.uint8)
+    for _ in range(5):
+        gr = rng.standard_normal(n).astype(np.float32)
+        orc.adagrad_apply(arr, ssq, gr, ones, lr, eps)
+        p_.grad = torch.from_numpy(gr.copy())
+        opt.step()
+        np.testing.assert_allclose(arr, p_.detach().numpy(), rtol=0, atol=5e-7)
+
+
 def test_dense_sgd_apply_hand_values_and_agreement_with_the_fused_step():
     # data-parallel step: every slot gets fma(-lr, g, M); hand values (exact in fp32)
     arr = np.array([1.0, 2.0, 3.0, -0.0, 0.5], dtype=np.float32)
