@@ -373,7 +373,6 @@ bwd_atomic_lanehash_kernel(BwdArgs a, uint32_t padj) {
 
     LaneChunks<EPL> lc;
     lc.init(mp, lane, padj);
-    const uint32_t m = mp.m;
     const uint64_t pol = l2_keep_policy(a.l2_keep != 0);
     const int64_t nwarps = (int64_t)gridDim.x * 8;
     const int64_t gw = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
@@ -385,7 +384,7 @@ bwd_atomic_lanehash_kernel(BwdArgs a, uint32_t padj) {
         for (int u = 0; u < EPL; ++u)
             if (lc.live[u]) {
                 const uint32_t j = lc.template slot<M30>(u, bm_g, thr_g);
-                if (ROBE_CHK(j < m, ROBE_DBG_ARRAY_SLOT)) red_add(a.target + j, gv[u], pol);
+                if (ROBE_CHK(j < mp.m, ROBE_DBG_ARRAY_SLOT)) red_add(a.target + j, gv[u], pol);
             }
     };
 

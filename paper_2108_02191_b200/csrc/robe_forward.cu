@@ -443,7 +443,6 @@ fwd_lanehash_kernel(FwdArgs a, uint32_t padj) {
 
     LaneChunks<EPL> lc;
     lc.init(mp, lane, padj);
-    const uint32_t m = mp.m;
 
     // the loads of U ids (the owned elements of each) are issued together
     auto gather_ids = [&](uint32_t bm, uint64_t thr, uint32_t g0, uint32_t n, float (&v)[U][EPL]) {
@@ -457,7 +456,7 @@ fwd_lanehash_kernel(FwdArgs a, uint32_t padj) {
                 v[gg][u] = 0.0f;
                 if (lc.live[u]) {
                     const uint32_t j = lc.template slot<M30>(u, bm_g, thr_g);
-                    if (ROBE_CHK(j < m, ROBE_DBG_ARRAY_SLOT)) v[gg][u] = gather_elem<DT>(a.array, j);
+                    if (ROBE_CHK(j < mp.m, ROBE_DBG_ARRAY_SLOT)) v[gg][u] = gather_elem<DT>(a.array, j);
                 }
             }
         }
