@@ -99,26 +99,59 @@ def forward_byte_models(w, nbags, nnz, bags, id_bytes=8):
 
 
 class ClockSampler:
-    """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
+    """SM clock and throttle-reason samples taken while the timed region runs.
+
+    Reads (never sets) the clocks: through NVML in a background thread, every 2 ms, so that even a
+    40 ms timed region yields a dozen samples; if NVML cannot be loaded, through `nvidia-smi -lms`,
+    whose loop delivers a sample every 10-15 ms.  stop(window) keeps the samples taken inside the
+    timed region (the sampler is started before the warm-up so that it is delivering by then)."""
 
     Q = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
          "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
-    PERIOD_MS = 10
+    PERIOD_S = 0.002
 
     def __init__(self, gpu_index: int):
         self.gpu = gpu_index
         self.proc = None
         self.path = None
+        self.thread = None
+        self.samples = []   # (time.time(), sm_mhz, reasons bit mask)
+        self.max_mhz = None
+        self._stop = False
+
+    def _nvml_loop(self, nvml, handle):
+        reasons_of = getattr(nvml, "nvmlDeviceGetCurrentClocksEventReasons", None) or \
+            nvml.nvmlDeviceGetCurrentClocksThrottleReasons
+        while not self._stop:
+            try:
+                mhz = nvml.nvmlDeviceGetClockInfo(handle, nvml.NVML_CLOCK_SM)
+                mask = reasons_of(handle)
+                self.samples.append((time.time(), float(mhz), int(mask)))
+            except Exception:
+                pass
+            time.sleep(self.PERIOD_S)
 
     def start(self):
+        try:
+            import threading
+
+            import pynvml as nvml
+            nvml.nvmlInit()
+            handle = nvml.nvmlDeviceGetHandleByIndex(self.gpu)
+            self.max_mhz = float(nvml.nvmlDeviceGetMaxClockInfo(handle, nvml.NVML_CLOCK_SM))
+            self.nvml = nvml
+            self.thread = threading.Thread(target=self._nvml_loop, args=(nvml, handle), daemon=True)
+            self.thread.start()
+            return
+        except Exception:
+            self.thread = None
         try:
             fd, self.path = tempfile.mkstemp(suffix=".csv")
             os.close(fd)
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms",
-                 str(self.PERIOD_MS), "-i", str(self.gpu)], stdout=open(self.path, "w"),
-                stderr=subprocess.DEVNULL)
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "10",
+                 "-i", str(self.gpu)], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
@@ -129,10 +162,27 @@ class ClockSampler:
         return datetime.datetime.strptime(text, "%Y/%m/%d %H:%M:%S.%f").timestamp()
 
     def stop(self, window=None):
-        """Stops sampling.  window = (t0, t1) in time.time() seconds keeps only the samples taken
-        inside the timed region (the sampler itself is started before the warm-up so that it is
-        already delivering when the region begins)."""
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        if self.thread is not None:
+            self._stop = True
+            self.thread.join(timeout=2)
+            nvml = self.nvml
+            names = {"hw_slowdown": "HwSlowdown", "hw_thermal_slowdown": "HwThermalSlowdown",
+                     "sw_thermal_slowdown": "SwThermalSlowdown", "sw_power_cap": "SwPowerCap"}
+            bits = {k: getattr(nvml, "nvmlClocksEventReason" + v, None) or getattr(nvml, "nvmlClocksThrottleReason" + v)
+                    for k, v in names.items()}
+            kept = [smp for smp in self.samples if window is None or window[0] <= smp[0] <= window[1]]
+            if kept:
+                out["sm_mhz"] = float(np.median([smp[1] for smp in kept]))
+                out["sm_max_mhz"] = self.max_mhz
+                out["samples"] = len(kept)
+                out["reasons"] = sorted(k for k, bit in bits.items() if any(smp[2] & bit for smp in kept))
+            out["source"] = "nvml"
+            try:
+                nvml.nvmlShutdown()
+            except Exception:
+                pass
+            return out
         if self.proc is None:
             return out
         self.proc.terminate()
@@ -167,6 +217,7 @@ class ClockSampler:
             out["sm_max_mhz"] = float(max(mx))
             out["samples"] = len(sm)
         out["reasons"] = sorted(reasons)
+        out["source"] = "nvidia-smi"
         return out
 
 
