@@ -127,3 +127,50 @@ def test_sort_based_variants_refuse_sizes_beyond_their_32_bit_numbering():
     assert lib.robe_backward(h, dummy, dummy, None, big, big - 1, dummy, 0.0, None, 0, None) \
         == robe.ROBE_ERR_INVALID_ARG
     robe.robe_destroy(h)
+
+
+def test_header_is_plain_c_and_cpp(tmp_path):
+    # the boundary is a C ABI: the header must compile as C11 and as C++ with nothing but itself
+    import subprocess
+    inc = os.path.join(ROOT, "include")
+    for comp, std, ext in (("gcc", "-std=c11", "c"), ("g++", "-std=c++11", "cpp")):
+        src = tmp_path / f"use_robe.{ext}"
+        src.write_text('#include "robe.h"\nint main(void) { robe_handle_t h = 0; return robe_destroy(h) == ROBE_OK; }\n')
+        r = subprocess.run([comp, std, "-Wall", "-Wextra", "-Werror", "-pedantic", "-fsyntax-only", "-I", inc, str(src)],
+                           capture_output=True, text=True)
+        assert r.returncode == 0, r.stderr
+
+
+C_PROGRAM = r"""
+#include <stdio.h>
+#include <string.h>
+#include "robe.h"
+int main(void) {
+    robe_handle_t h = 0;
+    uint64_t k[9];
+    if (robe_create(&h, 4096, 4, 16, 4, 7) != ROBE_OK) return 1;
+    if (robe_get_hash_constants(h, k) != ROBE_OK || k[0] != ((1ull << 61) - 1)) return 2;
+    if (robe_set_option(h, ROBE_OPT_SIGN, 1) != ROBE_OK) return 3;
+    if (robe_forward(h, (const void*)0x1000, 0, 2, 8, (float*)0x1000, 0) != ROBE_ERR_NO_ARRAY) return 4;
+    if (robe_create(&h, 10, 12, 4, 1, 7) != ROBE_ERR_INVALID_ARG) return 5;  /* Z > d, not a multiple */
+    if (strcmp(robe_status_string(ROBE_ERR_WORKSPACE), "workspace missing, misaligned or too small") != 0) return 6;
+    printf("%llu\n", (unsigned long long)k[1]);
+    return 0;
+}
+"""
+
+
+def test_c_program_links_and_calls_the_library(tmp_path):
+    # a C caller, not ctypes: compile against include/robe.h, link librobe.so, run the host-only calls
+    import subprocess
+    src = tmp_path / "caller.c"
+    src.write_text(C_PROGRAM)
+    exe = tmp_path / "caller"
+    lib_dir = os.path.dirname(robe.LIB_PATH)
+    r = subprocess.run(["gcc", "-std=c11", "-Wall", "-Werror", "-I", os.path.join(ROOT, "include"), str(src), "-o",
+                        str(exe), "-L", lib_dir, "-l:" + os.path.basename(robe.LIB_PATH), "-Wl,-rpath," + lib_dir],
+                       capture_output=True, text=True)
+    assert r.returncode == 0, r.stderr
+    r = subprocess.run([str(exe)], capture_output=True, text=True, timeout=120)
+    assert r.returncode == 0, (r.returncode, r.stderr)
+    assert int(r.stdout.strip()) == int(orc.hash_constants(7)[1])  # A_h as the oracle draws it

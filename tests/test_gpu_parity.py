@@ -104,6 +104,24 @@ def test_forward_vector_kernel_refuses_what_it_cannot_do():
             c.forward(3)
 
 
+def test_two_handles_of_different_dimension_share_one_array():
+    # Section 3.1, multiple embedding tables: tables of different embedding size live in the same array.
+    # One handle per dimension, both attached to the same device array; a fused SGD step through one
+    # handle is what the other one reads afterwards.
+    wa = small(d=16, Z=4, M=5003, hash_seed=11)
+    wb = small(d=48, Z=16, M=5003, hash_seed=12, num_tables=2, vocab_arg=(300, 9), bag_rule=(3, 0, 9))
+    with Case(wa) as a, Case(wb, array=a.array) as b:
+        assert b.array.data_ptr() == a.array.data_ptr()
+        assert_bits_equal(a.forward().cpu().numpy(), a.oracle_forward(), "handle A")
+        assert_bits_equal(b.forward().cpu().numpy(), b.oracle_forward(), "handle B")
+        g_h, g_d = _grad(a, 9)
+        can, touched = a.oracle.backward_canonical(g_h, a.indices_h, a.offsets_h, a.B)
+        a.backward(g_d, "det", sgd=True, lr=0.5)
+        orc.sgd_apply(b.array_h, can, touched, 0.5)   # the oracle twin of the shared array
+        assert_bits_equal(b.array.cpu().numpy(), b.array_h, "shared array after A's step")
+        assert_bits_equal(b.forward().cpu().numpy(), b.oracle_forward(), "handle B reads A's update")
+
+
 def test_forward_bf16_array():
     w = small(array_dtype="bf16", d=64, Z=16, M=5000, bag_rule=(4, 0, 12))
     with Case(w) as c:
